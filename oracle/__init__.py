@@ -1,0 +1,15 @@
+"""fp64 CPU oracle of the EmbedPart hot path -- TEST INFRASTRUCTURE, not the product.
+
+Only ``tests/``, the smoke check and the CPU-baseline leg of ``bench.py`` may
+import this package.  It never imports the CUDA package and the CUDA package
+never imports it.
+"""
+from .ep_oracle import (  # noqa: F401
+    build,
+    kmeans,
+    assign_step,
+    partition_quality,
+    reorder,
+    num_threads,
+    set_num_threads,
+)

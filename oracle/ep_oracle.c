@@ -1,0 +1,212 @@
+/*
+ * ep_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, fp64 CPU statement of what the EmbedPart hot path computes:
+ *   - Lloyd K-Means over dense node embeddings  (Algorithm 3, line 1: P <- KMeans(E, k))
+ *   - edge cut and per-partition loads           (Section 2.1.1, Eq. 1 and Eq. 2)
+ *   - the partition-ordered vertex permutation   (Section 4.5.1, "Adapting EmbedPart for Reordering")
+ *
+ * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call
+ * this file.  It shares no code, header, table or helper with the CUDA library
+ * and the CUDA library never calls it.
+ *
+ * Every function is pinned by CPU tests (brute force over all labelings, hand-
+ * computed fixtures, closed forms, invariants, library special cases); none is
+ * "parity unpinned".
+ *
+ * Arithmetic: every floating-point operation is IEEE double.  Embeddings and
+ * initial centroids arrive as fp32 and are widened exactly.  Counters are 64-bit.
+ * OpenMP, where used, only splits loops whose iterations are independent (or an
+ * integer sum), so the result does not depend on the thread count.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/*
+ * Assignment step of Lloyd's algorithm: every row goes to the centroid with the
+ * smallest squared Euclidean distance, written in the direct form
+ * sum_j (x_ij - c_kj)^2.  Centroids are scanned k = 0..K-1 with a strict '<',
+ * so of several equidistant centroids the lowest index wins.
+ *
+ * best1[i] / best2[i] (either may be NULL) receive the smallest and the second
+ * smallest distance of row i (best2 = +inf when K == 1); tests use them to find
+ * rows whose two nearest centroids are too close to call in fp32.
+ */
+void oracle_assign(const float *emb, int64_t N, int32_t d,
+                   const double *C, int32_t K,
+                   int32_t *assign, double *best1, double *best2)
+{
+    int64_t i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < N; ++i) {
+        const float *x = emb + i * (int64_t)d;
+        double m1 = INFINITY, m2 = INFINITY;
+        int32_t a = 0;
+        for (int32_t k = 0; k < K; ++k) {
+            const double *c = C + (int64_t)k * d;
+            double dist = 0.0;
+            for (int32_t j = 0; j < d; ++j) {
+                double diff = (double)x[j] - c[j];
+                dist += diff * diff;
+            }
+            if (dist < m1) {
+                m2 = m1;
+                m1 = dist;
+                a = k;
+            } else if (dist < m2) {
+                m2 = dist;
+            }
+        }
+        assign[i] = a;
+        if (best1) best1[i] = m1;
+        if (best2) best2[i] = m2;
+    }
+}
+
+/*
+ * Lloyd K-Means, exactly `iters` iterations, no early stop (Algorithm 3 line 1
+ * under the reading: squared Euclidean distance, explicit initial centroids,
+ * full batch).
+ *
+ *   C_0 = init
+ *   for t = 1..T:
+ *       a_i  = argmin_k |x_i - C_{t-1}[k]|^2          (oracle_assign)
+ *       J_t  = sum_i |x_i - C_{t-1}[a_i]|^2
+ *       C_t[k] = mean of the rows with a_i = k, or C_{t-1}[k] when no row has a_i = k
+ *
+ * Returns the assignment of iteration T (made against C_{T-1}) together with
+ * C_T, so every non-empty centroid is exactly the mean of the rows that carry
+ * its label.  With iters == 0 the rows are assigned against C_0, centroids =
+ * C_0 and objective[0] = the objective of that assignment.
+ *
+ * objective: max(iters,1) doubles, or NULL.  best1/best2: per-row two smallest
+ * distances of the returned assignment, or NULL.
+ * Returns 0, or -1 when scratch memory cannot be had.
+ */
+int oracle_kmeans(const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                  const float *init_centroids,
+                  int32_t *assign, double *centroids, double *objective,
+                  double *best1, double *best2)
+{
+    int64_t KD = (int64_t)K * d;
+    double *prev = (double *)malloc(sizeof(double) * (size_t)KD);
+    double *sum = (double *)malloc(sizeof(double) * (size_t)KD);
+    int64_t *cnt = (int64_t *)malloc(sizeof(int64_t) * (size_t)K);
+    double *m1 = best1 ? best1 : (double *)malloc(sizeof(double) * (size_t)N);
+    if (!prev || !sum || !cnt || !m1) {
+        free(prev); free(sum); free(cnt);
+        if (!best1) free(m1);
+        return -1;
+    }
+    for (int64_t q = 0; q < KD; ++q) centroids[q] = (double)init_centroids[q];
+
+    int32_t T = iters > 0 ? iters : 1;
+    for (int32_t t = 0; t < T; ++t) {
+        memcpy(prev, centroids, sizeof(double) * (size_t)KD);
+        oracle_assign(emb, N, d, prev, K, assign, m1, best2);
+
+        double J = 0.0;
+        for (int64_t i = 0; i < N; ++i) J += m1[i];
+        if (objective) objective[t] = J;
+        if (iters == 0) break;
+
+        memset(sum, 0, sizeof(double) * (size_t)KD);
+        memset(cnt, 0, sizeof(int64_t) * (size_t)K);
+        for (int64_t i = 0; i < N; ++i) {
+            int32_t a = assign[i];
+            const float *x = emb + i * (int64_t)d;
+            double *s = sum + (int64_t)a * d;
+            for (int32_t j = 0; j < d; ++j) s[j] += (double)x[j];
+            cnt[a] += 1;
+        }
+        for (int32_t k = 0; k < K; ++k) {
+            if (cnt[k] > 0) {
+                for (int32_t j = 0; j < d; ++j)
+                    centroids[(int64_t)k * d + j] = sum[(int64_t)k * d + j] / (double)cnt[k];
+            } /* an empty cluster keeps its previous centroid */
+        }
+    }
+    free(prev); free(sum); free(cnt);
+    if (!best1) free(m1);
+    return 0;
+}
+
+/*
+ * Edge cut and partition loads (Eq. 1 numerator; the operands of Eq. 2).
+ *
+ *   edge_cut         = number of stored CSR entries (u -> v) with pid(u) != pid(v)
+ *   part_vertices[p] = |{v : pid(v) = p}|
+ *   part_edges[p]    = sum of the out-degrees of the vertices in p
+ *
+ * Entries are counted as stored: a symmetric CSR counts an undirected cut edge
+ * twice, a self-loop is never cut, a duplicate entry counts each time.
+ */
+void oracle_partition_quality(const int64_t *rowptr, const int32_t *colidx,
+                              const int32_t *assign, int64_t N, int32_t K,
+                              uint64_t *edge_cut, int64_t *part_vertices, int64_t *part_edges)
+{
+    int64_t cut = 0;
+    int64_t u;
+#pragma omp parallel for schedule(dynamic, 4096) reduction(+ : cut)
+    for (u = 0; u < N; ++u) {
+        int32_t pu = assign[u];
+        for (int64_t e = rowptr[u]; e < rowptr[u + 1]; ++e)
+            if (assign[colidx[e]] != pu) cut += 1;
+    }
+    *edge_cut = (uint64_t)cut;
+
+    for (int32_t p = 0; p < K; ++p) { part_vertices[p] = 0; part_edges[p] = 0; }
+    for (int64_t v = 0; v < N; ++v) {
+        part_vertices[assign[v]] += 1;
+        part_edges[assign[v]] += rowptr[v + 1] - rowptr[v];
+    }
+}
+
+/*
+ * Partition-ordered relabelling (Section 4.5.1): vertices of the same partition
+ * get consecutive new ids.  Partitions come in ascending order and, inside a
+ * partition, vertices keep their original order, i.e. perm lists the vertex ids
+ * sorted by the pair (pid(v), v).  Written as a stable counting sort.
+ *
+ *   perm[new_id]   = old vertex id
+ *   inv_perm[v]    = new id of vertex v        (the paper's pi; may be NULL)
+ * Returns 0, or -1 when scratch memory cannot be had.
+ */
+int oracle_reorder(const int32_t *assign, int64_t N, int32_t K,
+                   int32_t *perm, int32_t *inv_perm)
+{
+    int64_t *next = (int64_t *)calloc((size_t)K + 1, sizeof(int64_t));
+    if (!next) return -1;
+    for (int64_t v = 0; v < N; ++v) next[assign[v] + 1] += 1;
+    for (int32_t p = 0; p < K; ++p) next[p + 1] += next[p];   /* next[p] = first new id of partition p */
+    for (int64_t v = 0; v < N; ++v) {
+        int64_t pos = next[assign[v]]++;
+        perm[pos] = (int32_t)v;
+        if (inv_perm) inv_perm[v] = (int32_t)pos;
+    }
+    free(next);
+    return 0;
+}

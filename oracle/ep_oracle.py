@@ -1,0 +1,155 @@
+"""ctypes wrapper around ``ep_oracle.c`` (numpy in, numpy out).
+
+TEST INFRASTRUCTURE.  The C file holds all of the arithmetic; this module only
+compiles it with gcc and marshals arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import NamedTuple, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ep_oracle.c")
+_LIB = os.path.join(_HERE, "libep_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP on) and return the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True, capture_output=True, text=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        p = ctypes.c_void_p
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
+        lib.oracle_assign.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, ctypes.c_int32, p, p, p]
+        lib.oracle_assign.restype = None
+        lib.oracle_kmeans.argtypes = [p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                      p, p, p, p, p, p]
+        lib.oracle_kmeans.restype = ctypes.c_int
+        lib.oracle_partition_quality.argtypes = [p, p, p, ctypes.c_int64, ctypes.c_int32, p, p, p]
+        lib.oracle_partition_quality.restype = None
+        lib.oracle_reorder.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, p]
+        lib.oracle_reorder.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().oracle_set_num_threads(int(n))
+
+
+def _f32_matrix(a, name: str) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    if a.ndim != 2:
+        raise ValueError(f"{name} must be 2-D")
+    return a
+
+
+def _labels(a, n: int, K: int) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    if a.shape != (n,):
+        raise ValueError("assign must have one entry per vertex")
+    if n and (a.min() < 0 or a.max() >= K):
+        raise ValueError("assign value outside [0, K)")
+    return a
+
+
+class KMeansResult(NamedTuple):
+    assign: np.ndarray      # int32 [N]
+    centroids: np.ndarray   # float64 [K, d]
+    objective: np.ndarray   # float64 [max(iters, 1)]
+    best1: np.ndarray       # float64 [N]  smallest distance of the returned assignment
+    best2: np.ndarray       # float64 [N]  second smallest (inf when K == 1)
+
+
+def kmeans(emb, K: int, iters: int, init_centroids) -> KMeansResult:
+    emb = _f32_matrix(emb, "emb")
+    init = _f32_matrix(init_centroids, "init_centroids")
+    N, d = emb.shape
+    if init.shape != (K, d):
+        raise ValueError("init_centroids must be K x d")
+    if iters < 0 or K < 1 or N < 1:
+        raise ValueError("bad K / iters / N")
+    assign = np.empty(N, np.int32)
+    cent = np.empty((K, d), np.float64)
+    obj = np.empty(max(iters, 1), np.float64)
+    b1 = np.empty(N, np.float64)
+    b2 = np.empty(N, np.float64)
+    rc = _load().oracle_kmeans(_ptr(emb), N, d, K, iters, _ptr(init), _ptr(assign), _ptr(cent),
+                               _ptr(obj), _ptr(b1), _ptr(b2))
+    if rc != 0:
+        raise MemoryError("oracle_kmeans")
+    return KMeansResult(assign, cent, obj, b1, b2)
+
+
+def assign_step(emb, centroids):
+    """One assignment step against fp64 centroids: (assign, best1, best2)."""
+    emb = _f32_matrix(emb, "emb")
+    C = np.ascontiguousarray(centroids, dtype=np.float64)
+    N, d = emb.shape
+    K = C.shape[0]
+    if C.shape != (K, d):
+        raise ValueError("centroids must be K x d")
+    assign = np.empty(N, np.int32)
+    b1 = np.empty(N, np.float64)
+    b2 = np.empty(N, np.float64)
+    _load().oracle_assign(_ptr(emb), N, d, _ptr(C), K, _ptr(assign), _ptr(b1), _ptr(b2))
+    return assign, b1, b2
+
+
+class QualityResult(NamedTuple):
+    edge_cut: int
+    part_vertices: np.ndarray  # int64 [K]
+    part_edges: np.ndarray     # int64 [K]
+
+
+def partition_quality(rowptr, colidx, assign, K: int) -> QualityResult:
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    N = rowptr.shape[0] - 1
+    assign = _labels(assign, N, K)
+    if rowptr[0] != 0 or rowptr[-1] != colidx.shape[0] or np.any(np.diff(rowptr) < 0):
+        raise ValueError("rowptr is not a CSR row pointer for colidx")
+    if colidx.size and (colidx.min() < 0 or colidx.max() >= N):
+        raise ValueError("colidx value outside [0, N)")
+    cut = ctypes.c_uint64(0)
+    pv = np.empty(K, np.int64)
+    pe = np.empty(K, np.int64)
+    _load().oracle_partition_quality(_ptr(rowptr), _ptr(colidx), _ptr(assign), N, K,
+                                     ctypes.addressof(cut), _ptr(pv), _ptr(pe))
+    return QualityResult(int(cut.value), pv, pe)
+
+
+def reorder(assign, K: int):
+    """(perm, inv_perm): perm[new_id] = old id, inv_perm[old id] = new id."""
+    assign = np.ascontiguousarray(assign, dtype=np.int32)
+    N = assign.shape[0]
+    assign = _labels(assign, N, K)
+    perm = np.empty(N, np.int32)
+    inv = np.empty(N, np.int32)
+    rc = _load().oracle_reorder(_ptr(assign), N, K, _ptr(perm), _ptr(inv))
+    if rc != 0:
+        raise MemoryError("oracle_reorder")
+    return perm, inv

@@ -1,0 +1,142 @@
+"""Pins for the oracle's edge cut / partition loads and reordering (CPU only)."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _cases():
+    with open(os.path.join(GOLDEN, "edge_cut_hand_cases.json")) as f:
+        return json.load(f)["cases"]
+
+
+@pytest.mark.parametrize("case", _cases(), ids=lambda c: c["name"][:40])
+def test_hand_counted_graphs(case):
+    q = oracle.partition_quality(case["rowptr"], case["colidx"], case["assign"], case["K"])
+    assert q.edge_cut == case["edge_cut"]
+    assert q.part_vertices.tolist() == case["part_vertices"]
+    assert q.part_edges.tolist() == case["part_edges"]
+
+
+def _random_csr(rng, N, p, symmetric=True, loops=False):
+    A = rng.random((N, N)) < p
+    if symmetric:
+        A = A | A.T
+    if not loops:
+        np.fill_diagonal(A, False)
+    rowptr = np.concatenate([[0], np.cumsum(A.sum(1))]).astype(np.int64)
+    colidx = np.nonzero(A)[1].astype(np.int32)
+    return A, rowptr, colidx
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_brute_force_dense_adjacency(seed):
+    rng = np.random.default_rng(seed)
+    N, K = int(rng.integers(2, 11)), int(rng.integers(1, 5))
+    A, rowptr, colidx = _random_csr(rng, N, 0.4, symmetric=bool(seed % 2), loops=True)
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    cut = sum(1 for u in range(N) for v in range(N) if A[u, v] and assign[u] != assign[v])
+    q = oracle.partition_quality(rowptr, colidx, assign, K)
+    assert q.edge_cut == cut
+    assert q.part_vertices.tolist() == [int((assign == p).sum()) for p in range(K)]
+    assert q.part_edges.tolist() == [int(A[assign == p].sum()) for p in range(K)]
+
+
+def test_closed_forms_and_ranges():
+    rng = np.random.default_rng(42)
+    N = 300
+    A, rowptr, colidx = _random_csr(rng, N, 0.05, symmetric=True, loops=True)
+    nnz = len(colidx)
+    loops = int(np.trace(A))
+    assert loops > 0
+    same = oracle.partition_quality(rowptr, colidx, np.zeros(N, np.int32), 3)
+    assert same.edge_cut == 0 and same.part_vertices.tolist() == [N, 0, 0] and same.part_edges.tolist() == [nnz, 0, 0]
+    # balance = max/mean = K when one partition holds everything (Eq. 2)
+    assert same.part_vertices.max() / (N / 3) == 3
+    alone = oracle.partition_quality(rowptr, colidx, np.arange(N, dtype=np.int32), N)
+    assert alone.edge_cut == nnz - loops                   # every entry but the self-loops is cut
+    mod = oracle.partition_quality(rowptr, colidx, (np.arange(N) % 4).astype(np.int32), 4)
+    assert mod.part_vertices.tolist() == [75] * 4          # balance exactly 1 when K divides N
+    assert mod.part_vertices.max() / (N / 4) == 1
+    assert 0 <= mod.edge_cut <= nnz and mod.edge_cut % 2 == 0     # symmetric graph: cut entries pair up
+    assert mod.part_vertices.sum() == N and mod.part_edges.sum() == nnz
+
+
+def test_library_special_case_scipy():
+    sp = pytest.importorskip("scipy.sparse")
+    rng = np.random.default_rng(3)
+    N, K = 500, 7
+    _, rowptr, colidx = _random_csr(rng, N, 0.03)
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    M = sp.csr_matrix((np.ones(len(colidx)), colidx, rowptr), shape=(N, N))
+    onehot = sp.csr_matrix((np.ones(N), (np.arange(N), assign)), shape=(N, K))
+    block = (onehot.T @ M @ onehot).toarray()              # block[p, q] = entries from p to q
+    q = oracle.partition_quality(rowptr, colidx, assign, K)
+    assert q.edge_cut == int(block.sum() - np.trace(block))
+    assert q.part_edges.tolist() == block.sum(1).astype(int).tolist()
+
+
+def test_random_assignment_cuts_about_one_minus_one_over_k():
+    """Statistical sanity: a uniform random partition cuts a fraction 1 - sum (n_p/N)^2 of the entries."""
+    rng = np.random.default_rng(4)
+    N, K = 2000, 8
+    _, rowptr, colidx = _random_csr(rng, N, 0.02)
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    q = oracle.partition_quality(rowptr, colidx, assign, K)
+    expect = 1 - ((q.part_vertices / N) ** 2).sum()
+    assert abs(q.edge_cut / len(colidx) - expect) < 0.01
+
+
+def test_rejects_bad_inputs():
+    with pytest.raises(ValueError):
+        oracle.partition_quality([0, 1], [0], [2], 2)
+    with pytest.raises(ValueError):
+        oracle.partition_quality([0, 1], [5], [0], 2)
+    with pytest.raises(ValueError):
+        oracle.reorder([0, 3], 3)
+
+
+# ---------------------------------------------------------------------------------------------- reorder
+@pytest.mark.parametrize("seed", range(8))
+def test_reorder_equals_sorting_by_label_then_id(seed):
+    rng = np.random.default_rng(seed)
+    N, K = int(rng.integers(1, 200)), int(rng.integers(1, 12))
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    perm, inv = oracle.reorder(assign, K)
+    assert perm.tolist() == sorted(range(N), key=lambda v: (int(assign[v]), v))
+    np.testing.assert_array_equal(perm, np.argsort(assign, kind="stable"))
+    assert sorted(perm.tolist()) == list(range(N))                       # bijection
+    np.testing.assert_array_equal(inv[perm], np.arange(N))
+    np.testing.assert_array_equal(perm[inv], np.arange(N))
+
+
+def test_reorder_brute_force_definition():
+    # "vertices of the same partition get consecutive ids": walk partitions in order, vertices in order
+    assign = np.array([2, 0, 2, 1, 0, 2, 1, 1, 0, 3], np.int32)
+    want = [v for p in range(5) for v in range(len(assign)) if assign[v] == p]
+    perm, inv = oracle.reorder(assign, 5)
+    assert perm.tolist() == want == [1, 4, 8, 3, 6, 7, 0, 2, 5, 9]
+    assert inv.tolist() == [6, 0, 7, 3, 1, 8, 4, 5, 2, 9]
+
+
+def test_reorder_structure_on_a_larger_case():
+    rng = np.random.default_rng(77)
+    N, K = 50_000, 300
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    assign[assign == 17] = 18                                            # an empty partition
+    perm, inv = oracle.reorder(assign, K)
+    lab = assign[perm]
+    assert np.all(np.diff(lab) >= 0)                                     # grouped, ascending partitions
+    same = np.diff(lab) == 0
+    assert np.all(np.diff(perm)[same] > 0)                               # original order inside a partition
+    counts = np.bincount(assign, minlength=K)
+    starts = np.concatenate([[0], np.cumsum(counts)[:-1]])
+    for p in (0, 16, 18, K - 1):
+        seg = perm[starts[p]: starts[p] + counts[p]]
+        assert np.all(assign[seg] == p)
+    assert counts[17] == 0

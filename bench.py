@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the EmbedPart hot path on B200.
+
+A "step" is one pass of the whole hot path over one synthetic workload held in HBM:
+  ep_kmeans (K partitions)  [+ ep_kmeans (reorder_K clusters) when the workload has a reordering run]
+  -> ep_partition_quality on the K-partition labels -> ep_reorder on the finest labels.
+value = embedding rows x Lloyd iterations per second over the timed steps (whole job, all ranks).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl ours|reference]
+
+N > 1 is launched by torch.distributed.run; the path needs no exchange between GPUs here, so every
+rank runs an independent replica of the workload ("replicas only", weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio used to derive the TF32 roof from the bf16 one
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax = float(f[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------ workload
+def describe(w):
+    s = f"{w.name}: N={w.N} d={w.d} K={w.K} x{w.iters} iters"
+    if w.reorder_K:
+        s += f" + K={w.reorder_K} x{w.reorder_iters} iters (reordering run)"
+    return s
+
+
+def make_device_inputs(w, device):
+    rowptr, colidx = synth.graph(w, device=device)
+    torch.cuda.empty_cache()
+    emb = synth.embeddings(w, device=device)
+    rows = synth.init_centroid_rows(w, max(w.K, w.reorder_K), device=device)
+    init = emb[rows[: w.K]].contiguous()
+    init2 = emb[rows[: w.reorder_K]].contiguous() if w.reorder_K else None
+    return {"emb": emb, "init": init, "init2": init2, "rowptr": rowptr, "colidx": colidx}
+
+
+def step_device(ctx, w, x):
+    ctx.set_timer_group(0)
+    km = ctx.kmeans(x["emb"], w.K, w.iters, x["init"])
+    fine, fineK = km, w.K
+    if w.reorder_K:
+        ctx.set_timer_group(1)
+        fine, fineK = ctx.kmeans(x["emb"], w.reorder_K, w.reorder_iters, x["init2"]), w.reorder_K
+        ctx.set_timer_group(0)
+    q = ctx.partition_quality(x["rowptr"], x["colidx"], km.assign, w.K)
+    r = ctx.reorder(fine.assign, fineK)
+    return km, fine, q, r
+
+
+def make_host_inputs(x):
+    return {k: (v.cpu().pin_memory() if v is not None else None) for k, v in x.items()}
+
+
+def make_host_outputs(w):
+    pin = lambda *shape, dtype: torch.empty(shape, dtype=dtype).pin_memory()   # noqa: E731
+    from paper_2604_01000_b200.binding import KMeansResult, QualityResult, ReorderResult
+    out = {"km": KMeansResult(pin(w.N, dtype=torch.int32), pin(w.K, w.d, dtype=torch.float32), None),
+           "q": QualityResult(pin(1, dtype=torch.int64), pin(w.K, dtype=torch.int64), pin(w.K, dtype=torch.int64)),
+           "r": ReorderResult(pin(w.N, dtype=torch.int32), pin(w.N, dtype=torch.int32))}
+    if w.reorder_K:
+        out["fine"] = KMeansResult(pin(w.N, dtype=torch.int32), pin(w.reorder_K, w.d, dtype=torch.float32), None)
+    return out
+
+
+def step_host(ctx, w, h, out):
+    """The same pass through the host-buffer C-ABI calls: every call uploads its inputs and downloads its results."""
+    km = ctx.kmeans_host(h["emb"], w.K, w.iters, h["init"], out=out["km"])
+    fine, fineK = km, w.K
+    if w.reorder_K:
+        fine, fineK = ctx.kmeans_host(h["emb"], w.reorder_K, w.reorder_iters, h["init2"], out=out["fine"]), w.reorder_K
+    ctx.partition_quality_host(h["rowptr"], h["colidx"], km.assign, w.K, out=out["q"])
+    ctx.reorder_host(fine.assign, fineK, out=out["r"])
+
+
+def host_traffic(w, h):
+    nb = lambda t: t.numel() * t.element_size()   # noqa: E731
+    runs = 2 if w.reorder_K else 1
+    h2d = runs * nb(h["emb"]) + nb(h["init"]) + (nb(h["init2"]) if w.reorder_K else 0)
+    h2d += nb(h["rowptr"]) + nb(h["colidx"]) + 4 * w.N + 4 * w.N               # graph + labels for quality and reorder
+    d2h = runs * 4 * w.N + 4 * w.d * (w.K + w.reorder_K) + 8 * (2 * w.K + 1) + 8 * w.N
+    return h2d, d2h
+
+
+# ------------------------------------------------------------------------------------------------ CPU (oracle) leg
+def oracle_sample_run(w, sample_rows, graph_rows, threads=None):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: K-Means on the first
+    `sample_rows` rows (same K and iteration counts), edge cut / loads and reordering on a graph of the
+    same recipe with `graph_rows` vertices.  Returns (seconds, detail)."""
+    import numpy as np
+    import oracle
+    if threads:
+        oracle.set_num_threads(threads)
+    ws = synth.scaled(w, sample_rows)
+    emb = synth.embeddings(ws).numpy()
+    rows = synth.init_centroid_rows(ws, min(sample_rows, max(w.K, w.reorder_K))).numpy()
+    wg = synth.scaled(w, graph_rows)
+    rowptr, colidx = synth.graph(wg)
+    rowptr, colidx = rowptr.numpy().astype(np.int64), colidx.numpy()
+    labels = (synth.component_labels(wg, torch.arange(graph_rows)) % w.K).to(torch.int32).numpy()
+    t0 = time.perf_counter()
+    oracle.kmeans(emb, w.K, w.iters, emb[rows[: w.K]])
+    fineK = w.K
+    if w.reorder_K:
+        fineK = min(w.reorder_K, sample_rows)
+        oracle.kmeans(emb, fineK, w.reorder_iters, emb[rows[:fineK]])
+    t1 = time.perf_counter()
+    oracle.partition_quality(rowptr, colidx, labels, w.K)
+    oracle.reorder(labels, w.K)
+    t2 = time.perf_counter()
+    iters = w.iters + w.reorder_iters
+    detail = {"kmeans_s": t1 - t0, "graph_s": t2 - t1, "rows": sample_rows, "row_iters": sample_rows * iters,
+              "graph_vertices": graph_rows, "graph_entries": int(colidx.size), "threads": oracle.num_threads()}
+    return t2 - t0, detail
+
+
+def pick_sample_rows(w, budget_s):
+    """Rows for the oracle sample so that its K-Means takes about budget_s seconds on this host."""
+    import oracle
+    probe = 512
+    ws = synth.scaled(w, probe)
+    emb = synth.embeddings(ws).numpy()
+    t0 = time.perf_counter()
+    oracle.kmeans(emb, min(w.K, probe), 1, emb[: min(w.K, probe)])
+    t1 = time.perf_counter()
+    full = (t1 - t0) / probe * w.iters
+    if w.reorder_K:
+        kk = min(w.reorder_K, probe)
+        oracle.kmeans(emb, kk, 1, emb[:kk])
+        full += (time.perf_counter() - t1) / probe * (w.reorder_K / kk) * w.reorder_iters
+    rows = int(budget_s / max(full, 1e-9))
+    return int(max(max(w.K, w.reorder_K, 1024), min(w.N, rows)))
+
+
+def cpu_baseline(w, budget_s=15.0):
+    rows = pick_sample_rows(w, budget_s)
+    graph_rows = min(w.N, 200_000)
+    secs, det = oracle_sample_run(w, rows, graph_rows)
+    return {"value": det["row_iters"] / det["kmeans_s"], "unit": "rows*iters/s", "cores": det["threads"],
+            "kind": "oracle",
+            "sample": (f"fp64 oracle K-Means on the first {rows} rows of {w.name} (same K and iteration counts), "
+                       f"{det['kmeans_s']:.1f} s; edge cut + reorder on a {graph_rows}-vertex graph of the same recipe: "
+                       f"{det['graph_entries'] / max(det['graph_s'], 1e-9):.3g} entries/s"),
+            "edge_cut_entries_per_s": det["graph_entries"] / max(det["graph_s"], 1e-9)}
+
+
+def run_reference(args, w, rank):
+    """Reference arm: the oracle on this machine's host cores, each step a bounded sample of the workload."""
+    if rank != 0:
+        return
+    rows = pick_sample_rows(w, 4.0)
+    graph_rows = min(w.N, 100_000)
+    for _ in range(args.warmup):
+        oracle_sample_run(w, min(rows, 2048), min(graph_rows, 20_000))
+    t_total, row_iters, det = 0.0, 0, None
+    for _ in range(args.steps):
+        secs, det = oracle_sample_run(w, rows, graph_rows)
+        t_total += det["kmeans_s"]
+        row_iters += det["row_iters"]
+    value = row_iters / t_total
+    line = {"impl": "reference", "metric": "kmeans_rows_iters_per_s", "value": value, "unit": "rows*iters/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(w), "reference": "fp64 CPU oracle of this repository (the paper ships no code)"},
+            "cpu_baseline": {"value": value, "unit": "rows*iters/s", "cores": det["threads"], "kind": "oracle",
+                             "sample": f"each step: oracle K-Means on the first {rows} rows (same K, iterations)"},
+            "e2e": {"value": value, "unit": "rows*iters/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg4", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer measurement")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--kmeans-path", default="auto", choices=["auto", "simt", "tensor"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    w = synth.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    import paper_2604_01000_b200 as ep
+
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    ctx = ep.Context(local_rank)
+    ctx.set_kmeans_path(args.kmeans_path)
+    peaks = load_peaks()
+
+    x = make_device_inputs(w, device)
+    nnz = x["colidx"].numel()
+    for _ in range(args.warmup):
+        step_device(ctx, w, x)
+    torch.cuda.synchronize()
+    ctx.check()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps, inputs resident in HBM ------------------------------------------------
+    for g in (0, 1):
+        for t in ep.binding.TIMERS:
+            ctx.profile_read(t, g)
+    ctx.set_profile(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for _ in range(args.steps):
+        step_device(ctx, w, x)
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = start.elapsed_time(stop)
+    launches = ctx.launch_count() - launches0
+    ctx.set_profile(False)
+    timers = {(g, t): ctx.profile_read(t, g) for g in (0, 1) for t in ep.binding.TIMERS}
+    ctx.check()
+    if dist is not None:
+        tms = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+
+    row_iters = w.N * (w.iters + w.reorder_iters)
+    value = world * row_iters * args.steps / (ms * 1e-3)
+
+    # ---- per-pass rates and rooflines from the library's event timers -----------------------------------
+    hbm = peaks["hbm_gbs"]
+    tf32_peak = peaks["bf16_tflops_sustained"] * TF32_OVER_BF16
+    rp_bytes = x["rowptr"].element_size()
+    passes = {}
+
+    def add_pass(name, key, unit_count, unit, bytes_per_launch=None, flops_per_launch=None):
+        tot, n = timers[key]
+        if n == 0:
+            return
+        per = tot / n * 1e-3
+        e = {"launches_timed": n, "ms_per_launch": per * 1e3, "rate": unit_count / per, "unit": unit}
+        if bytes_per_launch is not None:
+            e["roofline"] = {"bound": "hbm", "achieved": bytes_per_launch / per / 1e9, "peak": hbm, "unit": "GB/s",
+                             "frac": bytes_per_launch / per / 1e9 / hbm, "traffic": None,
+                             "peak_source": peaks["_source"]}
+        if flops_per_launch is not None:
+            e["roofline"] = {"bound": "tensor", "achieved": flops_per_launch / per / 1e12, "peak": tf32_peak,
+                             "unit": "TFLOP/s", "frac": flops_per_launch / per / 1e12 / tf32_peak, "traffic": None,
+                             "peak_source": peaks["_source"] + " bf16 sustained x nominal tf32/bf16 ratio"}
+        e["share_of_step"] = tot / ms
+        passes[name] = e
+
+    add_pass(f"kmeans_assign_K{w.K}", (0, "kmeans_assign"), w.N, "rows*iters/s", bytes_per_launch=w.N * (4 * w.d + 4))
+    add_pass(f"kmeans_update_K{w.K}", (0, "kmeans_update"), w.N, "rows*iters/s")
+    if w.reorder_K:
+        add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s",
+                 flops_per_launch=2.0 * w.N * w.reorder_K * w.d)
+        add_pass(f"kmeans_update_K{w.reorder_K}", (1, "kmeans_update"), w.N, "rows*iters/s")
+    add_pass("edge_cut", (0, "edge_cut"), nnz, "edges/s", bytes_per_launch=4 * nnz + rp_bytes * (w.N + 1) + w.N)
+    add_pass("quality_prep", (0, "quality_prep"), w.N, "vertices/s", bytes_per_launch=(4 + rp_bytes) * w.N)
+    add_pass("reorder", (0, "reorder"), w.N, "vertices/s", bytes_per_launch=12 * w.N)
+    dominant = max((p for p in passes.values() if "roofline" in p), key=lambda p: p["share_of_step"])
+    dominant_name = [k for k, v in passes.items() if v is dominant][0]
+    roofline = dict(dominant["roofline"])
+    roofline["kernel"] = dominant_name
+    roofline["ms_per_launch"] = dominant["ms_per_launch"]
+
+    # ---- end to end: the same pass through the host-buffer C ABI (uploads and downloads timed) ---------
+    e2e = None
+    if not args.no_e2e:
+        h = make_host_inputs(x)
+        out = make_host_outputs(w)
+        h2d, d2h = host_traffic(w, h)
+        del x
+        torch.cuda.empty_cache()
+        for _ in range(2):
+            step_host(ctx, w, h, out)
+        barrier()
+        e_steps = max(1, min(args.steps, 3))
+        start.record()
+        for _ in range(e_steps):
+            step_host(ctx, w, h, out)
+        stop.record()
+        barrier()
+        ems = start.elapsed_time(stop)
+        if dist is not None:
+            tms = torch.tensor([ems], dtype=torch.float64, device=device)
+            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+            ems = float(tms.item())
+        ctx.check()
+        e2e = {"value": world * row_iters * e_steps / (ems * 1e-3), "unit": "rows*iters/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ems / e_steps, "steps": e_steps,
+               "api": "ep_kmeans_host / ep_partition_quality_host / ep_reorder_host with page-locked host buffers"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(w)
+
+    if rank == 0:
+        line = {
+            "metric": "kmeans_rows_iters_per_s", "value": value, "unit": "rows*iters/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "nnz": nnz, "l2": "inputs larger than L2, no flush"
+                       if w.N * w.d * 4 > 126e6 else "inputs fit in L2: effective bandwidth, not HBM",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU", "kmeans_path": args.kmeans_path},
+            "edge_cut_edges_per_s": passes.get("edge_cut", {}).get("rate"),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+            "passes": passes,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,187 @@
+/*
+ * embedpart.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path of
+ * embedding-driven graph partitioning:
+ *
+ *   ep_kmeans             Lloyd K-Means over dense node embeddings -> partition of every vertex
+ *                         (Algorithm 3, line 1:  P <- KMeans(E, k))
+ *   ep_partition_quality  edge cut and per-partition loads of a partition over a CSR graph
+ *                         (Section 2.1.1, Eq. 1 "edge-cut ratio" and Eq. 2 "vertex balance")
+ *   ep_reorder            partition-ordered vertex relabelling for graph reordering
+ *                         (Section 4.5.1: vertices of the same partition get consecutive ids)
+ *
+ * Conventions shared by every call
+ *   - Pointers marked [dev] are CUDA device pointers on the context's device, owned by the
+ *     caller; the library neither frees nor keeps them after the call.  Pointers marked [host]
+ *     are ordinary host pointers.  Inputs are never modified.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and the call returns without waiting.  Outputs are valid once the stream has drained.
+ *   - `workspace` [dev] is scratch the caller provides; its minimum size comes from the matching
+ *     *_workspace_bytes query, it must be 256-byte aligned, and its contents are undefined on
+ *     entry and exit.  Two calls that overlap on the GPU must not share a workspace.
+ *   - The return value is a status code (EP_OK = 0).  Argument errors are found on the host before
+ *     anything is launched.  Errors only the device can see (an out-of-range label or column
+ *     index, a non-monotone row pointer, a bounded device wait that ran out) never fault: the
+ *     offending element is skipped, a device status word is raised, and ep_poll_status returns
+ *     it after the caller has synchronised.
+ *   - No function prints, aborts or throws.  Nothing falls back to the CPU: on a device that is
+ *     not compute capability 10.x, ep_create fails with EP_ERR_UNSUPPORTED.
+ */
+#ifndef EMBEDPART_H
+#define EMBEDPART_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    EP_OK = 0,
+    EP_ERR_INVALID_ARG = 1, /* null or misaligned pointer, size out of range */
+    EP_ERR_UNSUPPORTED = 2, /* device is not sm_100, or a shape the library does not handle */
+    EP_ERR_WORKSPACE = 3,   /* workspace too small or misaligned */
+    EP_ERR_BAD_INDEX = 4,   /* device saw a label outside [0,K), a column outside [0,N) or a bad row pointer */
+    EP_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired */
+    EP_ERR_CUDA = 6         /* a CUDA runtime or driver call failed; see ep_last_error */
+};
+
+/* Integer knobs for ep_set_option. */
+enum {
+    EP_OPT_KMEANS_PATH = 1, /* 0 = choose by shape (default), 1 = CUDA-core kernels only, 2 = tensor-core
+                               (tcgen05) kernels wherever the shape allows */
+    EP_OPT_PROFILE = 2,     /* 1 = bracket the main kernels with CUDA events on the launching stream
+                               (read with ep_profile_read); 0 = off (default) */
+    EP_OPT_TIMER_GROUP = 3  /* 0..3: calls made while group g is selected log into timers
+                               g * EP_TIMER_COUNT + timer, so a caller can tell two calls apart */
+};
+
+/* Timers kept while EP_OPT_PROFILE is 1. */
+enum {
+    EP_TIMER_KMEANS_ASSIGN = 0,  /* the assign(-and-accumulate) kernel of every Lloyd iteration */
+    EP_TIMER_KMEANS_UPDATE = 1,  /* everything else of an iteration: grouping, sums, centroid update */
+    EP_TIMER_EDGE_CUT = 2,       /* the tiled edge-cut kernel */
+    EP_TIMER_QUALITY_PREP = 3,   /* label repacking, partition loads, tile start rows */
+    EP_TIMER_REORDER = 4,        /* all kernels of ep_reorder */
+    EP_TIMER_COUNT = 5
+};
+
+typedef struct ep_ctx ep_ctx; /* opaque: device id, device properties, device status word, options */
+
+/* Creates a context bound to CUDA device `device`.  Allocates a few bytes of device memory for the
+ * status word.  Fails with EP_ERR_UNSUPPORTED unless the device is compute capability 10.x. */
+int ep_create(ep_ctx **out, int device);
+/* Releases the context.  The caller must have drained every stream that used it. */
+int ep_destroy(ep_ctx *ctx);
+/* Static, human-readable name of a status code. */
+const char *ep_status_string(int status);
+/* Text of the most recent host-side failure on this context ("" if none). */
+const char *ep_last_error(const ep_ctx *ctx);
+/* Reads and clears the device status word.  Synchronises the device; returns EP_OK or the most
+ * severe EP_ERR_* raised by kernels since the last poll. */
+int ep_poll_status(ep_ctx *ctx);
+int ep_set_option(ep_ctx *ctx, int option, int value);
+int ep_get_option(const ep_ctx *ctx, int option, int *value /* [host] */);
+/* Sum of the event-timed durations (milliseconds) and the number of timed intervals recorded for
+ * `timer` (group * EP_TIMER_COUNT + one of the EP_TIMER_* ids) since it was last read; waits for
+ * the recorded events, then clears the timer.  total_ms and intervals are [host] and may be NULL. */
+int ep_profile_read(ep_ctx *ctx, int timer, double *total_ms, int64_t *intervals);
+/* Number of kernels this context has launched since it was created. */
+int64_t ep_launch_count(const ep_ctx *ctx);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_kmeans -- Lloyd K-Means (Algorithm 3, line 1).
+ *
+ * Squared Euclidean distance; exactly `iters` iterations from the given initial centroids, no
+ * early stop.  In iteration t every row is assigned to its nearest centroid of C_{t-1} (of several
+ * equidistant centroids the lowest index wins), then every centroid becomes the mean of its rows;
+ * a centroid that received no row keeps its previous value.  Returned are the assignment of the
+ * last iteration (made against C_{iters-1}) and C_iters, so each non-empty centroid is the mean of
+ * the rows carrying its label.  iters == 0 assigns the rows against init_centroids and returns
+ * those centroids unchanged.
+ *
+ *   emb            [dev] N x d fp32, row-major, 16-byte aligned
+ *   N              rows, 1 <= N < 2^31
+ *   d              columns, a multiple of 4 in [4, 1024]
+ *   K              clusters, 1 <= K <= min(N, 65536)
+ *   iters          >= 0
+ *   init_centroids [dev] K x d fp32 row-major
+ *   assign         [dev] out, N int32 in [0, K)
+ *   centroids      [dev] out, K x d fp32 row-major (may alias init_centroids)
+ *   objective      [dev] out or NULL: max(iters,1) doubles; entry t-1 is
+ *                  J_t = sum_i |x_i - C_{t-1}[a_i]|^2 of iteration t
+ *
+ * Distances are evaluated as |c|^2 - 2 x.c in fp32 (on the tensor-core path a TF32 product screens
+ * the candidates and every row whose two best scores are closer than the TF32 error bound is
+ * re-evaluated in fp32).  Sums for the means are fp32 per thread block and fp64 across blocks, in a
+ * fixed order: the result is the same from run to run on the same device.  A row holding NaN gets
+ * some valid label and poisons that centroid; nothing faults.
+ */
+size_t ep_kmeans_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K); /* 0 = invalid shape */
+int ep_kmeans(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+              const float *init_centroids, int32_t *assign, float *centroids, double *objective,
+              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_partition_quality -- edge cut and partition loads (Eq. 1 numerator, Eq. 2 operands).
+ *
+ *   edge_cut         = number of stored CSR entries (u -> v) with assign[u] != assign[v]; entries
+ *                      count as stored (both directions of a symmetric graph, duplicates each
+ *                      time, self-loops never)
+ *   part_vertices[p] = number of vertices with assign[v] == p
+ *   part_edges[p]    = sum of the out-degrees of those vertices
+ * The caller forms ECR = edge_cut / nnz and balance = max(part_vertices) / (N / K).
+ *
+ *   rowptr   [dev] N+1 row offsets, int32 or int64 as rowptr_is_int64 says, rowptr[0] = 0,
+ *            non-decreasing, rowptr[N] = nnz
+ *   colidx   [dev] nnz int32 column ids in [0, N), 16-byte aligned
+ *   assign   [dev] N int32 labels in [0, K)
+ *   N, nnz   1 <= N < 2^31, 0 <= nnz < 2^62;  1 <= K <= 2^24
+ *   edge_cut [dev] out, 1 uint64;  part_vertices, part_edges [dev] out, K int64 each
+ * All arithmetic is integer, so the result does not depend on scheduling.
+ */
+size_t ep_quality_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t K);
+int ep_partition_quality(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                         int64_t nnz, const int32_t *assign, int64_t N, int32_t K, uint64_t *edge_cut,
+                         int64_t *part_vertices, int64_t *part_edges, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_reorder -- partition-ordered relabelling (Section 4.5.1).
+ *
+ * perm lists the vertex ids sorted by (assign[v], v): partitions in ascending order, original
+ * order inside a partition (a stable counting sort), so exactly one output is correct.
+ *
+ *   assign   [dev] N int32 labels in [0, K);  1 <= N < 2^31;  1 <= K <= 2^24
+ *   perm     [dev] out, N int32: perm[new_id] = old vertex id
+ *   inv_perm [dev] out or NULL, N int32: inv_perm[v] = new id of v (the paper's bijection pi)
+ */
+size_t ep_reorder_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t K);
+int ep_reorder(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
+               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * Host-buffer variants.  Same operations and the same kernels; inputs and outputs are [host]
+ * pointers.  Each call copies its inputs into `arena` (a [dev] scratch block of at least
+ * *_host_arena_bytes bytes, 256-byte aligned, which also holds the kernel workspace), runs, and
+ * copies the outputs back, all enqueued on `cuda_stream` with cudaMemcpyAsync: with page-locked
+ * host buffers the call returns at once and the outputs are valid when the stream has drained;
+ * with pageable buffers the copies block the calling thread as cudaMemcpyAsync documents.
+ */
+size_t ep_kmeans_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int32_t iters);
+int ep_kmeans_host(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                   const float *init_centroids, int32_t *assign, float *centroids, double *objective,
+                   void *arena, size_t arena_bytes, void *cuda_stream);
+size_t ep_quality_host_arena_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t K, int32_t rowptr_is_int64);
+int ep_partition_quality_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                              int64_t nnz, const int32_t *assign, int64_t N, int32_t K, uint64_t *edge_cut,
+                              int64_t *part_vertices, int64_t *part_edges, void *arena, size_t arena_bytes,
+                              void *cuda_stream);
+size_t ep_reorder_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t K);
+int ep_reorder_host(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
+                    void *arena, size_t arena_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMBEDPART_H */

@@ -1,0 +1,363 @@
+"""ctypes binding of the C ABI in include/embedpart.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from typing import NamedTuple, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libembedpart.so"
+
+EXPORTED_SYMBOLS = (
+    "ep_create", "ep_destroy", "ep_status_string", "ep_last_error", "ep_poll_status", "ep_set_option",
+    "ep_get_option", "ep_kmeans_workspace_bytes", "ep_kmeans", "ep_quality_workspace_bytes",
+    "ep_partition_quality", "ep_reorder_workspace_bytes", "ep_reorder", "ep_profile_read", "ep_launch_count",
+    "ep_kmeans_host_arena_bytes", "ep_kmeans_host", "ep_quality_host_arena_bytes", "ep_partition_quality_host",
+    "ep_reorder_host_arena_bytes", "ep_reorder_host",
+)
+
+EP_OK = 0
+EP_OPT_KMEANS_PATH = 1
+EP_OPT_PROFILE = 2
+EP_OPT_TIMER_GROUP = 3
+TIMER_COUNT = 5
+TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4}
+KMEANS_PATHS = {"auto": 0, "simt": 1, "tensor": 2}
+
+
+class EmbedPartError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"embedpart status {status}: {what}")
+        self.status = status
+
+
+def library_path() -> str:
+    return os.path.join(_PKG, _LIB_NAME)
+
+
+_lib = None
+_lib_lock = threading.Lock()
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the built library; raises if it is missing (there is no fallback)."""
+    global _lib
+    with _lib_lock:
+        if _lib is None:
+            path = library_path()
+            if not os.path.exists(path):
+                raise FileNotFoundError(
+                    f"{path} is missing: build it with `python -m paper_2604_01000_b200.build` "
+                    "(needs nvcc); this package has no CPU fallback")
+            lib = ctypes.CDLL(path)
+            vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+            lib.ep_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+            lib.ep_create.restype = ctypes.c_int
+            lib.ep_destroy.argtypes = [vp]
+            lib.ep_destroy.restype = ctypes.c_int
+            lib.ep_status_string.argtypes = [ctypes.c_int]
+            lib.ep_status_string.restype = ctypes.c_char_p
+            lib.ep_last_error.argtypes = [vp]
+            lib.ep_last_error.restype = ctypes.c_char_p
+            lib.ep_poll_status.argtypes = [vp]
+            lib.ep_poll_status.restype = ctypes.c_int
+            lib.ep_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+            lib.ep_set_option.restype = ctypes.c_int
+            lib.ep_get_option.argtypes = [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+            lib.ep_get_option.restype = ctypes.c_int
+            lib.ep_kmeans_workspace_bytes.argtypes = [vp, i64, i32, i32]
+            lib.ep_kmeans_workspace_bytes.restype = sz
+            lib.ep_kmeans.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+            lib.ep_kmeans.restype = ctypes.c_int
+            lib.ep_quality_workspace_bytes.argtypes = [vp, i64, i64, i32]
+            lib.ep_quality_workspace_bytes.restype = sz
+            lib.ep_partition_quality.argtypes = [vp, vp, i32, vp, i64, vp, i64, i32, vp, vp, vp, vp, sz, vp]
+            lib.ep_partition_quality.restype = ctypes.c_int
+            lib.ep_reorder_workspace_bytes.argtypes = [vp, i64, i32]
+            lib.ep_reorder_workspace_bytes.restype = sz
+            lib.ep_reorder.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
+            lib.ep_reorder.restype = ctypes.c_int
+            lib.ep_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(ctypes.c_int64)]
+            lib.ep_profile_read.restype = ctypes.c_int
+            lib.ep_launch_count.argtypes = [vp]
+            lib.ep_launch_count.restype = ctypes.c_int64
+            lib.ep_kmeans_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32]
+            lib.ep_kmeans_host_arena_bytes.restype = sz
+            lib.ep_kmeans_host.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+            lib.ep_kmeans_host.restype = ctypes.c_int
+            lib.ep_quality_host_arena_bytes.argtypes = [vp, i64, i64, i32, i32]
+            lib.ep_quality_host_arena_bytes.restype = sz
+            lib.ep_partition_quality_host.argtypes = [vp, vp, i32, vp, i64, vp, i64, i32, vp, vp, vp, vp, sz, vp]
+            lib.ep_partition_quality_host.restype = ctypes.c_int
+            lib.ep_reorder_host_arena_bytes.argtypes = [vp, i64, i32]
+            lib.ep_reorder_host_arena_bytes.restype = sz
+            lib.ep_reorder_host.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
+            lib.ep_reorder_host.restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def _dev_ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check_cuda(t: torch.Tensor, dtype, name: str, device: torch.device) -> torch.Tensor:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda or t.device != device:
+        raise ValueError(f"{name} must be a CUDA tensor on {device}")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+class Context:
+    """Owns an ep_ctx for one device and a grow-only workspace tensor."""
+
+    def __init__(self, device: int | torch.device | None = None):
+        if device is None:
+            device = torch.cuda.current_device()
+        self.device = torch.device("cuda", device if isinstance(device, int) else (device.index or 0))
+        self._lib = load_library()
+        h = ctypes.c_void_p()
+        rc = self._lib.ep_create(ctypes.byref(h), self.device.index)
+        if rc != EP_OK:
+            raise EmbedPartError(rc, self._lib.ep_status_string(rc).decode())
+        self._h = h
+        self._ws: Optional[torch.Tensor] = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.ep_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers ------------------------------------------------------------------------------
+    def _raise(self, rc: int):
+        msg = self._lib.ep_status_string(rc).decode()
+        detail = self._lib.ep_last_error(self._h).decode()
+        raise EmbedPartError(rc, f"{msg}: {detail}" if detail else msg)
+
+    def workspace(self, nbytes: int) -> torch.Tensor:
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = None
+            self._ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def poll_status(self) -> int:
+        return int(self._lib.ep_poll_status(self._h))
+
+    def check(self):
+        """Synchronises and raises if a kernel flagged bad input since the last check."""
+        rc = self.poll_status()
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_kmeans_path(self, path: str):
+        rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_PATH, KMEANS_PATHS[path])
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_profile(self, on: bool):
+        rc = self._lib.ep_set_option(self._h, EP_OPT_PROFILE, 1 if on else 0)
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_timer_group(self, group: int):
+        rc = self._lib.ep_set_option(self._h, EP_OPT_TIMER_GROUP, group)
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def profile_read(self, timer: str, group: int = 0):
+        """(total milliseconds, timed intervals) of one library timer since its last read."""
+        ms, n = ctypes.c_double(0), ctypes.c_int64(0)
+        rc = self._lib.ep_profile_read(self._h, group * TIMER_COUNT + TIMERS[timer], ctypes.byref(ms),
+                                       ctypes.byref(n))
+        if rc != EP_OK:
+            self._raise(rc)
+        return ms.value, n.value
+
+    def launch_count(self) -> int:
+        return int(self._lib.ep_launch_count(self._h))
+
+    def _stream(self):
+        return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+
+    # -- calls --------------------------------------------------------------------------------
+    def kmeans(self, emb, K: int, iters: int, init_centroids, objective: bool = False):
+        emb = _check_cuda(emb, torch.float32, "emb", self.device)
+        init = _check_cuda(init_centroids, torch.float32, "init_centroids", self.device)
+        if emb.dim() != 2 or init.dim() != 2 or init.shape != (K, emb.shape[1]):
+            raise ValueError("emb must be N x d and init_centroids K x d")
+        N, d = emb.shape
+        need = self._lib.ep_kmeans_workspace_bytes(self._h, N, d, K)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} d={d} K={K}")
+        ws = self.workspace(need)
+        assign = torch.empty(N, dtype=torch.int32, device=self.device)
+        cent = torch.empty((K, d), dtype=torch.float32, device=self.device)
+        obj = torch.empty(max(iters, 1), dtype=torch.float64, device=self.device) if objective else None
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_kmeans(self._h, _dev_ptr(emb), N, d, K, iters, _dev_ptr(init), _dev_ptr(assign),
+                                     _dev_ptr(cent), _dev_ptr(obj), _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return KMeansResult(assign, cent, obj)
+
+    def partition_quality(self, rowptr, colidx, assign, K: int):
+        if rowptr.dtype not in (torch.int32, torch.int64):
+            raise ValueError("rowptr must be int32 or int64")
+        rowptr = _check_cuda(rowptr, rowptr.dtype, "rowptr", self.device)
+        colidx = _check_cuda(colidx, torch.int32, "colidx", self.device)
+        assign = _check_cuda(assign, torch.int32, "assign", self.device)
+        N, nnz = assign.numel(), colidx.numel()
+        if rowptr.numel() != N + 1:
+            raise ValueError("rowptr must have N + 1 entries")
+        need = self._lib.ep_quality_workspace_bytes(self._h, N, nnz, K)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} nnz={nnz} K={K}")
+        ws = self.workspace(need)
+        cut = torch.empty(1, dtype=torch.int64, device=self.device)
+        pv = torch.empty(K, dtype=torch.int64, device=self.device)
+        pe = torch.empty(K, dtype=torch.int64, device=self.device)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_partition_quality(self._h, _dev_ptr(rowptr), int(rowptr.dtype == torch.int64),
+                                                _dev_ptr(colidx), nnz, _dev_ptr(assign), N, K, _dev_ptr(cut),
+                                                _dev_ptr(pv), _dev_ptr(pe), _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return QualityResult(cut, pv, pe)
+
+    def reorder(self, assign, K: int, inverse: bool = True):
+        assign = _check_cuda(assign, torch.int32, "assign", self.device)
+        N = assign.numel()
+        need = self._lib.ep_reorder_workspace_bytes(self._h, N, K)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} K={K}")
+        ws = self.workspace(need)
+        perm = torch.empty(N, dtype=torch.int32, device=self.device)
+        inv = torch.empty(N, dtype=torch.int32, device=self.device) if inverse else None
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_reorder(self._h, _dev_ptr(assign), N, K, _dev_ptr(perm), _dev_ptr(inv), _dev_ptr(ws),
+                                      ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return ReorderResult(perm, inv)
+
+
+    # -- host-buffer calls (inputs and outputs are CPU tensors; copies are part of the call) -----
+    def _host(self, t, dtype, name):
+        if not isinstance(t, torch.Tensor) or t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CPU tensor of dtype {dtype}")
+        return t
+
+    def kmeans_host(self, emb, K: int, iters: int, init_centroids, objective: bool = False, out=None):
+        emb = self._host(emb, torch.float32, "emb")
+        init = self._host(init_centroids, torch.float32, "init_centroids")
+        N, d = emb.shape
+        need = self._lib.ep_kmeans_host_arena_bytes(self._h, N, d, K, iters)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} d={d} K={K}")
+        ws = self.workspace(need)
+        if out is None:
+            out = KMeansResult(torch.empty(N, dtype=torch.int32).pin_memory(),
+                               torch.empty((K, d), dtype=torch.float32).pin_memory(),
+                               torch.empty(max(iters, 1), dtype=torch.float64).pin_memory() if objective else None)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_kmeans_host(self._h, _dev_ptr(emb), N, d, K, iters, _dev_ptr(init),
+                                          _dev_ptr(out.assign), _dev_ptr(out.centroids), _dev_ptr(out.objective),
+                                          _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+    def partition_quality_host(self, rowptr, colidx, assign, K: int, out=None):
+        rowptr = self._host(rowptr, rowptr.dtype, "rowptr")
+        colidx = self._host(colidx, torch.int32, "colidx")
+        assign = self._host(assign, torch.int32, "assign")
+        N, nnz = assign.numel(), colidx.numel()
+        is64 = int(rowptr.dtype == torch.int64)
+        need = self._lib.ep_quality_host_arena_bytes(self._h, N, nnz, K, is64)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} nnz={nnz} K={K}")
+        ws = self.workspace(need)
+        if out is None:
+            out = QualityResult(torch.empty(1, dtype=torch.int64).pin_memory(),
+                                torch.empty(K, dtype=torch.int64).pin_memory(),
+                                torch.empty(K, dtype=torch.int64).pin_memory())
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_partition_quality_host(self._h, _dev_ptr(rowptr), is64, _dev_ptr(colidx), nnz,
+                                                     _dev_ptr(assign), N, K, _dev_ptr(out.edge_cut),
+                                                     _dev_ptr(out.part_vertices), _dev_ptr(out.part_edges),
+                                                     _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+    def reorder_host(self, assign, K: int, inverse: bool = True, out=None):
+        assign = self._host(assign, torch.int32, "assign")
+        N = assign.numel()
+        need = self._lib.ep_reorder_host_arena_bytes(self._h, N, K)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} K={K}")
+        ws = self.workspace(need)
+        if out is None:
+            out = ReorderResult(torch.empty(N, dtype=torch.int32).pin_memory(),
+                                torch.empty(N, dtype=torch.int32).pin_memory() if inverse else None)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_reorder_host(self._h, _dev_ptr(assign), N, K, _dev_ptr(out.perm), _dev_ptr(out.inv_perm),
+                                           _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+
+class KMeansResult(NamedTuple):
+    assign: torch.Tensor                 # int32 [N]
+    centroids: torch.Tensor              # float32 [K, d]
+    objective: Optional[torch.Tensor]    # float64 [max(iters, 1)] or None
+
+
+class QualityResult(NamedTuple):
+    edge_cut: torch.Tensor               # int64 [1]: cut CSR entries
+    part_vertices: torch.Tensor          # int64 [K]
+    part_edges: torch.Tensor             # int64 [K]
+
+
+class ReorderResult(NamedTuple):
+    perm: torch.Tensor                   # int32 [N]: perm[new_id] = old id
+    inv_perm: Optional[torch.Tensor]     # int32 [N]: inv_perm[old id] = new id
+
+
+_default: dict[int, Context] = {}
+
+
+def default_context(device: Optional[int] = None) -> Context:
+    idx = torch.cuda.current_device() if device is None else device
+    if idx not in _default:
+        _default[idx] = Context(idx)
+    return _default[idx]
+
+
+def ep_kmeans(emb, K, iters, init_centroids, objective=False) -> KMeansResult:
+    """Lloyd K-Means: (assign, centroids, objective).  Asynchronous on the current stream."""
+    return default_context(emb.device.index).kmeans(emb, K, iters, init_centroids, objective)
+
+
+def ep_partition_quality(rowptr, colidx, assign, K) -> QualityResult:
+    """Edge cut and partition loads of `assign` over the CSR graph."""
+    return default_context(assign.device.index).partition_quality(rowptr, colidx, assign, K)
+
+
+def ep_reorder(assign, K, inverse=True) -> ReorderResult:
+    """Partition-ordered permutation (and its inverse)."""
+    return default_context(assign.device.index).reorder(assign, K, inverse)

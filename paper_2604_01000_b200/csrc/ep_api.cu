@@ -1,0 +1,391 @@
+// C ABI entry points: argument checks on the host, then the kernels of the other translation units.
+#include "ep_common.cuh"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+namespace ep {
+
+int fail(ep_ctx *ctx, int status, const char *fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->last_error, sizeof(ctx->last_error), fmt, ap);
+        va_end(ap);
+    }
+    return status;
+}
+
+int cuda_fail(ep_ctx *ctx, cudaError_t e, const char *what) {
+    return fail(ctx, EP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+Timed::Timed(ep_ctx *c, cudaStream_t s, int t) : ctx(c), stream(s), timer(c->opt_timer_group * EP_TIMER_COUNT + t) {
+    if (!ctx->opt_profile) return;
+    if (!ctx->spare_events.empty()) {
+        start = ctx->spare_events.back();
+        ctx->spare_events.pop_back();
+    } else if (cudaEventCreate(&start) != cudaSuccess) {
+        start = nullptr;
+        return;
+    }
+    cudaEventRecord(start, stream);
+}
+
+void Timed::end(int kernels) {
+    ctx->launches += kernels;
+    if (!start) return;
+    cudaEvent_t stop = nullptr;
+    if (!ctx->spare_events.empty()) {
+        stop = ctx->spare_events.back();
+        ctx->spare_events.pop_back();
+    } else if (cudaEventCreate(&stop) != cudaSuccess) {
+        ctx->spare_events.push_back(start);
+        start = nullptr;
+        return;
+    }
+    cudaEventRecord(stop, stream);
+    ctx->intervals.push_back({timer, start, stop});
+    start = nullptr;
+}
+
+}  // namespace ep
+
+using namespace ep;
+
+extern "C" {
+
+const char *ep_status_string(int status) {
+    switch (status) {
+        case EP_OK: return "ok";
+        case EP_ERR_INVALID_ARG: return "invalid argument";
+        case EP_ERR_UNSUPPORTED: return "unsupported device or shape";
+        case EP_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case EP_ERR_BAD_INDEX: return "label, column index or row pointer out of range";
+        case EP_ERR_TIMEOUT: return "bounded device wait expired";
+        case EP_ERR_CUDA: return "CUDA call failed";
+        default: return "unknown status";
+    }
+}
+
+int ep_create(ep_ctx **out, int device) {
+    if (!out) return EP_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) return EP_ERR_UNSUPPORTED;   // no CUDA device at all
+    if (device < 0 || device >= count) return EP_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return EP_ERR_CUDA;
+    if (prop.major != 10) return EP_ERR_UNSUPPORTED;
+    ep_ctx *ctx = new (std::nothrow) ep_ctx();
+    if (!ctx) return EP_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    ctx->opt_kmeans_path = 0;
+    ctx->opt_profile = 0;
+    ctx->opt_timer_group = 0;
+    ctx->launches = 0;
+    ctx->last_error[0] = 0;
+    DeviceGuard g(device);
+    if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
+        delete ctx;
+        return EP_ERR_CUDA;
+    }
+    *out = ctx;
+    return EP_OK;
+}
+
+int ep_destroy(ep_ctx *ctx) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    cudaFree(ctx->d_status);
+    for (auto &iv : ctx->intervals) {
+        cudaEventDestroy(iv.start);
+        cudaEventDestroy(iv.stop);
+    }
+    for (auto e : ctx->spare_events) cudaEventDestroy(e);
+    delete ctx;
+    return EP_OK;
+}
+
+const char *ep_last_error(const ep_ctx *ctx) { return ctx ? ctx->last_error : ""; }
+
+int ep_poll_status(ep_ctx *ctx) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    int word = 0;
+    EP_CUDA(ctx, cudaDeviceSynchronize());
+    EP_CUDA(ctx, cudaMemcpy(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word != 0) EP_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int)));
+    return word;
+}
+
+int ep_set_option(ep_ctx *ctx, int option, int value) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (option == EP_OPT_KMEANS_PATH && value >= 0 && value <= 2) {
+        ctx->opt_kmeans_path = value;
+        return EP_OK;
+    }
+    if (option == EP_OPT_PROFILE && (value == 0 || value == 1)) {
+        ctx->opt_profile = value;
+        return EP_OK;
+    }
+    if (option == EP_OPT_TIMER_GROUP && value >= 0 && value < 4) {
+        ctx->opt_timer_group = value;
+        return EP_OK;
+    }
+    return fail(ctx, EP_ERR_INVALID_ARG, "unknown option %d or value %d", option, value);
+}
+
+int ep_get_option(const ep_ctx *ctx, int option, int *value) {
+    if (!ctx || !value) return EP_ERR_INVALID_ARG;
+    if (option == EP_OPT_KMEANS_PATH) {
+        *value = ctx->opt_kmeans_path;
+        return EP_OK;
+    }
+    if (option == EP_OPT_PROFILE) {
+        *value = ctx->opt_profile;
+        return EP_OK;
+    }
+    if (option == EP_OPT_TIMER_GROUP) {
+        *value = ctx->opt_timer_group;
+        return EP_OK;
+    }
+    return EP_ERR_INVALID_ARG;
+}
+
+int ep_profile_read(ep_ctx *ctx, int timer, double *total_ms, int64_t *intervals) {
+    if (!ctx || timer < 0 || timer >= 4 * EP_TIMER_COUNT) return EP_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    double ms = 0.0;
+    int64_t n = 0;
+    std::vector<ep_timed_interval> keep;
+    for (auto &iv : ctx->intervals) {
+        if (iv.timer != timer) {
+            keep.push_back(iv);
+            continue;
+        }
+        float t = 0.f;
+        EP_CUDA(ctx, cudaEventSynchronize(iv.stop));
+        EP_CUDA(ctx, cudaEventElapsedTime(&t, iv.start, iv.stop));
+        ms += t;
+        n += 1;
+        ctx->spare_events.push_back(iv.start);
+        ctx->spare_events.push_back(iv.stop);
+    }
+    ctx->intervals.swap(keep);
+    if (total_ms) *total_ms = ms;
+    if (intervals) *intervals = n;
+    return EP_OK;
+}
+
+int64_t ep_launch_count(const ep_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+// ---------------------------------------------------------------------------------------------- k-means
+size_t ep_kmeans_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K) {
+    KMeansPlan plan;
+    if (!ctx || !kmeans_make_plan(ctx, N, d, K, &plan)) return 0;
+    return kmeans_workspace_layout(ctx, plan, nullptr, nullptr);
+}
+
+int ep_kmeans(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+              const float *init_centroids, int32_t *assign, float *centroids, double *objective, void *workspace,
+              size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !init_centroids || !assign || !centroids) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!aligned(emb, 16) || !aligned(init_centroids, 16) || !aligned(centroids, 16) || !aligned(assign, 4) ||
+        (objective && !aligned(objective, 8)))
+        return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    if (iters < 0) return fail(ctx, EP_ERR_INVALID_ARG, "iters < 0");
+    KMeansPlan plan;
+    if (!kmeans_make_plan(ctx, N, d, K, &plan))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld d=%d K=%d", (long long)N, d, K);
+    const size_t need = kmeans_workspace_layout(ctx, plan, nullptr, nullptr);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "k-means workspace: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    return kmeans_run(ctx, plan, emb, iters, init_centroids, assign, centroids, objective, workspace,
+                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------------------------- quality
+static bool quality_shape_ok(int64_t N, int64_t nnz, int32_t K) {
+    return N >= 1 && N < (int64_t(1) << 31) && nnz >= 0 && nnz < (int64_t(1) << 62) && K >= 1 && K <= (1 << 24);
+}
+
+size_t ep_quality_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t K) {
+    if (!ctx || !quality_shape_ok(N, nnz, K)) return 0;
+    return quality_workspace_bytes(N, nnz, K);
+}
+
+int ep_partition_quality(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                         int64_t nnz, const int32_t *assign, int64_t N, int32_t K, uint64_t *edge_cut,
+                         int64_t *part_vertices, int64_t *part_edges, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!quality_shape_ok(N, nnz, K))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld K=%d", (long long)N, (long long)nnz, K);
+    if (!rowptr || (!colidx && nnz > 0) || !assign || !edge_cut || !part_vertices || !part_edges)
+        return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!rowptr_is_int64 && nnz >= (int64_t(1) << 31))
+        return fail(ctx, EP_ERR_INVALID_ARG, "nnz needs a 64-bit row pointer");
+    if (!aligned(rowptr, rowptr_is_int64 ? 8 : 4) || !aligned(colidx, 16) || !aligned(assign, 4) ||
+        !aligned(edge_cut, 8) || !aligned(part_vertices, 8) || !aligned(part_edges, 8))
+        return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    const size_t need = quality_workspace_bytes(N, nnz, K);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "quality workspace: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    return quality_run(ctx, rowptr, rowptr_is_int64 != 0, colidx, nnz, assign, N, K,
+                       reinterpret_cast<unsigned long long *>(edge_cut), reinterpret_cast<long long *>(part_vertices),
+                       reinterpret_cast<long long *>(part_edges), workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------------------------- reorder
+static bool reorder_shape_ok(int64_t N, int32_t K) {
+    return N >= 1 && N < (int64_t(1) << 31) && K >= 1 && K <= (1 << 24);
+}
+
+size_t ep_reorder_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t K) {
+    if (!ctx || !reorder_shape_ok(N, K)) return 0;
+    return reorder_workspace_bytes(N, K);
+}
+
+int ep_reorder(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
+               void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!reorder_shape_ok(N, K))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld K=%d", (long long)N, K);
+    if (!assign || !perm) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!aligned(assign, 4) || !aligned(perm, 4) || (inv_perm && !aligned(inv_perm, 4)))
+        return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    const size_t need = reorder_workspace_bytes(N, K);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "reorder workspace: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    return reorder_run(ctx, assign, N, K, perm, inv_perm, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------------------------- host buffers
+size_t ep_kmeans_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int32_t iters) {
+    const size_t ws = ep_kmeans_workspace_bytes(ctx, N, d, K);
+    if (ws == 0 || iters < 0) return 0;
+    Arena a(nullptr);
+    a.take<float>((size_t)N * d);
+    a.take<float>((size_t)K * d);
+    a.take<int32_t>(N);
+    a.take<double>(iters > 0 ? iters : 1);
+    return a.used + ws;
+}
+
+int ep_kmeans_host(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                   const float *init_centroids, int32_t *assign, float *centroids, double *objective, void *arena,
+                   size_t arena_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !init_centroids || !assign || !centroids) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    const size_t need = ep_kmeans_host_arena_bytes(ctx, N, d, K, iters);
+    if (need == 0) return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld d=%d K=%d", (long long)N, d, K);
+    if (!arena || !aligned(arena, 256) || arena_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "k-means host arena: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Arena a(arena);
+    float *d_emb = a.take<float>((size_t)N * d);
+    float *d_cent = a.take<float>((size_t)K * d);
+    int32_t *d_assign = a.take<int32_t>(N);
+    const int T = iters > 0 ? iters : 1;
+    double *d_obj = a.take<double>(T);
+    void *ws = a.base + a.used;
+    EP_CUDA(ctx, cudaMemcpyAsync(d_emb, emb, sizeof(float) * N * d, cudaMemcpyHostToDevice, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(d_cent, init_centroids, sizeof(float) * K * d, cudaMemcpyHostToDevice, st));
+    int rc = ep_kmeans(ctx, d_emb, N, d, K, iters, d_cent, d_assign, d_cent, objective ? d_obj : nullptr, ws,
+                       arena_bytes - a.used, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(assign, d_assign, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(centroids, d_cent, sizeof(float) * K * d, cudaMemcpyDeviceToHost, st));
+    if (objective) EP_CUDA(ctx, cudaMemcpyAsync(objective, d_obj, sizeof(double) * T, cudaMemcpyDeviceToHost, st));
+    return EP_OK;
+}
+
+size_t ep_quality_host_arena_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t K, int32_t rowptr_is_int64) {
+    const size_t ws = ep_quality_workspace_bytes(ctx, N, nnz, K);
+    if (ws == 0) return 0;
+    Arena a(nullptr);
+    a.take<char>((size_t)(N + 1) * (rowptr_is_int64 ? 8 : 4));
+    a.take<int32_t>(nnz);
+    a.take<int32_t>(N);
+    a.take<int64_t>(2 * (size_t)K + 1);
+    return a.used + ws;
+}
+
+int ep_partition_quality_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                              int64_t nnz, const int32_t *assign, int64_t N, int32_t K, uint64_t *edge_cut,
+                              int64_t *part_vertices, int64_t *part_edges, void *arena, size_t arena_bytes,
+                              void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!rowptr || (!colidx && nnz > 0) || !assign || !edge_cut || !part_vertices || !part_edges)
+        return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    const size_t need = ep_quality_host_arena_bytes(ctx, N, nnz, K, rowptr_is_int64);
+    if (need == 0)
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld K=%d", (long long)N, (long long)nnz, K);
+    if (!arena || !aligned(arena, 256) || arena_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "quality host arena: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Arena a(arena);
+    const size_t rp_bytes = (size_t)(N + 1) * (rowptr_is_int64 ? 8 : 4);
+    char *d_rp = a.take<char>(rp_bytes);
+    int32_t *d_ci = a.take<int32_t>(nnz);
+    int32_t *d_as = a.take<int32_t>(N);
+    int64_t *d_out = a.take<int64_t>(2 * (size_t)K + 1);      // [cut | part_vertices | part_edges]
+    void *ws = a.base + a.used;
+    EP_CUDA(ctx, cudaMemcpyAsync(d_rp, rowptr, rp_bytes, cudaMemcpyHostToDevice, st));
+    if (nnz > 0) EP_CUDA(ctx, cudaMemcpyAsync(d_ci, colidx, sizeof(int32_t) * nnz, cudaMemcpyHostToDevice, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(d_as, assign, sizeof(int32_t) * N, cudaMemcpyHostToDevice, st));
+    int rc = ep_partition_quality(ctx, d_rp, rowptr_is_int64, d_ci, nnz, d_as, N, K,
+                                  reinterpret_cast<uint64_t *>(d_out), d_out + 1, d_out + 1 + K, ws,
+                                  arena_bytes - a.used, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(edge_cut, d_out, sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(part_vertices, d_out + 1, sizeof(int64_t) * K, cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(part_edges, d_out + 1 + K, sizeof(int64_t) * K, cudaMemcpyDeviceToHost, st));
+    return EP_OK;
+}
+
+size_t ep_reorder_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t K) {
+    const size_t ws = ep_reorder_workspace_bytes(ctx, N, K);
+    if (ws == 0) return 0;
+    Arena a(nullptr);
+    a.take<int32_t>(N);
+    a.take<int32_t>(N);
+    a.take<int32_t>(N);
+    return a.used + ws;
+}
+
+int ep_reorder_host(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
+                    void *arena, size_t arena_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!assign || !perm) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    const size_t need = ep_reorder_host_arena_bytes(ctx, N, K);
+    if (need == 0) return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld K=%d", (long long)N, K);
+    if (!arena || !aligned(arena, 256) || arena_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "reorder host arena: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Arena a(arena);
+    int32_t *d_as = a.take<int32_t>(N);
+    int32_t *d_perm = a.take<int32_t>(N);
+    int32_t *d_inv = a.take<int32_t>(N);
+    void *ws = a.base + a.used;
+    EP_CUDA(ctx, cudaMemcpyAsync(d_as, assign, sizeof(int32_t) * N, cudaMemcpyHostToDevice, st));
+    int rc = ep_reorder(ctx, d_as, N, K, d_perm, inv_perm ? d_inv : nullptr, ws, arena_bytes - a.used, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(perm, d_perm, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    if (inv_perm) EP_CUDA(ctx, cudaMemcpyAsync(inv_perm, d_inv, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    return EP_OK;
+}
+
+}  // extern "C"

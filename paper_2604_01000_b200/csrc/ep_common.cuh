@@ -1,0 +1,112 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include <vector>
+
+#include "embedpart.h"
+
+struct ep_timed_interval {
+    int timer;
+    cudaEvent_t start, stop;
+};
+
+struct ep_ctx {
+    int device;
+    int sm_count;
+    int smem_optin;        // max dynamic shared memory per block (opt-in), bytes
+    int *d_status;         // device status word (max of EP_ERR_* raised by kernels)
+    int opt_kmeans_path;   // EP_OPT_KMEANS_PATH
+    int opt_profile;       // EP_OPT_PROFILE
+    int opt_timer_group;   // EP_OPT_TIMER_GROUP
+    long long launches;    // kernels launched through this context
+    std::vector<ep_timed_interval> intervals;   // pending event pairs (profile mode)
+    std::vector<cudaEvent_t> spare_events;
+    char last_error[256];
+};
+
+namespace ep {
+
+// ---- host helpers ---------------------------------------------------------------------------
+int fail(ep_ctx *ctx, int status, const char *fmt, ...);
+int cuda_fail(ep_ctx *ctx, cudaError_t e, const char *what);
+
+#define EP_CUDA(ctx, call)                                                   \
+    do {                                                                     \
+        cudaError_t _e = (call);                                             \
+        if (_e != cudaSuccess) return ep::cuda_fail((ctx), _e, #call);      \
+    } while (0)
+
+// Makes the context's device current for the lifetime of the object.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+// Bump allocator over the caller's workspace; every block is 256-byte aligned.
+struct Arena {
+    char *base;
+    size_t used;
+    explicit Arena(void *p) : base(static_cast<char *>(p)), used(0) {}
+    template <typename T>
+    T *take(size_t count) {
+        size_t bytes = (count * sizeof(T) + 255) & ~size_t(255);
+        T *p = base ? reinterpret_cast<T *>(base + used) : nullptr;
+        used += bytes;
+        return p;
+    }
+};
+
+// Brackets a region of stream work with CUDA events when profiling is on; counts its kernels always.
+struct Timed {
+    ep_ctx *ctx;
+    cudaStream_t stream;
+    int timer;
+    cudaEvent_t start = nullptr;
+    Timed(ep_ctx *c, cudaStream_t s, int t);
+    void end(int kernels);   // records the stop event and adds `kernels` to the launch counter
+};
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- k-means (kmeans_simt.cu) ------------------------------------------------------------------
+struct KMeansPlan {
+    int64_t N;
+    int d, K;
+    bool fused;        // centroids + per-warp sums live in shared memory, one pass per iteration
+    int warps;         // warps per block of the assign kernel
+    int grid;          // blocks of the assign kernel (fused: also the number of partial sums)
+    int parts;         // partial-sum slabs the update kernel reduces (fused: grid; otherwise splits per cluster)
+    size_t smem;       // dynamic shared memory of the assign kernel
+};
+bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *plan);
+size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &plan, void *workspace, struct KMeansBuffers *out);
+int kmeans_run(ep_ctx *ctx, const KMeansPlan &plan, const float *emb, int iters, const float *init,
+               int32_t *assign, float *centroids, double *objective, void *workspace, cudaStream_t stream);
+
+// ---- reorder (reorder.cu) -----------------------------------------------------------------------
+size_t reorder_workspace_bytes(int64_t N, int K);
+// Stable sort of vertex ids by label.  timed = false when a caller brackets the call itself.
+int reorder_run(ep_ctx *ctx, const int32_t *assign, int64_t N, int K, int32_t *perm, int32_t *inv_perm,
+                void *workspace, cudaStream_t stream, bool timed = true);
+
+// ---- quality (quality.cu) -----------------------------------------------------------------------
+size_t quality_workspace_bytes(int64_t N, int64_t nnz, int K);
+int quality_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *colidx, int64_t nnz,
+                const int32_t *assign, int64_t N, int K, unsigned long long *edge_cut, long long *part_vertices,
+                long long *part_edges, void *workspace, cudaStream_t stream);
+
+}  // namespace ep
+
+// ---- device helpers -------------------------------------------------------------------------------
+__device__ __forceinline__ void ep_raise(int *status, int code) { atomicMax(status, code); }

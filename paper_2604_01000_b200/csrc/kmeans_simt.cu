@@ -1,0 +1,590 @@
+// Lloyd K-Means on CUDA cores (Algorithm 3, line 1): the assign-and-accumulate pass, the centroid
+// update and the per-call driver.  A warp owns whole rows; lane l holds the 16-byte slices
+// l, l+32, ... of a row in registers, so a row is read from HBM exactly once, coalesced.
+#include "ep_common.cuh"
+
+#include <math_constants.h>
+
+#include <algorithm>
+#include <type_traits>
+
+namespace {
+
+constexpr int KC = 8;          // centroids reduced together by one butterfly
+constexpr int UPD_THREADS = 128;
+constexpr unsigned FULL = 0xffffffffu;
+
+__device__ __forceinline__ float4 ldg_stream(const float4 *p) {
+    float4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float dot4(const float4 &a, const float4 &b, float acc) {
+    acc = fmaf(a.x, b.x, acc);
+    acc = fmaf(a.y, b.y, acc);
+    acc = fmaf(a.z, b.z, acc);
+    acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+
+// Sums 8 per-lane values across the warp with 9 shuffles instead of 40: each exchange halves the
+// number of values a lane still carries.  On return every lane holds the warp-wide total of value
+// index ((lane>>4)&1)*4 + ((lane>>3)&1)*2 + ((lane>>2)&1).
+__device__ __forceinline__ float reduce8_transposed(const float (&a)[KC], int lane) {
+    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
+    float b[4], c[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float send = h16 ? a[i] : a[i + 4];
+        float keep = h16 ? a[i + 4] : a[i];
+        b[i] = keep + __shfl_xor_sync(FULL, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        float send = h8 ? b[i] : b[i + 2];
+        float keep = h8 ? b[i + 2] : b[i];
+        c[i] = keep + __shfl_xor_sync(FULL, send, 8);
+    }
+    float send = h4 ? c[0] : c[1];
+    float keep = h4 ? c[1] : c[0];
+    float v = keep + __shfl_xor_sync(FULL, send, 4);
+    v += __shfl_xor_sync(FULL, v, 2);
+    v += __shfl_xor_sync(FULL, v, 1);
+    return v;
+}
+
+__device__ __forceinline__ int lane_chunk_slot(int lane) {
+    return ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+}
+
+template <int VPL, int R>
+struct Rows {
+    float4 x[R][VPL];
+};
+
+template <int VPL, int R>
+__device__ __forceinline__ void load_rows(Rows<VPL, R> &r, const float *emb, int64_t row, int64_t row_end, int d4,
+                                          int lane) {
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            int q = lane + 32 * v;
+            if (row + i < row_end && q < d4)
+                r.x[i][v] = ldg_stream(reinterpret_cast<const float4 *>(emb) + (row + i) * (int64_t)d4 + q);
+            else
+                r.x[i][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+}
+
+// Scores R rows against the kcount (multiple of KC) centroids staged at cs (row pitch DP4 float4,
+// zero padded) with |c|^2 at cn (+inf for padding), and folds them into the per-lane running best.
+// Score of (row, k) = |c_k|^2 - 2 x.c_k; the row's |x|^2 does not change the argmin.
+template <int VPL, int R>
+__device__ __forceinline__ void score_chunk(const Rows<VPL, R> &rows, const float4 *cs, const float *cn, int kbase,
+                                            int kcount, int lane, float (&best)[R], int (&bidx)[R]) {
+    constexpr int DP4 = VPL * 32;
+    const int slot = lane_chunk_slot(lane);
+    for (int kb = 0; kb < kcount; kb += KC) {
+        float acc[R][KC];
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+#pragma unroll
+            for (int kk = 0; kk < KC; ++kk) acc[i][kk] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < KC; ++kk) {
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                float4 c = cs[(kb + kk) * DP4 + lane + 32 * v];
+#pragma unroll
+                for (int i = 0; i < R; ++i) acc[i][kk] = dot4(rows.x[i][v], c, acc[i][kk]);
+            }
+        }
+        float cnk = cn[kb + slot];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            float dot = reduce8_transposed(acc[i], lane);
+            float s = fmaf(-2.f, dot, cnk);
+            s = (s == s) ? s : CUDART_INF_F;          // a NaN score never wins
+            if (s < best[i]) {                         // strict: the earlier (lower) index keeps a tie
+                best[i] = s;
+                bidx[i] = kbase + kb + slot;
+            }
+        }
+    }
+}
+
+// Warp-wide argmin of (best, bidx) with the lowest index winning ties; every lane gets the result.
+__device__ __forceinline__ int warp_argmin(float best, int bidx) {
+#pragma unroll
+    for (int m = 16; m >= 4; m >>= 1) {
+        float ov = __shfl_xor_sync(FULL, best, m);
+        int oi = __shfl_xor_sync(FULL, bidx, m);
+        if (ov < best || (ov == best && oi < bidx)) {
+            best = ov;
+            bidx = oi;
+        }
+    }
+    return bidx;
+}
+
+// Copies centroids [k0, k0+kcount) into shared memory with row pitch DP4 float4, zero-filling the
+// padding columns and the rows at or beyond K, and their squared norms (+inf beyond K).
+__device__ __forceinline__ void stage_centroids(float4 *cs, float *cn, const float *C, const float *cnorm, int k0,
+                                                int kcount, int K, int d4, int DP4) {
+    for (int i = threadIdx.x; i < kcount * DP4; i += blockDim.x) {
+        int k = i / DP4, q = i - k * DP4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (k0 + k < K && q < d4) v = __ldg(reinterpret_cast<const float4 *>(C) + (int64_t)(k0 + k) * d4 + q);
+        cs[i] = v;
+    }
+    for (int k = threadIdx.x; k < kcount; k += blockDim.x) cn[k] = (k0 + k < K) ? cnorm[k0 + k] : CUDART_INF_F;
+}
+
+// Fused pass for small K: centroids and one private sum table per warp live in shared memory.
+// Each warp walks a contiguous run of rows, so the order of every addition is fixed by the launch
+// shape alone.  Block b leaves its partial sums in psum[b] and its label counts in pcnt[b].
+template <int VPL, int R>
+__global__ void __launch_bounds__(256) kmeans_assign_fused(const float *__restrict__ emb, int64_t N, int d, int K,
+                                                           int Kpad, const float *__restrict__ C,
+                                                           const float *__restrict__ cnorm,
+                                                           int32_t *__restrict__ assign, float *__restrict__ psum,
+                                                           int *__restrict__ pcnt, int64_t rows_per_block,
+                                                           int64_t rows_per_warp) {
+    constexpr int DP4 = VPL * 32;
+    extern __shared__ float4 smem4[];
+    const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int d4 = d >> 2;
+    float4 *cs = smem4;                                   // [Kpad][DP4]
+    float4 *sw = cs + (size_t)Kpad * DP4;                 // [W][K][DP4]
+    float *cn = reinterpret_cast<float *>(sw + (size_t)W * K * DP4);   // [Kpad]
+    int *cw = reinterpret_cast<int *>(cn + Kpad);         // [W][K]
+
+    stage_centroids(cs, cn, C, cnorm, 0, Kpad, K, d4, DP4);
+    for (int i = threadIdx.x; i < W * K * DP4; i += blockDim.x) sw[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = threadIdx.x; i < W * K; i += blockDim.x) cw[i] = 0;
+    __syncthreads();
+
+    const int64_t blk0 = (int64_t)blockIdx.x * rows_per_block;
+    const int64_t blk1 = min(N, blk0 + rows_per_block);
+    const int64_t w0 = min(blk1, blk0 + (int64_t)warp * rows_per_warp);
+    const int64_t w1 = min(blk1, w0 + rows_per_warp);
+    float4 *mysum = sw + (size_t)warp * K * DP4;
+    int *mycnt = cw + warp * K;
+
+    Rows<VPL, R> cur, nxt;
+    load_rows(cur, emb, w0, w1, d4, lane);
+    for (int64_t row = w0; row < w1; row += R) {
+        load_rows(nxt, emb, row + R, w1, d4, lane);
+        float best[R];
+        int bidx[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            best[i] = CUDART_INF_F;
+            bidx[i] = 0;
+        }
+        score_chunk<VPL, R>(cur, cs, cn, 0, Kpad, lane, best, bidx);
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            if (row + i < w1) {
+                int a = warp_argmin(best[i], bidx[i]);
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) {
+                    float4 s = mysum[a * DP4 + lane + 32 * v];
+                    s.x += cur.x[i][v].x;
+                    s.y += cur.x[i][v].y;
+                    s.z += cur.x[i][v].z;
+                    s.w += cur.x[i][v].w;
+                    mysum[a * DP4 + lane + 32 * v] = s;
+                }
+                if (lane == 0) {
+                    mycnt[a] += 1;
+                    assign[row + i] = a;
+                }
+            }
+        }
+        cur = nxt;
+    }
+    __syncthreads();
+    // fold the warps' tables in warp order and publish this block's partials
+    float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
+    for (int i = threadIdx.x; i < K * d4; i += blockDim.x) {
+        int k = i / d4, q = i - k * d4;
+        float4 s = sw[k * DP4 + q];
+        for (int w = 1; w < W; ++w) {
+            float4 t = sw[((size_t)w * K + k) * DP4 + q];
+            s.x += t.x;
+            s.y += t.y;
+            s.z += t.z;
+            s.w += t.w;
+        }
+        out[i] = s;
+    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        int c = 0;
+        for (int w = 0; w < W; ++w) c += cw[w * K + k];
+        pcnt[(size_t)blockIdx.x * K + k] = c;
+    }
+}
+
+// Label-only pass for K too large for the fused kernel: a block keeps W*R rows in registers and
+// streams the centroid table through shared memory in chunks.
+template <int VPL, int R>
+__global__ void __launch_bounds__(256) kmeans_assign_chunked(const float *__restrict__ emb, int64_t N, int d, int K,
+                                                             int Kpad, int kchunk, const float *__restrict__ C,
+                                                             const float *__restrict__ cnorm,
+                                                             int32_t *__restrict__ assign) {
+    constexpr int DP4 = VPL * 32;
+    extern __shared__ float4 smem4[];
+    const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int d4 = d >> 2;
+    float4 *cs = smem4;                                            // [kchunk][DP4]
+    float *cn = reinterpret_cast<float *>(cs + (size_t)kchunk * DP4);   // [kchunk]
+    const int64_t batch = (int64_t)W * R;
+    for (int64_t b0 = (int64_t)blockIdx.x * batch; b0 < N; b0 += (int64_t)gridDim.x * batch) {
+        const int64_t row = b0 + (int64_t)warp * R;
+        Rows<VPL, R> cur;
+        load_rows(cur, emb, row, N, d4, lane);
+        float best[R];
+        int bidx[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            best[i] = CUDART_INF_F;
+            bidx[i] = 0;
+        }
+        for (int k0 = 0; k0 < Kpad; k0 += kchunk) {
+            const int kc = min(kchunk, Kpad - k0);
+            __syncthreads();
+            stage_centroids(cs, cn, C, cnorm, k0, kc, K, d4, DP4);
+            __syncthreads();
+            score_chunk<VPL, R>(cur, cs, cn, k0, kc, lane, best, bidx);
+        }
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            int a = warp_argmin(best[i], bidx[i]);
+            if (lane == 0 && row + i < N) assign[row + i] = a;
+        }
+    }
+}
+
+// Sums the rows of each cluster for the label-only path.  order lists the row ids grouped by label
+// (ascending ids inside a group), off[k] is the first position of cluster k.  Block (k, s) adds up
+// slice s of cluster k in a fixed order and leaves the result in psum[s][k], the count in pcnt[s][k].
+template <int VPL>
+__global__ void __launch_bounds__(256) kmeans_segment_sums(const float *__restrict__ emb, int d, int K,
+                                                           const int32_t *__restrict__ order,
+                                                           const int64_t *__restrict__ off,
+                                                           float *__restrict__ psum, int *__restrict__ pcnt) {
+    __shared__ float4 red[8][VPL * 32];
+    const int k = blockIdx.x, s = blockIdx.y, S = gridDim.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
+    const int64_t n = off[k + 1] - off[k];
+    const int64_t p0 = off[k] + n * s / S, p1 = off[k] + n * (s + 1) / S;
+    float4 acc[VPL];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t p = p0 + warp; p < p1; p += 8) {
+        const int64_t row = order[p];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            int q = lane + 32 * v;
+            if (q < d4) {
+                float4 x = ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q);
+                acc[v].x += x.x;
+                acc[v].y += x.y;
+                acc[v].z += x.z;
+                acc[v].w += x.w;
+            }
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) red[warp][lane + 32 * v] = acc[v];
+    __syncthreads();
+    float4 *out = reinterpret_cast<float4 *>(psum) + ((size_t)s * K + k) * d4;
+    for (int q = threadIdx.x; q < d4; q += blockDim.x) {
+        float4 t = red[0][q];
+        for (int w = 1; w < 8; ++w) {
+            t.x += red[w][q].x;
+            t.y += red[w][q].y;
+            t.z += red[w][q].z;
+            t.w += red[w][q].w;
+        }
+        out[q] = t;
+    }
+    if (threadIdx.x == 0) pcnt[(size_t)s * K + k] = (int)(p1 - p0);
+}
+
+// hist[k] = number of rows labelled k (integer atomics: exact whatever the order).
+__global__ void label_histogram(const int32_t *__restrict__ assign, int64_t N, int K, unsigned long long *hist) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += (int64_t)gridDim.x * blockDim.x)
+        atomicAdd(&hist[assign[i]], 1ull);
+}
+
+// off[0..K] = exclusive prefix sum of hist (one block; K <= 65536).
+__global__ void label_offsets(const unsigned long long *__restrict__ hist, int K, int64_t *off) {
+    __shared__ long long part[256];
+    const int per = (K + 255) / 256;
+    const int k0 = min(K, (int)threadIdx.x * per), k1 = min(K, k0 + per);
+    long long s = 0;
+    for (int k = k0; k < k1; ++k) s += (long long)hist[k];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long run = 0;
+        for (int t = 0; t < 256; ++t) {
+            long long v = part[t];
+            part[t] = run;
+            run += v;
+        }
+    }
+    __syncthreads();
+    long long run = part[threadIdx.x];
+    for (int k = k0; k < k1; ++k) {
+        off[k] = run;
+        run += (long long)hist[k];
+    }
+    if (k1 == K && k0 <= K) off[K] = run;
+}
+
+template <int T>
+__device__ __forceinline__ double block_sum_fixed(double v, double *buf) {
+    buf[threadIdx.x] = v;
+    __syncthreads();
+#pragma unroll
+    for (int s = T / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) buf[threadIdx.x] += buf[threadIdx.x + s];
+        __syncthreads();
+    }
+    double r = buf[0];
+    __syncthreads();
+    return r;
+}
+
+// |c_k|^2 of the initial centroids (fp64 sum, rounded once).
+__global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__restrict__ C, int d, float *cnorm) {
+    __shared__ double buf[UPD_THREADS];
+    const int k = blockIdx.x;
+    double t = 0.0;
+    for (int j = threadIdx.x; j < d; j += UPD_THREADS) {
+        double c = C[(size_t)k * d + j];
+        t += c * c;
+    }
+    t = block_sum_fixed<UPD_THREADS>(t, buf);
+    if (threadIdx.x == 0) cnorm[k] = (float)t;
+}
+
+// Centroid update, one block per cluster: S_k = sum over the partial slabs (fp64, slab order),
+// c_k <- S_k / n_k when n_k > 0, else unchanged; also |c_k|^2 of the new centroid and this
+// cluster's share of the objective, n_k |c|^2 - 2 c.S_k with c the centroid the rows were assigned
+// against (the rows' own sum of |x|^2 is added once by objective_finalize).
+__global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__restrict__ psum,
+                                                               const int *__restrict__ pcnt, int parts, int K, int d,
+                                                               float *C, float *cnorm, double *objterm,
+                                                               int keep_centroids) {
+    __shared__ double buf[UPD_THREADS];
+    const int k = blockIdx.x;
+    long long n = 0;
+    for (int p = 0; p < parts; ++p) n += pcnt[(size_t)p * K + k];
+    double t_cs = 0.0, t_cc = 0.0, t_nn = 0.0;
+    for (int j = threadIdx.x; j < d; j += UPD_THREADS) {
+        double S = 0.0;
+        for (int p = 0; p < parts; ++p) S += (double)psum[((size_t)p * K + k) * d + j];
+        const float cold = C[(size_t)k * d + j];
+        float cnew = cold;
+        if (n > 0 && !keep_centroids) cnew = (float)(S / (double)n);
+        t_cs += (double)cold * S;
+        t_cc += (double)cold * (double)cold;
+        t_nn += (double)cnew * (double)cnew;
+        C[(size_t)k * d + j] = cnew;
+    }
+    t_cs = block_sum_fixed<UPD_THREADS>(t_cs, buf);
+    t_cc = block_sum_fixed<UPD_THREADS>(t_cc, buf);
+    t_nn = block_sum_fixed<UPD_THREADS>(t_nn, buf);
+    if (threadIdx.x == 0) {
+        cnorm[k] = (float)t_nn;
+        objterm[k] = (double)n * t_cc - 2.0 * t_cs;
+    }
+}
+
+// x2part[b] = sum of squares of block b's share of the embedding matrix (fp64).
+__global__ void __launch_bounds__(256) sum_of_squares(const float *__restrict__ emb, int64_t n4, double *x2part) {
+    __shared__ double buf[256];
+    const int64_t per = (n4 + gridDim.x - 1) / gridDim.x;
+    const int64_t i0 = blockIdx.x * per, i1 = min(n4, i0 + per);
+    double t = 0.0;
+    for (int64_t i = i0 + threadIdx.x; i < i1; i += 256) {
+        float4 x = ldg_stream(reinterpret_cast<const float4 *>(emb) + i);
+        t += (double)x.x * x.x + (double)x.y * x.y + (double)x.z * x.z + (double)x.w * x.w;
+    }
+    t = block_sum_fixed<256>(t, buf);
+    if (threadIdx.x == 0) x2part[blockIdx.x] = t;
+}
+
+// objective[t] = sum_i |x_i|^2 + sum_k objterm[k], both summed in index order.
+__global__ void __launch_bounds__(256) objective_finalize(const double *__restrict__ x2part, int nparts,
+                                                          const double *__restrict__ objterm, int K, double *out) {
+    __shared__ double buf[256];
+    double t = 0.0;
+    for (int i = threadIdx.x; i < nparts; i += 256) t += x2part[i];
+    for (int k = threadIdx.x; k < K; k += 256) t += objterm[k];
+    t = block_sum_fixed<256>(t, buf);
+    if (threadIdx.x == 0) *out = t;
+}
+
+constexpr int X2_BLOCKS = 1184;
+
+template <typename F>
+int dispatch_vpl(int d, F &&f) {
+    if (d <= 128) return f(std::integral_constant<int, 1>{});
+    if (d <= 256) return f(std::integral_constant<int, 2>{});
+    if (d <= 512) return f(std::integral_constant<int, 4>{});
+    return f(std::integral_constant<int, 8>{});
+}
+
+}  // namespace
+
+namespace ep {
+
+struct KMeansBuffers {
+    float *cnorm;
+    float *psum;
+    int *pcnt;
+    double *objterm;
+    double *x2part;
+    unsigned long long *hist;
+    int64_t *off;
+    int32_t *order;
+    void *sort_ws;
+};
+
+static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
+static inline int rows_per_step(int vpl) { return vpl == 1 ? 4 : vpl == 2 ? 2 : 1; }
+
+bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *plan) {
+    if (N < 1 || N >= (int64_t(1) << 31) || d < 4 || d > 1024 || (d & 3) || K < 1 || K > 65536 || K > N) return false;
+    KMeansPlan p{};
+    p.N = N;
+    p.d = d;
+    p.K = K;
+    const int vpl = vpl_of(d);
+    const size_t row_bytes = (size_t)vpl * 512;                   // padded centroid row in shared memory
+    const int Kpad = (K + KC - 1) / KC * KC;
+    const size_t budget = (size_t)ctx->smem_optin - 1024;
+    // fused: Kpad centroid rows + W*K sum rows + norms + counts
+    int W = 0;
+    for (int w = 8; w >= 2; --w) {
+        size_t need = Kpad * row_bytes + (size_t)w * K * row_bytes + Kpad * 4 + (size_t)w * K * 4;
+        if (need <= budget) {
+            W = w;
+            break;
+        }
+    }
+    p.fused = W >= 4 && K <= 256;
+    if (p.fused) {
+        p.warps = W;
+        p.smem = Kpad * row_bytes + (size_t)W * K * row_bytes + Kpad * 4 + (size_t)W * K * 4;
+        const int64_t step = (int64_t)W * rows_per_step(vpl);
+        const int per_sm = (2 * (p.smem + 1024) <= (size_t)ctx->smem_optin) ? 2 : 1;   // registers allow two blocks
+        p.grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)ctx->sm_count * per_sm, ceil_div(N, step)));
+        p.parts = p.grid;
+    } else {
+        p.warps = 8;
+        int kchunk = (int)std::min<size_t>(Kpad, (96 * 1024) / row_bytes / KC * KC);
+        p.smem = (size_t)kchunk * row_bytes + (size_t)kchunk * 4;
+        const int64_t batch = 8 * rows_per_step(vpl);
+        p.grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)ctx->sm_count * 2, ceil_div(N, batch)));
+        p.parts = (int)std::max<int64_t>(1, std::min<int64_t>(64, ceil_div(2048, K)));
+    }
+    *plan = p;
+    return true;
+}
+
+size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *workspace, KMeansBuffers *out) {
+    (void)ctx;
+    Arena a(workspace);
+    KMeansBuffers b{};
+    b.cnorm = a.take<float>(p.K);
+    b.psum = a.take<float>((size_t)p.parts * p.K * p.d);
+    b.pcnt = a.take<int>((size_t)p.parts * p.K);
+    b.objterm = a.take<double>(p.K);
+    b.x2part = a.take<double>(X2_BLOCKS);
+    if (!p.fused) {
+        b.hist = a.take<unsigned long long>(p.K);
+        b.off = a.take<int64_t>(p.K + 1);
+        b.order = a.take<int32_t>(p.N);
+        b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
+    }
+    if (out) *out = b;
+    return a.used;
+}
+
+int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, const float *init, int32_t *assign,
+               float *centroids, double *objective, void *workspace, cudaStream_t stream) {
+    KMeansBuffers b;
+    kmeans_workspace_layout(ctx, p, workspace, &b);
+    const int K = p.K, d = p.d;
+    const int Kpad = (K + KC - 1) / KC * KC;
+    const int64_t N = p.N;
+
+    if (centroids != init)
+        EP_CUDA(ctx, cudaMemcpyAsync(centroids, init, sizeof(float) * K * d, cudaMemcpyDeviceToDevice, stream));
+    {
+        Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
+        centroid_norms<<<K, UPD_THREADS, 0, stream>>>(centroids, d, b.cnorm);
+        if (objective) sum_of_squares<<<X2_BLOCKS, 256, 0, stream>>>(emb, N * (d / 4), b.x2part);
+        tm.end(objective ? 2 : 1);
+    }
+
+    const int T = iters > 0 ? iters : 1;
+    for (int t = 0; t < T; ++t) {
+        int rc = dispatch_vpl(d, [&](auto vpl_c) -> int {
+            constexpr int VPL = decltype(vpl_c)::value;
+            constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
+            if (p.fused) {
+                auto kern = kmeans_assign_fused<VPL, R>;
+                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+                int64_t rpw = ceil_div(ceil_div(N, p.grid), p.warps);
+                rpw = ceil_div(rpw, R) * R;
+                int64_t rpb = rpw * p.warps;
+                Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
+                kern<<<p.grid, p.warps * 32, p.smem, stream>>>(emb, N, d, K, Kpad, centroids, b.cnorm, assign, b.psum,
+                                                             b.pcnt, rpb, rpw);
+                tm.end(1);
+            } else {
+                auto kern = kmeans_assign_chunked<VPL, R>;
+                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+                const int row_bytes = VPL * 512;
+                int kchunk = (int)std::min<size_t>(Kpad, (96 * 1024) / row_bytes / KC * KC);
+                {
+                    Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
+                    kern<<<p.grid, 256, p.smem, stream>>>(emb, N, d, K, Kpad, kchunk, centroids, b.cnorm, assign);
+                    tm.end(1);
+                }
+                // group the rows by label, then sum each group in a fixed order
+                Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
+                EP_CUDA(ctx, cudaMemsetAsync(b.hist, 0, sizeof(unsigned long long) * K, stream));
+                label_histogram<<<ctx->sm_count * 4, 256, 0, stream>>>(assign, N, K, b.hist);
+                label_offsets<<<1, 256, 0, stream>>>(b.hist, K, b.off);
+                int r2 = reorder_run(ctx, assign, N, K, b.order, nullptr, b.sort_ws, stream, /*timed=*/false);
+                if (r2 != EP_OK) return r2;
+                kmeans_segment_sums<VPL><<<dim3(K, p.parts), 256, 0, stream>>>(emb, d, K, b.order, b.off, b.psum, b.pcnt);
+                tm.end(3);
+            }
+            return EP_OK;
+        });
+        if (rc != EP_OK) return rc;
+        Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
+        centroid_update<<<K, UPD_THREADS, 0, stream>>>(b.psum, b.pcnt, p.parts, K, d, centroids, b.cnorm, b.objterm,
+                                                       iters == 0 ? 1 : 0);
+        if (objective) objective_finalize<<<1, 256, 0, stream>>>(b.x2part, X2_BLOCKS, b.objterm, K, objective + t);
+        tm.end(objective ? 2 : 1);
+    }
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
+}
+
+}  // namespace ep

@@ -1,0 +1,268 @@
+// Edge cut and partition loads (Section 2.1.1, Eq. 1 and Eq. 2) over a CSR graph.
+//
+// The work is split by EDGES, not by rows, so a power-law degree distribution cannot unbalance it:
+// every block takes tiles of QT_EDGES consecutive CSR entries, streams their column ids with 16-byte
+// loads, and recovers the source vertex of each entry from a bitmap of row starts built in shared
+// memory.  Labels are first repacked to the narrowest integer that holds K values so that the
+// per-entry label gather touches as few cache lines as possible.
+#include "ep_common.cuh"
+
+#include <algorithm>
+
+namespace {
+
+constexpr int QT_THREADS = 256;
+constexpr int QT_VEC = 8;                                   // 16-byte loads per thread per tile
+constexpr int QT_EDGES = QT_THREADS * QT_VEC * 4;           // 8192 entries per tile
+constexpr int QT_WORDS = QT_EDGES / 32;                     // 256 bitmap words, one per thread
+constexpr int HIST_SMEM_K = 2048;
+constexpr unsigned FULL = 0xffffffffu;
+
+// tile_row[t] = last row r in [0, N) whose first entry is at or before t * QT_EDGES; tile_row[ntiles] = N-1.
+template <typename RowT>
+__global__ void tile_start_rows(const RowT *__restrict__ rowptr, int64_t N, int64_t ntiles, int32_t *tile_row) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t > ntiles) return;
+    if (t == ntiles) {
+        tile_row[t] = (int32_t)(N - 1);
+        return;
+    }
+    const int64_t e = t * QT_EDGES;
+    int64_t lo = 0, hi = N - 1;                             // rowptr[0] = 0 <= e always
+    while (lo < hi) {
+        int64_t mid = (lo + hi + 1) >> 1;
+        if ((int64_t)rowptr[mid] <= e)
+            lo = mid;
+        else
+            hi = mid - 1;
+    }
+    tile_row[t] = (int32_t)lo;
+}
+
+// Validates and repacks the labels, and accumulates part_vertices / part_edges.
+template <typename RowT, typename LabT>
+__global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restrict__ rowptr,
+                                                             const int32_t *__restrict__ assign, int64_t N,
+                                                             int64_t nnz, int K, LabT *__restrict__ lab,
+                                                             unsigned long long *part_vertices,
+                                                             unsigned long long *part_edges, int *status) {
+    __shared__ unsigned int cv[HIST_SMEM_K];
+    __shared__ unsigned long long ce[HIST_SMEM_K];
+    const bool local = K <= HIST_SMEM_K;
+    if (local) {
+        for (int k = threadIdx.x; k < K; k += blockDim.x) {
+            cv[k] = 0u;
+            ce[k] = 0ull;
+        }
+        __syncthreads();
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if ((int64_t)rowptr[0] != 0 || (int64_t)rowptr[N] != nnz) ep_raise(status, EP_ERR_BAD_INDEX);
+    }
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < N; v += (int64_t)gridDim.x * blockDim.x) {
+        int a = assign[v];
+        if ((unsigned)a >= (unsigned)K) {
+            ep_raise(status, EP_ERR_BAD_INDEX);
+            a = 0;
+        }
+        lab[v] = (LabT)a;
+        long long deg = (long long)rowptr[v + 1] - (long long)rowptr[v];
+        if (deg < 0) {
+            ep_raise(status, EP_ERR_BAD_INDEX);
+            deg = 0;
+        }
+        if (local) {
+            atomicAdd(&cv[a], 1u);
+            atomicAdd(&ce[a], (unsigned long long)deg);
+        } else {
+            atomicAdd(&part_vertices[a], 1ull);
+            atomicAdd(&part_edges[a], (unsigned long long)deg);
+        }
+    }
+    if (local) {
+        __syncthreads();
+        for (int k = threadIdx.x; k < K; k += blockDim.x) {
+            if (cv[k]) atomicAdd(&part_vertices[k], (unsigned long long)cv[k]);
+            if (ce[k]) atomicAdd(&part_edges[k], ce[k]);
+        }
+    }
+}
+
+// Counts the cut entries.  For a tile [e0, e0+ne): the rows whose first entry falls inside the tile
+// set a bit at that position and park their label there; an entry's source label is the label at the
+// nearest set bit at or before it (or, before the first set bit, the label of the row that straddles
+// the tile start).
+template <typename RowT, typename LabT>
+__global__ void __launch_bounds__(QT_THREADS) edge_cut_tiles(const RowT *__restrict__ rowptr,
+                                                             const int32_t *__restrict__ colidx, int64_t nnz,
+                                                             const LabT *__restrict__ lab, int64_t N,
+                                                             const int32_t *__restrict__ tile_row, int64_t ntiles,
+                                                             unsigned long long *edge_cut, int *status) {
+    __shared__ unsigned bitmap[QT_WORDS];
+    __shared__ int lasthead[QT_WORDS];
+    __shared__ LabT headlab[QT_EDGES];
+    __shared__ int warp_max[QT_THREADS / 32];
+    __shared__ unsigned long long block_cut;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) block_cut = 0ull;
+    unsigned long long my_cut = 0ull;
+
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t e0 = tile * QT_EDGES;
+        const int ne = (int)min((int64_t)QT_EDGES, nnz - e0);
+        const int4 *src = reinterpret_cast<const int4 *>(colidx + e0);
+        // issue this tile's column loads first: they do not depend on anything below
+        int4 c[QT_VEC];
+#pragma unroll
+        for (int i = 0; i < QT_VEC; ++i) {
+            const int q = (i * QT_THREADS + tid) * 4;
+            if (q + 3 < ne) {
+                c[i] = __ldcs(src + (q >> 2));
+            } else {
+                c[i].x = q + 0 < ne ? colidx[e0 + q + 0] : -1;
+                c[i].y = q + 1 < ne ? colidx[e0 + q + 1] : -1;
+                c[i].z = q + 2 < ne ? colidx[e0 + q + 2] : -1;
+                c[i].w = -1;
+            }
+        }
+        __syncthreads();                                    // previous tile fully consumed
+        bitmap[tid] = 0u;
+        __syncthreads();
+        const int64_t r_lo = tile_row[tile], r_hi = tile_row[tile + 1];
+        const LabT carry = lab[r_lo];
+        for (int64_t r = r_lo + tid; r <= r_hi; r += QT_THREADS) {
+            const int64_t s = (int64_t)rowptr[r], e = (int64_t)rowptr[r + 1];
+            const int64_t h = s - e0;
+            if (e > s && h >= 0 && h < ne) {
+                atomicOr(&bitmap[h >> 5], 1u << (h & 31));
+                headlab[h] = lab[r];
+            }
+        }
+        __syncthreads();
+        {   // lasthead[w] = position of the last set bit in words < w, or -1
+            const unsigned wbits = bitmap[tid];
+            const int mine = wbits ? tid * 32 + 31 - __clz(wbits) : -1;
+            int inc = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(FULL, inc, o);
+                if (lane >= o) inc = max(inc, t);
+            }
+            if (lane == 31) warp_max[warp] = inc;
+            int excl = __shfl_up_sync(FULL, inc, 1);
+            if (lane == 0) excl = -1;
+            __syncthreads();
+            for (int w = 0; w < warp; ++w) excl = max(excl, warp_max[w]);
+            lasthead[tid] = excl;
+        }
+        __syncthreads();
+        unsigned cut = 0;
+#pragma unroll
+        for (int i = 0; i < QT_VEC; ++i) {
+            const int q = (i * QT_THREADS + tid) * 4;
+            if (q < ne) {
+                const int wd = q >> 5, b = q & 31;
+                const unsigned bits = bitmap[wd];
+                const unsigned upto = bits & (0xffffffffu >> (31 - b));
+                const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
+                LabT cur = head >= 0 ? headlab[head] : carry;
+                const int cols[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (j > 0 && ((bits >> (b + j)) & 1u)) cur = headlab[q + j];
+                    if (q + j < ne) {
+                        const int col = cols[j];
+                        if ((unsigned)col < (unsigned)N)
+                            cut += (__ldg(lab + col) != cur) ? 1u : 0u;
+                        else
+                            ep_raise(status, EP_ERR_BAD_INDEX);
+                    }
+                }
+            }
+        }
+        my_cut += cut;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) my_cut += __shfl_xor_sync(FULL, my_cut, o);
+    __syncthreads();
+    if (lane == 0 && my_cut) atomicAdd(&block_cut, my_cut);
+    __syncthreads();
+    if (tid == 0 && block_cut) atomicAdd(edge_cut, block_cut);
+}
+
+template <typename LabT>
+size_t lab_bytes(int64_t N) { return (size_t)N * sizeof(LabT); }
+
+}  // namespace
+
+namespace ep {
+
+static inline int label_width(int K) { return K <= 256 ? 1 : K <= 65536 ? 2 : 4; }
+
+struct QualityBuffers {
+    void *lab;
+    int32_t *tile_row;
+};
+
+static size_t quality_layout(int64_t N, int64_t nnz, int K, void *ws, QualityBuffers *out) {
+    Arena a(ws);
+    QualityBuffers b{};
+    b.lab = a.take<char>((size_t)N * label_width(K));
+    b.tile_row = a.take<int32_t>(ceil_div(nnz, QT_EDGES) + 1);
+    if (out) *out = b;
+    return a.used;
+}
+
+size_t quality_workspace_bytes(int64_t N, int64_t nnz, int K) { return quality_layout(N, nnz, K, nullptr, nullptr); }
+
+template <typename RowT, typename LabT>
+static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx, int64_t nnz, const int32_t *assign,
+                          int64_t N, int K, unsigned long long *edge_cut, unsigned long long *pv,
+                          unsigned long long *pe, const QualityBuffers &b, cudaStream_t stream) {
+    LabT *lab = static_cast<LabT *>(b.lab);
+    const int64_t ntiles = ceil_div(nnz, QT_EDGES);
+    const int pgrid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(N, 256)));
+    {
+        Timed tm(ctx, stream, EP_TIMER_QUALITY_PREP);
+        pack_labels_and_loads<RowT, LabT><<<pgrid, 256, 0, stream>>>(rowptr, assign, N, nnz, K, lab, pv, pe, ctx->d_status);
+        if (ntiles > 0)
+            tile_start_rows<RowT><<<(unsigned)ceil_div(ntiles + 1, 256), 256, 0, stream>>>(rowptr, N, ntiles, b.tile_row);
+        tm.end(ntiles > 0 ? 2 : 1);
+    }
+    if (ntiles > 0) {
+        Timed tm(ctx, stream, EP_TIMER_EDGE_CUT);
+        const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
+        edge_cut_tiles<RowT, LabT><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
+                                                                   edge_cut, ctx->d_status);
+        tm.end(1);
+    }
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
+}
+
+int quality_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *colidx, int64_t nnz,
+                const int32_t *assign, int64_t N, int K, unsigned long long *edge_cut, long long *part_vertices,
+                long long *part_edges, void *workspace, cudaStream_t stream) {
+    QualityBuffers b;
+    quality_layout(N, nnz, K, workspace, &b);
+    EP_CUDA(ctx, cudaMemsetAsync(edge_cut, 0, sizeof(unsigned long long), stream));
+    EP_CUDA(ctx, cudaMemsetAsync(part_vertices, 0, sizeof(long long) * K, stream));
+    EP_CUDA(ctx, cudaMemsetAsync(part_edges, 0, sizeof(long long) * K, stream));
+    auto *pv = reinterpret_cast<unsigned long long *>(part_vertices);
+    auto *pe = reinterpret_cast<unsigned long long *>(part_edges);
+    const int w = label_width(K);
+#define EP_Q(RowT, LabT) \
+    return quality_launch<RowT, LabT>(ctx, static_cast<const RowT *>(rowptr), colidx, nnz, assign, N, K, edge_cut, pv, pe, b, stream)
+    if (rowptr64) {
+        if (w == 1) EP_Q(int64_t, uint8_t);
+        if (w == 2) EP_Q(int64_t, uint16_t);
+        EP_Q(int64_t, int32_t);
+    } else {
+        if (w == 1) EP_Q(int32_t, uint8_t);
+        if (w == 2) EP_Q(int32_t, uint16_t);
+        EP_Q(int32_t, int32_t);
+    }
+#undef EP_Q
+}
+
+}  // namespace ep

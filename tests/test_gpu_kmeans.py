@@ -1,0 +1,146 @@
+"""GPU parity: ep_kmeans (through the C ABI) against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from parity import assert_centroids_close, assert_labels_match, assert_objective_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2604_01000_b200 as ep
+    c = ep.Context(0)
+    yield c
+    c.check()
+    c.close()
+
+
+def _inputs(w, device="cuda"):
+    emb = synth.embeddings(w, device=device)
+    init = emb[synth.init_centroid_rows(w, device=device)].contiguous()
+    return emb, init
+
+
+def _run_and_compare(ctx, emb, init, K, iters, path="auto", single_steps=True):
+    ctx.set_kmeans_path(path)
+    emb_h = emb.cpu().numpy()
+    init_h = init.cpu().numpy()
+    ref = oracle.kmeans(emb_h, K, iters, init_h)
+    got = ctx.kmeans(emb, K, iters, init, objective=True)
+    torch.cuda.synchronize()
+    ctx.check()
+    a = got.assign.cpu().numpy()
+    assert a.min() >= 0 and a.max() < K
+    prev = oracle.kmeans(emb_h, K, max(iters - 1, 0), init_h).centroids if iters > 0 else init_h.astype(np.float64)
+    flips = assert_labels_match(a, ref, emb_h, prev)
+    assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
+    assert_objective_close(got.objective.cpu().numpy(), ref.objective, emb_h)
+    if single_steps and iters > 1:
+        # pin each step on its own: one GPU iteration from the oracle's C_{t-1} (rounded to fp32)
+        for t in sorted({1, iters // 2, iters - 1}):
+            c_prev = oracle.kmeans(emb_h, K, t, init_h).centroids.astype(np.float32)
+            step_ref = oracle.kmeans(emb_h, K, 1, c_prev)
+            step = ctx.kmeans(emb, K, 1, torch.from_numpy(c_prev).cuda())
+            assert_labels_match(step.assign.cpu().numpy(), step_ref, emb_h, c_prev.astype(np.float64))
+            assert_centroids_close(step.centroids.cpu().numpy(), step_ref.centroids, emb_h)
+    ctx.set_kmeans_path("auto")
+    return flips
+
+
+def test_cfg1_full(ctx):
+    w = synth.WORKLOADS["cfg1"]
+    emb, init = _inputs(w)
+    _run_and_compare(ctx, emb, init, w.K, w.iters)
+
+
+@pytest.mark.parametrize("name,N,iters", [("cfg2", 20_011, 30), ("cfg3", 9_973, 30), ("cfg4", 30_011, 12),
+                                          ("cfg5", 25_013, 8)])
+def test_scaled_configs(ctx, name, N, iters):
+    """The paper-shaped configs at a row count the oracle finishes in seconds: several blocks, ragged tail."""
+    w = synth.scaled(synth.WORKLOADS[name], N)
+    emb, init = _inputs(w)
+    _run_and_compare(ctx, emb, init, w.K, iters)
+
+
+@pytest.mark.parametrize("K,N,d,iters", [(300, 12_007, 128, 3), (1024, 9_001, 64, 2), (4096, 20_003, 128, 2),
+                                         (65, 5_003, 256, 3), (200, 3_001, 512, 2)])
+def test_large_k_label_only_path(ctx, K, N, d, iters):
+    w = synth.scaled(synth.WORKLOADS["cfg4"], N, d=d, K=K)
+    emb, init = _inputs(w)
+    _run_and_compare(ctx, emb, init, K, iters, single_steps=False)
+
+
+@pytest.mark.parametrize("N,d,K", [(1, 4, 1), (2, 8, 2), (33, 4, 3), (257, 1024, 5), (1000, 12, 1), (515, 100, 9),
+                                   (64, 36, 64), (4097, 260, 17), (100, 516, 7)])
+def test_shapes_and_edges(ctx, N, d, K):
+    rng = np.random.default_rng(N * 131 + d)
+    centres = rng.normal(size=(max(K, 2), d)) * 3
+    emb_h = (centres[rng.integers(0, max(K, 2), size=N)] + rng.normal(size=(N, d))).astype(np.float32)
+    init_h = emb_h[rng.permutation(N)[:K]].copy()
+    emb, init = torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+    _run_and_compare(ctx, emb, init, K, 4, single_steps=False)
+
+
+def test_empty_cluster_duplicates_and_ties(ctx):
+    rng = np.random.default_rng(3)
+    base = rng.integers(-4, 5, size=(40, 16)).astype(np.float32)
+    emb_h = np.concatenate([base, base, base[:7]])                 # duplicate rows
+    init_h = np.concatenate([base[:3], base[:1], np.full((1, 16), 1e3, np.float32)])   # centroid 3 duplicates 0; 4 stays empty
+    emb, init = torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+    got = ctx.kmeans(emb, 5, 3, init, objective=True)
+    ref = oracle.kmeans(emb_h, 5, 3, init_h)
+    a = got.assign.cpu().numpy()
+    assert not (a == 4).any()
+    np.testing.assert_array_equal(got.centroids[4].cpu().numpy(), init_h[4])           # kept as it was
+    np.testing.assert_array_equal(a, ref.assign)                   # integer data: ties resolved to the lowest index
+    assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
+    assert_objective_close(got.objective.cpu().numpy(), ref.objective, emb_h)
+
+
+def test_iters_zero_assigns_only(ctx):
+    w = synth.scaled(synth.WORKLOADS["cfg2"], 7_777)
+    emb, init = _inputs(w)
+    got = ctx.kmeans(emb, w.K, 0, init, objective=True)
+    ref = oracle.kmeans(emb.cpu().numpy(), w.K, 0, init.cpu().numpy())
+    assert torch.equal(got.centroids, init)
+    assert_labels_match(got.assign.cpu().numpy(), ref)
+    assert_objective_close(got.objective.cpu().numpy(), ref.objective, emb.cpu().numpy())
+
+
+def test_runs_are_bit_identical_and_resumable(ctx):
+    w = synth.scaled(synth.WORKLOADS["cfg3"], 40_009)
+    emb, init = _inputs(w)
+    a = ctx.kmeans(emb, w.K, 6, init, objective=True)
+    b = ctx.kmeans(emb, w.K, 6, init, objective=True)
+    assert torch.equal(a.assign, b.assign) and torch.equal(a.centroids, b.centroids)
+    assert torch.equal(a.objective, b.objective)
+    first = ctx.kmeans(emb, w.K, 2, init, objective=True)
+    rest = ctx.kmeans(emb, w.K, 4, first.centroids, objective=True)
+    assert torch.equal(rest.assign, a.assign) and torch.equal(rest.centroids, a.centroids)
+    assert torch.equal(torch.cat([first.objective, rest.objective]), a.objective)
+    assert torch.all(a.objective[1:] <= a.objective[:-1] * (1 + 1e-7))               # never increases
+
+
+def test_argument_errors_are_reported_not_faulted(ctx):
+    import paper_2604_01000_b200 as ep
+    emb = torch.zeros((10, 8), device="cuda")
+    with pytest.raises(ep.EmbedPartError):
+        ctx.kmeans(emb, 11, 1, torch.zeros((11, 8), device="cuda"))                    # K > N
+    with pytest.raises(ep.EmbedPartError):
+        ctx.kmeans(torch.zeros((10, 6), device="cuda"), 2, 1, torch.zeros((2, 6), device="cuda"))   # d % 4
+    with pytest.raises(ep.EmbedPartError):
+        ctx.kmeans(emb, 2, -1, torch.zeros((2, 8), device="cuda"))
+    with pytest.raises(ValueError):
+        ctx.kmeans(emb.cpu(), 2, 1, torch.zeros((2, 8), device="cuda"))
+    lib = ep.load_library()
+    import ctypes
+    rc = lib.ep_kmeans(ctx._h, ctypes.c_void_p(emb.data_ptr()), 10, 8, 2, 1, ctypes.c_void_p(emb.data_ptr()),
+                       ctypes.c_void_p(emb.data_ptr()), ctypes.c_void_p(emb.data_ptr()), None, None, 0, None)
+    assert rc == 3                                                                      # EP_ERR_WORKSPACE
+    assert b"workspace" in lib.ep_last_error(ctx._h)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0

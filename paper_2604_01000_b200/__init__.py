@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     ep_kmeans,
     ep_partition_quality,
     ep_reorder,
+    ep_reorder_static,
     library_path,
     load_library,
     EXPORTED_SYMBOLS,

@@ -16,7 +16,7 @@ EXPORTED_SYMBOLS = (
     "ep_get_option", "ep_kmeans_workspace_bytes", "ep_kmeans", "ep_quality_workspace_bytes",
     "ep_partition_quality", "ep_reorder_workspace_bytes", "ep_reorder", "ep_profile_read", "ep_launch_count",
     "ep_kmeans_host_arena_bytes", "ep_kmeans_host", "ep_quality_host_arena_bytes", "ep_partition_quality_host",
-    "ep_reorder_host_arena_bytes", "ep_reorder_host",
+    "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static",
 )
 
 EP_OK = 0
@@ -97,6 +97,8 @@ def load_library() -> ctypes.CDLL:
             lib.ep_reorder_host_arena_bytes.restype = sz
             lib.ep_reorder_host.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
             lib.ep_reorder_host.restype = ctypes.c_int
+            lib.ep_reorder_static.argtypes = [vp, i64, i32, vp, vp, vp, vp]
+            lib.ep_reorder_static.restype = ctypes.c_int
             _lib = lib
     return _lib
 
@@ -361,3 +363,26 @@ def ep_partition_quality(rowptr, colidx, assign, K) -> QualityResult:
 def ep_reorder(assign, K, inverse=True) -> ReorderResult:
     """Partition-ordered permutation (and its inverse)."""
     return default_context(assign.device.index).reorder(assign, K, inverse)
+
+
+REORDER_STATIC_MAX_N = 1 << 22
+REORDER_STATIC_MAX_K = 256
+
+
+def ep_reorder_static(assign, K, inverse=True, status=None) -> ReorderResult:
+    """ep_reorder through the entry point that needs neither a context nor a workspace (its scratch is
+    built into the library); N <= REORDER_STATIC_MAX_N, K <= REORDER_STATIC_MAX_K.  `status`, if given,
+    is a one-element int32 CUDA tensor that receives the device status.  The output tensors are still
+    allocated here by torch: it is the library call that allocates nothing."""
+    lib = load_library()
+    if not assign.is_cuda or assign.dtype != torch.int32 or not assign.is_contiguous():
+        raise ValueError("assign must be a contiguous int32 CUDA tensor")
+    N = assign.numel()
+    perm = torch.empty(N, dtype=torch.int32, device=assign.device)
+    inv = torch.empty(N, dtype=torch.int32, device=assign.device) if inverse else None
+    with torch.cuda.device(assign.device):
+        rc = lib.ep_reorder_static(_dev_ptr(assign), N, K, _dev_ptr(perm), _dev_ptr(inv), _dev_ptr(status),
+                                   ctypes.c_void_p(torch.cuda.current_stream(assign.device).cuda_stream))
+    if rc != EP_OK:
+        raise EmbedPartError(rc, lib.ep_status_string(rc).decode())
+    return ReorderResult(perm, inv)

@@ -4,6 +4,7 @@
 #include "ep_common.cuh"
 
 #include <algorithm>
+#include <mutex>
 
 namespace {
 
@@ -261,3 +262,70 @@ int reorder_run(ep_ctx *ctx, const int32_t *assign, int64_t N, int K, int32_t *p
 }
 
 }  // namespace ep
+
+// ---------------------------------------------------------------------------------------------------
+// ep_reorder_static: the single-pass sort above with its scratch in a device array owned by the
+// library instead of a caller workspace, for callers that cannot obtain device memory themselves.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t STATIC_MAX_N = EP_REORDER_STATIC_MAX_N;
+constexpr int STATIC_MAX_K = EP_REORDER_STATIC_MAX_K;
+constexpr int64_t STATIC_TILES = (STATIC_MAX_N + SORT_TILE - 1) / SORT_TILE;
+constexpr int64_t STATIC_HIST = STATIC_TILES * RADIX;                        // per-tile digit counts
+constexpr int64_t STATIC_TOTALS = (STATIC_HIST + SCAN_TILE - 1) / SCAN_TILE; // one total per scan block
+constexpr int64_t STATIC_HEAD = 64;                                          // status word, padded to 256 bytes
+constexpr int64_t STATIC_WORDS = STATIC_HEAD + STATIC_HIST + (STATIC_TOTALS + 63) / 64 * 64;
+static_assert(STATIC_MAX_K <= RADIX, "the static variant is the one-pass sort");
+
+// About 1 MB in every GPU that loads the library, from load until the process exits.
+static __device__ __align__(256) int32_t g_static_scratch[STATIC_WORDS];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+int32_t *g_static_ptr[STATIC_MAX_DEVICES];   // device address of g_static_scratch on each device, once resolved
+std::mutex g_static_mutex;
+
+}  // namespace
+
+extern "C" int ep_reorder_static(const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
+                                 int32_t *device_status, void *cuda_stream) {
+    if (!assign || !perm) return EP_ERR_INVALID_ARG;
+    if (!ep::aligned(assign, 4) || !ep::aligned(perm, 4) || (inv_perm && !ep::aligned(inv_perm, 4)) ||
+        (device_status && !ep::aligned(device_status, 4)))
+        return EP_ERR_INVALID_ARG;
+    if (N < 1 || K < 1) return EP_ERR_INVALID_ARG;
+    if (N > STATIC_MAX_N || K > STATIC_MAX_K) return EP_ERR_UNSUPPORTED;   // beyond the built-in scratch
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return EP_ERR_UNSUPPORTED;
+    int32_t *base = nullptr;
+    {
+        // g_static_scratch names a host-side handle here, not device memory: the address a kernel may
+        // use has to be asked for, once per device, while that device is current.
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return EP_ERR_CUDA;
+            g_static_ptr[dev] = static_cast<int32_t *>(p);
+        }
+        base = g_static_ptr[dev];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int *status = device_status ? device_status : base;   // the array's first word when the caller wants none
+    int32_t *hist = base + STATIC_HEAD;
+    int32_t *totals = hist + STATIC_HIST;
+
+    const int ntiles = (int)ep::ceil_div(N, SORT_TILE);
+    const int64_t nhist = (int64_t)ntiles * RADIX;
+    const int nscan = (int)ep::ceil_div(nhist, SCAN_TILE);
+    // The array still holds the previous call's counts.  The status word is the only part read before
+    // it is written; every histogram and total this call reads is rewritten by its own kernels first.
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return EP_ERR_CUDA;
+    digit_histogram<<<ntiles, SORT_WARPS * 32, 0, stream>>>(assign, N, 0, ntiles, hist, K, status);
+    scan_tiles<<<nscan, SCAN_THREADS, 0, stream>>>(hist, nhist, totals);
+    scan_totals<<<1, SCAN_THREADS, 0, stream>>>(totals, nscan);
+    scan_add<<<nscan, SCAN_THREADS, 0, stream>>>(hist, nhist, totals);
+    digit_scatter<<<ntiles, SORT_WARPS * 32, 0, stream>>>(assign, nullptr, N, 0, ntiles, hist, nullptr, perm, inv_perm);
+    return cudaGetLastError() == cudaSuccess ? EP_OK : EP_ERR_CUDA;
+}

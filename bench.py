@@ -332,37 +332,55 @@ def main():
     rp_bytes = x["rowptr"].element_size()
     passes = {}
 
-    def add_pass(name, key, unit_count, unit, bytes_per_launch=None, flops_per_launch=None):
+    def add_pass(name, key, units, unit, passes_timed, bytes_per_unit=None, flops_per_unit=None):
+        """One library timer -> rate and roofline.  `units` = rows / entries / vertices one pass handles,
+        `passes_timed` = how many such passes the timed region ran (a pass may be several launches)."""
         tot, n = timers[key]
         if n == 0:
             return
-        per = tot / n * 1e-3
-        e = {"launches_timed": n, "ms_per_launch": per * 1e3, "rate": unit_count / per, "unit": unit}
-        if bytes_per_launch is not None:
-            e["roofline"] = {"bound": "hbm", "achieved": bytes_per_launch / per / 1e9, "peak": hbm, "unit": "GB/s",
-                             "frac": bytes_per_launch / per / 1e9 / hbm, "traffic": None,
-                             "peak_source": peaks["_source"]}
-        if flops_per_launch is not None:
-            e["roofline"] = {"bound": "tensor", "achieved": flops_per_launch / per / 1e12, "peak": tf32_peak,
-                             "unit": "TFLOP/s", "frac": flops_per_launch / per / 1e12 / tf32_peak, "traffic": None,
+        secs = tot * 1e-3
+        work = units * passes_timed
+        e = {"launches_timed": n, "ms_per_launch": tot / n, "ms_per_pass": tot / passes_timed, "rate": work / secs,
+             "unit": unit}
+        if bytes_per_unit is not None:
+            gbs = work * bytes_per_unit / secs / 1e9
+            e["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
+                             "traffic": None, "peak_source": peaks["_source"]}
+        if flops_per_unit is not None:
+            tfs = work * flops_per_unit / secs / 1e12
+            e["roofline"] = {"bound": "tensor", "achieved": tfs, "peak": tf32_peak, "unit": "TFLOP/s",
+                             "frac": tfs / tf32_peak, "traffic": None,
                              "peak_source": peaks["_source"] + " bf16 sustained x nominal tf32/bf16 ratio"}
         e["share_of_step"] = tot / ms
         passes[name] = e
 
-    add_pass(f"kmeans_assign_K{w.K}", (0, "kmeans_assign"), w.N, "rows*iters/s", bytes_per_launch=w.N * (4 * w.d + 4))
-    add_pass(f"kmeans_update_K{w.K}", (0, "kmeans_update"), w.N, "rows*iters/s")
+    S = args.steps
+    tensor_small = timers[(0, "kmeans_resolve")][1] > 0
+    tensor_large = timers[(1, "kmeans_resolve")][1] > 0
+    add_pass(f"kmeans_assign_K{w.K}", (0, "kmeans_assign"), w.N, "rows*iters/s", S * w.iters,
+             bytes_per_unit=4 * w.d + 4)
+    if tensor_small:
+        add_pass(f"kmeans_resolve_K{w.K}", (0, "kmeans_resolve"), w.N, "rows*iters/s", S * w.iters)
+    add_pass(f"kmeans_update_K{w.K}", (0, "kmeans_update"), w.N, "rows*iters/s", S * w.iters)
     if w.reorder_K:
-        add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s",
-                 flops_per_launch=2.0 * w.N * w.reorder_K * w.d)
-        add_pass(f"kmeans_update_K{w.reorder_K}", (1, "kmeans_update"), w.N, "rows*iters/s")
-    add_pass("edge_cut", (0, "edge_cut"), nnz, "edges/s", bytes_per_launch=4 * nnz + rp_bytes * (w.N + 1) + w.N)
-    add_pass("quality_prep", (0, "quality_prep"), w.N, "vertices/s", bytes_per_launch=(4 + rp_bytes) * w.N)
-    add_pass("reorder", (0, "reorder"), w.N, "vertices/s", bytes_per_launch=12 * w.N)
+        if tensor_large:
+            add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s", S * w.reorder_iters,
+                     flops_per_unit=2.0 * w.reorder_K * w.d)
+            add_pass(f"kmeans_resolve_K{w.reorder_K}", (1, "kmeans_resolve"), w.N, "rows*iters/s", S * w.reorder_iters)
+        else:   # CUDA cores: report against the same contraction's flops
+            add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s", S * w.reorder_iters,
+                     flops_per_unit=2.0 * w.reorder_K * w.d)
+        add_pass(f"kmeans_update_K{w.reorder_K}", (1, "kmeans_update"), w.N, "rows*iters/s", S * w.reorder_iters)
+    add_pass("edge_cut", (0, "edge_cut"), nnz, "edges/s", S,
+             bytes_per_unit=(4 * nnz + rp_bytes * (w.N + 1) + w.N) / max(nnz, 1))
+    add_pass("quality_prep", (0, "quality_prep"), w.N, "vertices/s", S, bytes_per_unit=4 + rp_bytes)
+    add_pass("reorder", (0, "reorder"), w.N, "vertices/s", S, bytes_per_unit=12)
     dominant = max((p for p in passes.values() if "roofline" in p), key=lambda p: p["share_of_step"])
     dominant_name = [k for k, v in passes.items() if v is dominant][0]
     roofline = dict(dominant["roofline"])
     roofline["kernel"] = dominant_name
     roofline["ms_per_launch"] = dominant["ms_per_launch"]
+    roofline["ms_per_pass"] = dominant["ms_per_pass"]
 
     # ---- end to end: the same pass through the host-buffer C ABI (uploads and downloads timed) ---------
     e2e = None

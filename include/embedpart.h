@@ -52,18 +52,24 @@ enum {
                                (tcgen05) kernels wherever the shape allows */
     EP_OPT_PROFILE = 2,     /* 1 = bracket the main kernels with CUDA events on the launching stream
                                (read with ep_profile_read); 0 = off (default) */
-    EP_OPT_TIMER_GROUP = 3  /* 0..3: calls made while group g is selected log into timers
+    EP_OPT_TIMER_GROUP = 3, /* 0..3: calls made while group g is selected log into timers
                                g * EP_TIMER_COUNT + timer, so a caller can tell two calls apart */
+    EP_OPT_KMEANS_CAND_MB = 4 /* 1..4096 (default 64): upper bound in MiB of the candidate-key buffer the
+                               tensor-core path keeps in the workspace; rows are processed in chunks that
+                               fit it (never less than one pass of the grid).  Set it before the workspace
+                               query: it changes the answer */
 };
 
 /* Timers kept while EP_OPT_PROFILE is 1. */
 enum {
-    EP_TIMER_KMEANS_ASSIGN = 0,  /* the assign(-and-accumulate) kernel of every Lloyd iteration */
+    EP_TIMER_KMEANS_ASSIGN = 0,  /* the assign(-and-accumulate) kernel of every Lloyd iteration; on the
+                                    tensor-core path the screening kernel (one interval per row chunk) */
     EP_TIMER_KMEANS_UPDATE = 1,  /* everything else of an iteration: grouping, sums, centroid update */
     EP_TIMER_EDGE_CUT = 2,       /* the tiled edge-cut kernel */
     EP_TIMER_QUALITY_PREP = 3,   /* label repacking, partition loads, tile start rows */
     EP_TIMER_REORDER = 4,        /* all kernels of ep_reorder */
-    EP_TIMER_COUNT = 5
+    EP_TIMER_KMEANS_RESOLVE = 5, /* tensor-core path: the fp32 kernel that decides the labels */
+    EP_TIMER_COUNT = 6
 };
 
 typedef struct ep_ctx ep_ctx; /* opaque: device id, device properties, device status word, options */

@@ -23,8 +23,10 @@ EP_OK = 0
 EP_OPT_KMEANS_PATH = 1
 EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
-TIMER_COUNT = 5
-TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4}
+EP_OPT_KMEANS_CAND_MB = 4
+TIMER_COUNT = 6
+TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
+          "kmeans_resolve": 5}
 KMEANS_PATHS = {"auto": 0, "simt": 1, "tensor": 2}
 
 
@@ -176,6 +178,12 @@ class Context:
 
     def set_timer_group(self, group: int):
         rc = self._lib.ep_set_option(self._h, EP_OPT_TIMER_GROUP, group)
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_kmeans_cand_mb(self, mib: int):
+        """Upper bound (MiB) of the tensor-core path's candidate buffer; set before calling kmeans."""
+        rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_CAND_MB, mib)
         if rc != EP_OK:
             self._raise(rc)
 

@@ -87,6 +87,7 @@ int ep_create(ep_ctx **out, int device) {
     ctx->opt_kmeans_path = 0;
     ctx->opt_profile = 0;
     ctx->opt_timer_group = 0;
+    ctx->opt_cand_mb = 64;
     ctx->launches = 0;
     ctx->last_error[0] = 0;
     DeviceGuard g(device);
@@ -137,6 +138,10 @@ int ep_set_option(ep_ctx *ctx, int option, int value) {
         ctx->opt_timer_group = value;
         return EP_OK;
     }
+    if (option == EP_OPT_KMEANS_CAND_MB && value >= 1 && value <= 4096) {
+        ctx->opt_cand_mb = value;
+        return EP_OK;
+    }
     return fail(ctx, EP_ERR_INVALID_ARG, "unknown option %d or value %d", option, value);
 }
 
@@ -152,6 +157,10 @@ int ep_get_option(const ep_ctx *ctx, int option, int *value) {
     }
     if (option == EP_OPT_TIMER_GROUP) {
         *value = ctx->opt_timer_group;
+        return EP_OK;
+    }
+    if (option == EP_OPT_KMEANS_CAND_MB) {
+        *value = ctx->opt_cand_mb;
         return EP_OK;
     }
     return EP_ERR_INVALID_ARG;

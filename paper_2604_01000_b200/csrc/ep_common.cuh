@@ -22,6 +22,7 @@ struct ep_ctx {
     int opt_kmeans_path;   // EP_OPT_KMEANS_PATH
     int opt_profile;       // EP_OPT_PROFILE
     int opt_timer_group;   // EP_OPT_TIMER_GROUP
+    int opt_cand_mb;       // EP_OPT_KMEANS_CAND_MB
     long long launches;    // kernels launched through this context
     std::vector<ep_timed_interval> intervals;   // pending event pairs (profile mode)
     std::vector<cudaEvent_t> spare_events;
@@ -84,6 +85,7 @@ struct KMeansPlan {
     int64_t N;
     int d, K;
     bool fused;        // centroids + per-warp sums live in shared memory, one pass per iteration
+    bool tensor;       // labels come from the tcgen05 screening kernel + fp32 resolve kernel
     int warps;         // warps per block of the assign kernel
     int grid;          // blocks of the assign kernel (fused: also the number of partial sums)
     int parts;         // partial-sum slabs the update kernel reduces (fused: grid; otherwise splits per cluster)
@@ -93,6 +95,15 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
 size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &plan, void *workspace, struct KMeansBuffers *out);
 int kmeans_run(ep_ctx *ctx, const KMeansPlan &plan, const float *emb, int iters, const float *init,
                int32_t *assign, float *centroids, double *objective, void *workspace, cudaStream_t stream);
+
+// ---- k-means on the tensor cores (kmeans_tc.cu) --------------------------------------------------
+struct TcState;                                   // tensor maps of one ep_kmeans call
+bool kmeans_tc_shape_ok(const ep_ctx *ctx, int d, int K);
+size_t kmeans_tc_state_bytes();
+size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K);
+int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st);
+int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K, const float *centroids,
+                     const float *cn, int32_t *assign, void *cand_ws, cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

@@ -2,6 +2,7 @@
 // update and the per-call driver.  A warp owns whole rows; lane l holds the 16-byte slices
 // l, l+32, ... of a row in registers, so a row is read from HBM exactly once, coalesced.
 #include "ep_common.cuh"
+#include "kmeans_device.cuh"
 
 #include <math_constants.h>
 
@@ -10,55 +11,9 @@
 
 namespace {
 
-constexpr int KC = 8;          // centroids reduced together by one butterfly
+using namespace epk;
+
 constexpr int UPD_THREADS = 128;
-constexpr unsigned FULL = 0xffffffffu;
-
-__device__ __forceinline__ float4 ldg_stream(const float4 *p) {
-    float4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
-                 : "l"(p));
-    return r;
-}
-
-__device__ __forceinline__ float dot4(const float4 &a, const float4 &b, float acc) {
-    acc = fmaf(a.x, b.x, acc);
-    acc = fmaf(a.y, b.y, acc);
-    acc = fmaf(a.z, b.z, acc);
-    acc = fmaf(a.w, b.w, acc);
-    return acc;
-}
-
-// Sums 8 per-lane values across the warp with 9 shuffles instead of 40: each exchange halves the
-// number of values a lane still carries.  On return every lane holds the warp-wide total of value
-// index ((lane>>4)&1)*4 + ((lane>>3)&1)*2 + ((lane>>2)&1).
-__device__ __forceinline__ float reduce8_transposed(const float (&a)[KC], int lane) {
-    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
-    float b[4], c[2];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float send = h16 ? a[i] : a[i + 4];
-        float keep = h16 ? a[i + 4] : a[i];
-        b[i] = keep + __shfl_xor_sync(FULL, send, 16);
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        float send = h8 ? b[i] : b[i + 2];
-        float keep = h8 ? b[i + 2] : b[i];
-        c[i] = keep + __shfl_xor_sync(FULL, send, 8);
-    }
-    float send = h4 ? c[0] : c[1];
-    float keep = h4 ? c[1] : c[0];
-    float v = keep + __shfl_xor_sync(FULL, send, 4);
-    v += __shfl_xor_sync(FULL, v, 2);
-    v += __shfl_xor_sync(FULL, v, 1);
-    return v;
-}
-
-__device__ __forceinline__ int lane_chunk_slot(int lane) {
-    return ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-}
 
 template <int VPL, int R>
 struct Rows {
@@ -436,6 +391,8 @@ __global__ void __launch_bounds__(256) objective_finalize(const double *__restri
 }
 
 constexpr int X2_BLOCKS = 1184;
+constexpr int TENSOR_MIN_K = 64;      // from here on the tensor-core path is chosen when the shape allows it
+constexpr int CN_PAD = 256;           // |c|^2 is padded to the tensor path's centroid tile
 
 template <typename F>
 int dispatch_vpl(int d, F &&f) {
@@ -459,6 +416,7 @@ struct KMeansBuffers {
     int64_t *off;
     int32_t *order;
     void *sort_ws;
+    void *cand;        // tensor path: screening keys of one row chunk
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -483,7 +441,9 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
             break;
         }
     }
-    p.fused = W >= 4 && K <= 256;
+    const bool tc_ok = kmeans_tc_shape_ok(ctx, d, K);
+    p.tensor = tc_ok && (ctx->opt_kmeans_path == 2 || (ctx->opt_kmeans_path == 0 && K >= TENSOR_MIN_K));
+    p.fused = !p.tensor && W >= 4 && K <= 256;
     if (p.fused) {
         p.warps = W;
         p.smem = Kpad * row_bytes + (size_t)W * K * row_bytes + Kpad * 4 + (size_t)W * K * 4;
@@ -507,7 +467,7 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
     (void)ctx;
     Arena a(workspace);
     KMeansBuffers b{};
-    b.cnorm = a.take<float>(p.K);
+    b.cnorm = a.take<float>((size_t)ceil_div(p.K, CN_PAD) * CN_PAD);
     b.psum = a.take<float>((size_t)p.parts * p.K * p.d);
     b.pcnt = a.take<int>((size_t)p.parts * p.K);
     b.objterm = a.take<double>(p.K);
@@ -518,6 +478,7 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.order = a.take<int32_t>(p.N);
         b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
     }
+    if (p.tensor) b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
     if (out) *out = b;
     return a.used;
 }
@@ -532,6 +493,15 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
 
     if (centroids != init)
         EP_CUDA(ctx, cudaMemcpyAsync(centroids, init, sizeof(float) * K * d, cudaMemcpyDeviceToDevice, stream));
+    alignas(64) unsigned char tc_state_mem[512];
+    TcState *tc_state = reinterpret_cast<TcState *>(tc_state_mem);
+    if (p.tensor) {
+        if (kmeans_tc_state_bytes() > sizeof(tc_state_mem)) return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
+        int rc = kmeans_tc_prepare(ctx, emb, N, d, K, centroids, tc_state);
+        if (rc != EP_OK) return rc;
+        // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38
+        EP_CUDA(ctx, cudaMemsetAsync(b.cnorm, 0x7F, sizeof(float) * (size_t)ceil_div(K, CN_PAD) * CN_PAD, stream));
+    }
     {
         Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
         centroid_norms<<<K, UPD_THREADS, 0, stream>>>(centroids, d, b.cnorm);
@@ -555,11 +525,14 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
                                                              b.pcnt, rpb, rpw);
                 tm.end(1);
             } else {
-                auto kern = kmeans_assign_chunked<VPL, R>;
-                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
-                const int row_bytes = VPL * 512;
-                int kchunk = (int)std::min<size_t>(Kpad, (96 * 1024) / row_bytes / KC * KC);
-                {
+                if (p.tensor) {
+                    int r1 = kmeans_tc_assign(ctx, *tc_state, emb, N, d, K, centroids, b.cnorm, assign, b.cand, stream);
+                    if (r1 != EP_OK) return r1;
+                } else {
+                    auto kern = kmeans_assign_chunked<VPL, R>;
+                    EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+                    const int row_bytes = VPL * 512;
+                    int kchunk = (int)std::min<size_t>(Kpad, (96 * 1024) / row_bytes / KC * KC);
                     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
                     kern<<<p.grid, 256, p.smem, stream>>>(emb, N, d, K, Kpad, kchunk, centroids, b.cnorm, assign);
                     tm.end(1);

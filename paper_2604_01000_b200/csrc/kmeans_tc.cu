@@ -1,0 +1,516 @@
+// Tensor-core assignment step of Lloyd K-Means (Algorithm 3, line 1) for many centroids.
+//
+// The scores |c_k|^2 - 2 x_i.c_k of a tile of 128 rows against all K centroids are a dense
+// contraction [128 x d].[d x K].  kmeans_tc_screen runs it on the 5th-generation tensor cores in TF32:
+//   - the 128-row tile of X stays in shared memory (TMA, 128-byte swizzle) for all centroid tiles;
+//   - centroid tiles of 256 rows stream through a ring of shared-memory stages (TMA, L2-resident);
+//   - one thread issues tcgen05.mma kind::tf32 into one of two 256-column TMEM accumulators;
+//   - eight epilogue warps read the other accumulator back (tcgen05.ld) and keep, per row and per group
+//     of 128 centroids, the two smallest scores with the column index packed into the low mantissa bits.
+// TF32 keeps 10 mantissa bits of each operand, so these scores only screen.  kmeans_tc_resolve then
+// re-evaluates in fp32 every centroid that the TF32 error bound cannot exclude: the best of each group
+// whose best is within the bound of the row's overall best, and a whole group when its second best is
+// within the bound as well (its hidden third might be).  The label is the exact fp32 argmin with the
+// lowest index winning ties, as on the CUDA-core path.
+#include "ep_common.cuh"
+#include "kmeans_device.cuh"
+
+#include <cuda.h>
+#include <math_constants.h>
+
+#include <algorithm>
+#include <mutex>
+
+namespace {
+
+using namespace epk;
+
+constexpr int BM = 128;                    // rows per tile = TMEM lanes
+constexpr int BN = 256;                    // centroids per accumulator
+constexpr int GROUP = 128;                 // centroids per candidate group: one epilogue warp's columns
+constexpr int KBLK = 32;                   // floats in one 128-byte swizzle row
+constexpr int MAX_KB = 8;                  // d <= 256
+constexpr int MAX_STAGES = 4;
+constexpr int X_KB_BYTES = BM * 128;       // one k-block of the X tile
+constexpr int C_STAGE_BYTES = BN * 128;    // one k-block of a centroid tile
+constexpr int TC_THREADS = 384;            // warp 0 TMA, warp 1 MMA, warp 2 TMEM, warp 3 idle, warps 4..11 epilogue
+constexpr int EPI_WARP0 = 4;
+constexpr int EPI_WARPS = 8;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s: far beyond any legitimate wait
+constexpr uint32_t KEY_INIT = 0x7F7FFFFFu;              // FLT_MAX: above every real key
+constexpr uint32_t IDX_MASK = GROUP - 1;
+
+// UMMA instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128.
+constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((BN >> 3) << 17) | ((BM >> 4) << 24);
+
+struct TcShared {
+    uint64_t x_full[MAX_KB], x_empty[MAX_KB];
+    uint64_t c_full[MAX_STAGES], c_empty[MAX_STAGES];
+    uint64_t t_full[2], t_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Waits for the phase of the given parity, but never for ever: after WAIT_LIMIT_CLOCKS, or once
+// another thread has given up, it sets the block's abort flag and returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    const uint32_t addr = smem_u32(bar);
+    long long t0 = 0;
+    for (uint32_t spins = 0;; ++spins) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (*abort_flag) return false;
+        if (spins == 64) t0 = clock64();
+        if (spins > 64 && (spins & 63) == 0 && clock64() - t0 > WAIT_LIMIT_CLOCKS) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+        : "memory");
+}
+// The barrier receives one arrival when every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Keeps the two smallest keys seen.  A key is a score whose low 7 mantissa bits hold the column's
+// index inside its group, compared as a float, so one min/max pair carries value and index.
+__device__ __forceinline__ void keep_two(float &b1, float &b2, float key) {
+    const float t = fmaxf(key, b1);
+    b1 = fminf(key, b1);
+    b2 = fminf(b2, t);
+}
+
+// Screening pass over the rows [row_begin, row_end): for row r and group g (centroids [128 g, 128 g + 128))
+// cand[(r - row_begin) * G + g] = the two smallest TF32 scores of the group as packed keys.
+// cn holds |c_k|^2 for k < K and a huge finite value up to the next multiple of 256.  key_mask is
+// ~(GROUP - 1); it arrives as an argument so that clearing the index bits and inserting the (compile-
+// time) index stay one three-input logic operation instead of two with an immediate each.
+__global__ void __launch_bounds__(TC_THREADS, 1)
+kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
+                 const float *__restrict__ cn, int64_t row_begin, int64_t row_end, int num_kb, int num_nt, int stages,
+                 int G, uint32_t key_mask, uint2 *__restrict__ cand, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *x_smem = smem;                                         // [num_kb][128 rows][128 B]
+    uint8_t *c_smem = x_smem + (size_t)num_kb * X_KB_BYTES;         // [stages][256 rows][128 B]
+    TcShared *sh = reinterpret_cast<TcShared *>(c_smem + (size_t)stages * C_STAGE_BYTES);
+    volatile int *abort_flag = &sh->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t num_tiles = (row_end - row_begin + BM - 1) / BM;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < MAX_KB; ++i) {
+            mbar_init(&sh->x_full[i], 1);
+            mbar_init(&sh->x_empty[i], 1);
+        }
+        for (int i = 0; i < MAX_STAGES; ++i) {
+            mbar_init(&sh->c_full[i], 1);
+            mbar_init(&sh->c_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh->t_full[i], 1);
+            mbar_init(&sh->t_empty[i], EPI_WARPS);
+        }
+        sh->abort = 0;
+        sh->tmem_base = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
+                const int row0 = (int)(row_begin + tile * BM);
+                for (int nt = 0; ok && nt < num_nt; ++nt) {
+                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                        if (nt == 0) {   // this tile's rows, one k-block at a time, as the previous tile lets go of them
+                            if (!(ok = mbar_wait(&sh->x_empty[kb], (uint32_t)(lt & 1) ^ 1u, abort_flag))) break;
+                            mbar_expect_tx(&sh->x_full[kb], X_KB_BYTES);
+                            tma_load_2d(x_smem + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK, row0, &sh->x_full[kb]);
+                        }
+                        const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
+                        if (!(ok = mbar_wait(&sh->c_empty[s], ph ^ 1u, abort_flag))) break;
+                        mbar_expect_tx(&sh->c_full[s], C_STAGE_BYTES);
+                        tma_load_2d(c_smem + (size_t)s * C_STAGE_BYTES, &map_c, kb * KBLK, nt * BN, &sh->c_full[s]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, acc = 0;
+            bool ok = true;
+            for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
+                for (int nt = 0; ok && nt < num_nt; ++nt, ++acc) {
+                    const uint32_t buf = acc & 1u, use = (acc >> 1) & 1u;
+                    if (!(ok = mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + buf * BN;
+                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                        if (nt == 0 && !(ok = mbar_wait(&sh->x_full[kb], (uint32_t)(lt & 1), abort_flag))) break;
+                        const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
+                        if (!(ok = mbar_wait(&sh->c_full[s], ph, abort_flag))) break;
+                        tc_fence_after();
+                        const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)kb * X_KB_BYTES));
+                        const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)s * C_STAGE_BYTES));
+#pragma unroll
+                        for (int ks = 0; ks < KBLK / 8; ++ks)   // 8 tf32 = 32 bytes per step: +2 in 16-byte units
+                            umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks),
+                                      (kb | ks) != 0 ? 1u : 0u);
+                        umma_commit(&sh->c_empty[s]);
+                        if (nt == num_nt - 1) umma_commit(&sh->x_empty[kb]);
+                    }
+                    if (ok) umma_commit(&sh->t_full[buf]);
+                }
+            }
+        }
+    } else if (warp >= EPI_WARP0) {
+        // ---------------------------------------------------------------- epilogue
+        const int quad = warp & 3;                         // TMEM lanes 32 quad .. 32 quad + 31 belong to this warp
+        const int half = (warp - EPI_WARP0) >> 2;          // which 128 of the accumulator's 256 columns
+        uint32_t acc = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const int64_t row = row_begin + tile * BM + quad * 32 + lane;
+            for (int nt = 0; ok && nt < num_nt; ++nt, ++acc) {
+                const uint32_t buf = acc & 1u, use = (acc >> 1) & 1u;
+                if (!(ok = mbar_wait(&sh->t_full[buf], use, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + half * GROUP;
+                const float *cn_grp = cn + (size_t)nt * BN + half * GROUP;
+                float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
+#pragma unroll
+                for (int c = 0; c < GROUP / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 n4 = __ldg(reinterpret_cast<const float4 *>(cn_grp + c * 32) + q);
+                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float s = fmaf(-2.f, __uint_as_float(v[q * 4 + j]), nn[j]);
+                            const float key =
+                                __uint_as_float((__float_as_uint(s) & key_mask) | (uint32_t)(c * 32 + q * 4 + j));
+                            if (j & 1)
+                                keep_two(b1, b2, key);
+                            else
+                                keep_two(a1, a2, key);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
+                const float k1 = fminf(a1, b1);
+                const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+                if (row < row_end)
+                    cand[(size_t)(row - row_begin) * G + (nt * 2 + half)] = make_uint2(__float_as_uint(k1), __float_as_uint(k2));
+            }
+        }
+    }
+    __syncthreads();
+    if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// Error allowance of a screened score, as a multiple of |x| max_k|c_k| plus a multiple of the largest
+// score magnitude:
+//   operands cut to 10 mantissa bits (each off by < 2^-10 relative): |x.c error| < (2^-9 + 2^-20) |x||c|,
+//     doubled by the factor -2 of the score;
+//   fp32 accumulation of d products inside the tensor core and the final fma: < (d + 2) 2^-23 each way,
+//     counted generously as d 2^-21 |x||c|;
+//   7 mantissa bits overwritten by the index: < 2^-16 of the score itself.
+__device__ __forceinline__ float screen_allowance(float xnorm, float cmax, float cmax2, int d) {
+    const float a = xnorm * cmax;
+    return a * (0.00392f + (float)d * 4.8e-7f) + 1.6e-5f * (cmax2 + 2.f * a);
+}
+
+// Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
+// lane l holds the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.
+template <int VPL>
+__global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin,
+                                                         int64_t row_end, int d, int K, int G,
+                                                         const float *__restrict__ C, const float *__restrict__ cn,
+                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign) {
+    __shared__ float red[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
+    // largest centroid norm (every block recomputes it: K loads)
+    float m2 = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) m2 = fmaxf(m2, cn[k]);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
+    if (lane == 0) red[warp] = m2;
+    __syncthreads();
+    float cmax2 = red[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) cmax2 = fmaxf(cmax2, red[w]);
+    const float cmax = sqrtf(cmax2);
+    const float4 *C4 = reinterpret_cast<const float4 *>(C);
+    const int slot = lane_chunk_slot(lane);
+
+    for (int64_t row = row_begin + (int64_t)blockIdx.x * 8 + warp; row < row_end; row += (int64_t)gridDim.x * 8) {
+        float4 x[VPL];
+        float x2 = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int q = lane + 32 * v;
+            x[v] = q < d4 ? ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x2 = dot4(x[v], x[v], x2);
+        }
+        x2 = warp_sum(x2);
+        const uint2 *cr = cand + (size_t)(row - row_begin) * G;
+        float lo = CUDART_INF_F;
+        for (int g = lane; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
+        const float thr = lo + 2.f * screen_allowance(sqrtf(x2), cmax, cmax2, d);
+
+        float best = CUDART_INF_F;
+        int bidx = 0x7fffffff;
+        for (int g0 = 0; g0 < G; g0 += 32) {
+            const int g = g0 + lane;
+            uint2 key = make_uint2(KEY_INIT, KEY_INIT);
+            if (g < G) key = cr[g];
+            unsigned m1 = __ballot_sync(FULL, __uint_as_float(key.x) <= thr);
+            const unsigned mboth = __ballot_sync(FULL, __uint_as_float(key.y) <= thr);
+            while (m1) {
+                const int src = __ffs(m1) - 1;
+                m1 &= m1 - 1;
+                const int kbase = (g0 + src) * GROUP;
+                const int kone = kbase + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
+                if ((mboth >> src) & 1u) {
+                    // two of this group's centroids cannot be told from the best: score the whole group
+                    const int kend = min(K, kbase + GROUP);
+                    for (int kb = kbase; kb < kend; kb += KC) {
+                        float acc[KC];
+#pragma unroll
+                        for (int kk = 0; kk < KC; ++kk) {
+                            acc[kk] = 0.f;
+                            if (kb + kk < kend) {
+#pragma unroll
+                                for (int v = 0; v < VPL; ++v) {
+                                    const int q = lane + 32 * v;
+                                    if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
+                                }
+                            }
+                        }
+                        const float dot = reduce8_transposed(acc, lane);
+                        const int k = kb + slot;
+                        float s = k < kend ? fmaf(-2.f, dot, cn[k]) : CUDART_INF_F;
+                        s = (s == s) ? s : CUDART_INF_F;
+                        if (s < best || (s == best && k < bidx)) {
+                            best = s;
+                            bidx = k;
+                        }
+                    }
+                } else if (kone < K) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) {
+                        const int q = lane + 32 * v;
+                        if (q < d4) acc = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc);
+                    }
+                    const float dot = warp_sum(acc);
+                    float s = fmaf(-2.f, dot, cn[kone]);
+                    s = (s == s) ? s : CUDART_INF_F;
+                    if (s < best || (s == best && kone < bidx)) {
+                        best = s;
+                        bidx = kone;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            const float ov = __shfl_xor_sync(FULL, best, o);
+            const int oi = __shfl_xor_sync(FULL, bidx, o);
+            if (ov < best || (ov == best && oi < bidx)) {
+                best = ov;
+                bidx = oi;
+            }
+        }
+        if (lane == 0) assign[row] = (bidx >= 0 && bidx < K) ? bidx : 0;   // a row of NaNs still gets a valid label
+    }
+}
+
+// ---- host ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Map over a row-major [rows x d] fp32 matrix whose boxes are `box_rows` rows of one 128-byte k-block.
+bool encode_kblock_map(CUtensorMap *map, const float *base, int64_t rows, int d, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)KBLK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace ep {
+
+struct TcState {
+    CUtensorMap map_x, map_c;
+};
+
+size_t kmeans_tc_state_bytes() { return sizeof(TcState); }
+
+bool kmeans_tc_shape_ok(const ep_ctx *ctx, int d, int K) {
+    (void)K;
+    if (d < KBLK || d > MAX_KB * KBLK) return false;
+    const int num_kb = (d + KBLK - 1) / KBLK;
+    return (size_t)num_kb * X_KB_BYTES + 2 * (size_t)C_STAGE_BYTES + sizeof(TcShared) + 1024 <= (size_t)ctx->smem_optin;
+}
+
+int kmeans_tc_groups(int K) { return (K + BN - 1) / BN * 2; }
+
+int64_t kmeans_tc_chunk_rows(const ep_ctx *ctx, int64_t N, int K) {
+    const int64_t wave = (int64_t)BM * ctx->sm_count;                       // rows one pass of the grid covers
+    const int64_t budget = ((int64_t)ctx->opt_cand_mb << 20) / ((int64_t)kmeans_tc_groups(K) * (int64_t)sizeof(uint2));
+    const int64_t rows = std::max<int64_t>(1, budget / wave) * wave;
+    return std::min<int64_t>(rows, ceil_div(N, BM) * BM);
+}
+
+size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K) {
+    return (size_t)kmeans_tc_chunk_rows(ctx, N, K) * kmeans_tc_groups(K) * sizeof(uint2);
+}
+
+int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st) {
+    if (!encode_kblock_map(&st->map_x, emb, N, d, BM) || !encode_kblock_map(&st->map_c, centroids, K, d, BN))
+        return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
+    return EP_OK;
+}
+
+// One assignment step on the tensor-core path: labels of all N rows against `centroids` / `cn`.
+int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K,
+                     const float *centroids, const float *cn, int32_t *assign, void *cand_ws, cudaStream_t stream) {
+    const int num_kb = (d + KBLK - 1) / KBLK;
+    const int num_nt = (K + BN - 1) / BN;
+    const int G = num_nt * 2;
+    const size_t fixed = (size_t)num_kb * X_KB_BYTES + sizeof(TcShared) + 1024;
+    const int stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / C_STAGE_BYTES);
+    const size_t smem = fixed + (size_t)stages * C_STAGE_BYTES;
+    EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_tc_screen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    uint2 *cand = static_cast<uint2 *>(cand_ws);
+    const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
+    int launches = 0;
+    for (int64_t r0 = 0; r0 < N; r0 += chunk) {
+        const int64_t r1 = std::min(N, r0 + chunk);
+        const int grid = (int)std::min<int64_t>(ctx->sm_count, ceil_div(r1 - r0, BM));
+        {
+            Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
+            kmeans_tc_screen<<<grid, TC_THREADS, smem, stream>>>(st.map_x, st.map_c, cn, r0, r1, num_kb, num_nt, stages, G,
+                                                               ~IDX_MASK, cand, ctx->d_status);
+            tm.end(1);
+        }
+        Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
+        const int rgrid = (int)std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(r1 - r0, 8));
+        if (d <= 128)
+            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cand, assign);
+        else
+            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cand, assign);
+        tm.end(1);
+        launches += 2;
+    }
+    (void)launches;
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
+}
+
+}  // namespace ep

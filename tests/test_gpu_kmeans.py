@@ -74,6 +74,54 @@ def test_large_k_label_only_path(ctx, K, N, d, iters):
     _run_and_compare(ctx, emb, init, K, iters, single_steps=False)
 
 
+@pytest.mark.parametrize("K,N,d,iters", [(2, 1_000, 32, 3), (5, 129, 64, 2), (32, 30_011, 128, 4), (64, 25_013, 128, 3),
+                                         (100, 7_001, 100, 2), (256, 9_973, 256, 2), (257, 6_007, 36, 2),
+                                         (300, 12_007, 128, 3), (1024, 9_001, 64, 2), (4096, 20_003, 128, 2),
+                                         (700, 3_001, 224, 2)])
+def test_tensor_core_path(ctx, K, N, d, iters):
+    """The tcgen05 screening + fp32 resolve path, forced for every shape it accepts: labels must be the
+    exact fp32 argmin, so the same tolerances apply as on the CUDA-core path."""
+    w = synth.scaled(synth.WORKLOADS["cfg4"], N, d=d, K=K)
+    emb, init = _inputs(w)
+    _run_and_compare(ctx, emb, init, K, iters, path="tensor", single_steps=False)
+
+
+def test_tensor_core_path_in_row_chunks(ctx):
+    """A candidate buffer of 1 MiB forces several row chunks per iteration; the result must not change."""
+    w = synth.scaled(synth.WORKLOADS["cfg4"], 60_013, K=2048)
+    emb, init = _inputs(w)
+    ctx.set_kmeans_path("tensor")
+    whole = ctx.kmeans(emb, w.K, 2, init, objective=True)
+    ctx.set_kmeans_cand_mb(1)
+    try:
+        parts = ctx.kmeans(emb, w.K, 2, init, objective=True)
+    finally:
+        ctx.set_kmeans_cand_mb(64)
+        ctx.set_kmeans_path("auto")
+    assert torch.equal(whole.assign, parts.assign) and torch.equal(whole.centroids, parts.centroids)
+    ref = oracle.kmeans(emb.cpu().numpy(), w.K, 2, init.cpu().numpy())
+    prev = oracle.kmeans(emb.cpu().numpy(), w.K, 1, init.cpu().numpy()).centroids
+    assert_labels_match(parts.assign.cpu().numpy(), ref, emb.cpu().numpy(), prev)
+    assert_centroids_close(parts.centroids.cpu().numpy(), ref.centroids, emb.cpu().numpy())
+
+
+def test_tensor_core_path_ties_and_duplicates(ctx):
+    """Integer-valued rows and duplicated centroids: TF32 is exact here, ties must go to the lowest index."""
+    rng = np.random.default_rng(5)
+    base = rng.integers(-4, 5, size=(300, 32)).astype(np.float32)
+    emb_h = np.concatenate([base, base[:77]])
+    init_h = np.concatenate([base[:150], base[:150], np.full((1, 32), 1e3, np.float32)])   # every centroid twice; last stays empty
+    emb, init = torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+    ctx.set_kmeans_path("tensor")
+    try:
+        got = ctx.kmeans(emb, 301, 2, init, objective=True)
+    finally:
+        ctx.set_kmeans_path("auto")
+    ref = oracle.kmeans(emb_h, 301, 2, init_h)
+    np.testing.assert_array_equal(got.assign.cpu().numpy(), ref.assign)
+    assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
+
+
 @pytest.mark.parametrize("N,d,K", [(1, 4, 1), (2, 8, 2), (33, 4, 3), (257, 1024, 5), (1000, 12, 1), (515, 100, 9),
                                    (64, 36, 64), (4097, 260, 17), (100, 516, 7)])
 def test_shapes_and_edges(ctx, N, d, K):

@@ -301,6 +301,7 @@ def main():
     for g in (0, 1):
         for t in ep.binding.TIMERS:
             ctx.profile_read(t, g)
+    ctx.debug_counters()
     ctx.set_profile(True)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -316,6 +317,7 @@ def main():
     ms = start.elapsed_time(stop)
     launches = ctx.launch_count() - launches0
     ctx.set_profile(False)
+    counters = ctx.debug_counters()
     timers = {(g, t): ctx.profile_read(t, g) for g in (0, 1) for t in ep.binding.TIMERS}
     ctx.check()
     if dist is not None:
@@ -424,6 +426,8 @@ def main():
             "edge_cut_edges_per_s": passes.get("edge_cut", {}).get("rate"),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "passes": passes,
+            "tensor_path_resolve": ({"rows": counters[0], "single_evals_per_row": counters[1] / counters[0],
+                                     "group_scans_per_row": counters[2] / counters[0]} if counters[0] else None),
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

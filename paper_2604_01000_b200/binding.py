@@ -16,7 +16,7 @@ EXPORTED_SYMBOLS = (
     "ep_get_option", "ep_kmeans_workspace_bytes", "ep_kmeans", "ep_quality_workspace_bytes",
     "ep_partition_quality", "ep_reorder_workspace_bytes", "ep_reorder", "ep_profile_read", "ep_launch_count",
     "ep_kmeans_host_arena_bytes", "ep_kmeans_host", "ep_quality_host_arena_bytes", "ep_partition_quality_host",
-    "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static",
+    "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static", "ep_debug_counters",
 )
 
 EP_OK = 0
@@ -85,6 +85,8 @@ def load_library() -> ctypes.CDLL:
             lib.ep_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_int64)]
             lib.ep_profile_read.restype = ctypes.c_int
+            lib.ep_debug_counters.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
+            lib.ep_debug_counters.restype = ctypes.c_int
             lib.ep_launch_count.argtypes = [vp]
             lib.ep_launch_count.restype = ctypes.c_int64
             lib.ep_kmeans_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32]
@@ -195,6 +197,14 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return ms.value, n.value
+
+    def debug_counters(self):
+        """The library's 8 diagnostic counters (kept while profiling is on); reading clears them."""
+        out = (ctypes.c_int64 * 8)()
+        rc = self._lib.ep_debug_counters(self._h, out)
+        if rc != EP_OK:
+            self._raise(rc)
+        return list(out)
 
     def launch_count(self) -> int:
         return int(self._lib.ep_launch_count(self._h))

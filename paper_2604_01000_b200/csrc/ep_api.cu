@@ -193,6 +193,15 @@ int ep_profile_read(ep_ctx *ctx, int timer, double *total_ms, int64_t *intervals
 
 int64_t ep_launch_count(const ep_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+int ep_debug_counters(ep_ctx *ctx, int64_t *out) {
+    if (!ctx || !out) return EP_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    EP_CUDA(ctx, cudaDeviceSynchronize());
+    EP_CUDA(ctx, cudaMemcpy(out, ctx->d_status + EP_COUNTER_WORD0, sizeof(int64_t) * EP_COUNTERS, cudaMemcpyDeviceToHost));
+    EP_CUDA(ctx, cudaMemset(ctx->d_status + EP_COUNTER_WORD0, 0, sizeof(int64_t) * EP_COUNTERS));
+    return EP_OK;
+}
+
 // ---------------------------------------------------------------------------------------------- k-means
 size_t ep_kmeans_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K) {
     KMeansPlan plan;

@@ -29,6 +29,11 @@ struct ep_ctx {
     char last_error[256];
 };
 
+// The 256-byte device block behind ep_ctx::d_status: word 0 is the status, the 64-bit diagnostic
+// counters start at this 32-bit word.
+constexpr int EP_COUNTER_WORD0 = 16;
+constexpr int EP_COUNTERS = 8;
+
 namespace ep {
 
 // ---- host helpers ---------------------------------------------------------------------------
@@ -103,7 +108,7 @@ size_t kmeans_tc_state_bytes();
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K);
 int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st);
 int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K, const float *centroids,
-                     const float *cn, int32_t *assign, void *cand_ws, cudaStream_t stream);
+                     const float *cn, const float *clo, int32_t *assign, void *cand_ws, cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

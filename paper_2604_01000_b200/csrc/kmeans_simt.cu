@@ -319,17 +319,37 @@ __device__ __forceinline__ double block_sum_fixed(double v, double *buf) {
     return r;
 }
 
-// |c_k|^2 of the initial centroids (fp64 sum, rounded once).
-__global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__restrict__ C, int d, float *cnorm) {
+// Nearest TF32 value (10 explicit mantissa bits) of an fp32 number, kept in an fp32 container.
+__device__ __forceinline__ float round_to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+// |c_k|^2 of the initial centroids (fp64 sum, rounded once).  When ct is given (tensor-core path) it
+// receives the centroids rounded to TF32 and clo[k] an upper bound of |c_k - ct_k|_2.
+__global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__restrict__ C, int d, float *cnorm,
+                                                              float *__restrict__ ct, float *__restrict__ clo) {
     __shared__ double buf[UPD_THREADS];
     const int k = blockIdx.x;
-    double t = 0.0;
+    double t = 0.0, tl = 0.0;
     for (int j = threadIdx.x; j < d; j += UPD_THREADS) {
-        double c = C[(size_t)k * d + j];
+        const float cf = C[(size_t)k * d + j];
+        const double c = cf;
         t += c * c;
+        if (ct) {
+            const float r = round_to_tf32(cf);
+            ct[(size_t)k * d + j] = r;
+            const double lo = (double)cf - (double)r;
+            tl += lo * lo;
+        }
     }
     t = block_sum_fixed<UPD_THREADS>(t, buf);
-    if (threadIdx.x == 0) cnorm[k] = (float)t;
+    if (ct) tl = block_sum_fixed<UPD_THREADS>(tl, buf);
+    if (threadIdx.x == 0) {
+        cnorm[k] = (float)t;
+        if (clo) clo[k] = (float)(sqrt(tl) * 1.000001);
+    }
 }
 
 // Centroid update, one block per cluster: S_k = sum over the partial slabs (fp64, slab order),
@@ -339,12 +359,13 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__res
 __global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__restrict__ psum,
                                                                const int *__restrict__ pcnt, int parts, int K, int d,
                                                                float *C, float *cnorm, double *objterm,
-                                                               int keep_centroids) {
+                                                               int keep_centroids, float *__restrict__ ct,
+                                                               float *__restrict__ clo) {
     __shared__ double buf[UPD_THREADS];
     const int k = blockIdx.x;
     long long n = 0;
     for (int p = 0; p < parts; ++p) n += pcnt[(size_t)p * K + k];
-    double t_cs = 0.0, t_cc = 0.0, t_nn = 0.0;
+    double t_cs = 0.0, t_cc = 0.0, t_nn = 0.0, t_lo = 0.0;
     for (int j = threadIdx.x; j < d; j += UPD_THREADS) {
         double S = 0.0;
         for (int p = 0; p < parts; ++p) S += (double)psum[((size_t)p * K + k) * d + j];
@@ -355,13 +376,21 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__re
         t_cc += (double)cold * (double)cold;
         t_nn += (double)cnew * (double)cnew;
         C[(size_t)k * d + j] = cnew;
+        if (ct) {   // tensor-core path: the TF32 copy the next screening pass multiplies with
+            const float r = round_to_tf32(cnew);
+            ct[(size_t)k * d + j] = r;
+            const double lo = (double)cnew - (double)r;
+            t_lo += lo * lo;
+        }
     }
+    if (ct) t_lo = block_sum_fixed<UPD_THREADS>(t_lo, buf);
     t_cs = block_sum_fixed<UPD_THREADS>(t_cs, buf);
     t_cc = block_sum_fixed<UPD_THREADS>(t_cc, buf);
     t_nn = block_sum_fixed<UPD_THREADS>(t_nn, buf);
     if (threadIdx.x == 0) {
         cnorm[k] = (float)t_nn;
         objterm[k] = (double)n * t_cc - 2.0 * t_cs;
+        if (clo) clo[k] = (float)(sqrt(t_lo) * 1.000001);
     }
 }
 
@@ -417,6 +446,8 @@ struct KMeansBuffers {
     int32_t *order;
     void *sort_ws;
     void *cand;        // tensor path: screening keys of one row chunk
+    float *ct;         // tensor path: centroids rounded to TF32
+    float *clo;        // tensor path: |c_k - ct_k|
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -478,7 +509,11 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.order = a.take<int32_t>(p.N);
         b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
     }
-    if (p.tensor) b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
+    if (p.tensor) {
+        b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
+        b.ct = a.take<float>((size_t)p.K * p.d);
+        b.clo = a.take<float>(p.K);
+    }
     if (out) *out = b;
     return a.used;
 }
@@ -497,14 +532,14 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     TcState *tc_state = reinterpret_cast<TcState *>(tc_state_mem);
     if (p.tensor) {
         if (kmeans_tc_state_bytes() > sizeof(tc_state_mem)) return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
-        int rc = kmeans_tc_prepare(ctx, emb, N, d, K, centroids, tc_state);
+        int rc = kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
         if (rc != EP_OK) return rc;
         // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38
         EP_CUDA(ctx, cudaMemsetAsync(b.cnorm, 0x7F, sizeof(float) * (size_t)ceil_div(K, CN_PAD) * CN_PAD, stream));
     }
     {
         Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
-        centroid_norms<<<K, UPD_THREADS, 0, stream>>>(centroids, d, b.cnorm);
+        centroid_norms<<<K, UPD_THREADS, 0, stream>>>(centroids, d, b.cnorm, b.ct, b.clo);
         if (objective) sum_of_squares<<<X2_BLOCKS, 256, 0, stream>>>(emb, N * (d / 4), b.x2part);
         tm.end(objective ? 2 : 1);
     }
@@ -526,7 +561,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
                 tm.end(1);
             } else {
                 if (p.tensor) {
-                    int r1 = kmeans_tc_assign(ctx, *tc_state, emb, N, d, K, centroids, b.cnorm, assign, b.cand, stream);
+                    int r1 = kmeans_tc_assign(ctx, *tc_state, emb, N, d, K, centroids, b.cnorm, b.clo, assign, b.cand, stream);
                     if (r1 != EP_OK) return r1;
                 } else {
                     auto kern = kmeans_assign_chunked<VPL, R>;
@@ -552,7 +587,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
         if (rc != EP_OK) return rc;
         Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
         centroid_update<<<K, UPD_THREADS, 0, stream>>>(b.psum, b.pcnt, p.parts, K, d, centroids, b.cnorm, b.objterm,
-                                                       iters == 0 ? 1 : 0);
+                                                       iters == 0 ? 1 : 0, b.ct, b.clo);
         if (objective) objective_finalize<<<1, 256, 0, stream>>>(b.x2part, X2_BLOCKS, b.objterm, K, objective + t);
         tm.end(objective ? 2 : 1);
     }

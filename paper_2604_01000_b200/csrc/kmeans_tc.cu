@@ -290,16 +290,18 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
 }
 
-// Error allowance of a screened score, as a multiple of |x| max_k|c_k| plus a multiple of the largest
-// score magnitude:
-//   operands cut to 10 mantissa bits (each off by < 2^-10 relative): |x.c error| < (2^-9 + 2^-20) |x||c|,
-//     doubled by the factor -2 of the score;
-//   fp32 accumulation of d products inside the tensor core and the final fma: < (d + 2) 2^-23 each way,
-//     counted generously as d 2^-21 |x||c|;
-//   7 mantissa bits overwritten by the index: < 2^-16 of the score itself.
-__device__ __forceinline__ float screen_allowance(float xnorm, float cmax, float cmax2, int d) {
+// Error allowance of a screened score s~ = |c|^2 - 2 fl(x~.c~) against the fp32 score, for a row x and
+// any centroid c.  x~ is what the tensor core makes of x (it drops the low 13 mantissa bits, or rounds:
+// either way |x - x~| <= |x - trunc(x)| element by element), c~ the TF32-rounded copy the update kernel
+// stores.  x.c - x~.c~ = (x - x~).c + x~.(c - c~), so by Cauchy-Schwarz
+//     |x.c - x~.c~| <= xlo * cmax + xnorm * clomax
+// with xlo = |x - trunc(x)|_2 measured on this very row and clomax = max_k |c_k - c~_k|_2 measured on the
+// centroids.  The products x~_j c~_j are exact in fp32; summing d of them and the final fma lose at most
+// (d + 2) 2^-23 of |x||c| each way, allowed for as d 2^-20; overwriting 7 mantissa bits with the index
+// moves a score by < 2^-16 of itself.
+__device__ __forceinline__ float screen_allowance(float xnorm, float xlo, float cmax, float cmax2, float clomax, int d) {
     const float a = xnorm * cmax;
-    return a * (0.00392f + (float)d * 4.8e-7f) + 1.6e-5f * (cmax2 + 2.f * a);
+    return 2.002f * (xlo * cmax + xnorm * clomax) + a * ((float)d * 9.6e-7f) + 1.6e-5f * (cmax2 + 2.f * a);
 }
 
 // Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
@@ -308,39 +310,61 @@ template <int VPL>
 __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin,
                                                          int64_t row_end, int d, int K, int G,
                                                          const float *__restrict__ C, const float *__restrict__ cn,
-                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign) {
-    __shared__ float red[8];
+                                                         const float *__restrict__ clo,
+                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign,
+                                                         unsigned long long *counters) {
+    __shared__ float red[2][8];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
-    // largest centroid norm (every block recomputes it: K loads)
-    float m2 = 0.f;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) m2 = fmaxf(m2, cn[k]);
+    // largest centroid norm and largest rounding residual (every block recomputes them: 2 K loads)
+    float m2 = 0.f, ml = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        m2 = fmaxf(m2, cn[k]);
+        ml = fmaxf(ml, clo[k]);
+    }
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
-    if (lane == 0) red[warp] = m2;
+    for (int o = 16; o >= 1; o >>= 1) {
+        m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
+        ml = fmaxf(ml, __shfl_xor_sync(FULL, ml, o));
+    }
+    if (lane == 0) {
+        red[0][warp] = m2;
+        red[1][warp] = ml;
+    }
     __syncthreads();
-    float cmax2 = red[0];
+    float cmax2 = red[0][0], clomax = red[1][0];
 #pragma unroll
-    for (int w = 1; w < 8; ++w) cmax2 = fmaxf(cmax2, red[w]);
-    const float cmax = sqrtf(cmax2);
+    for (int w = 1; w < 8; ++w) {
+        cmax2 = fmaxf(cmax2, red[0][w]);
+        clomax = fmaxf(clomax, red[1][w]);
+    }
+    const float cmax = sqrtf(cmax2) * 1.000001f;
+    unsigned long long n_single = 0, n_scan = 0, n_rows = 0;
     const float4 *C4 = reinterpret_cast<const float4 *>(C);
     const int slot = lane_chunk_slot(lane);
 
     for (int64_t row = row_begin + (int64_t)blockIdx.x * 8 + warp; row < row_end; row += (int64_t)gridDim.x * 8) {
         float4 x[VPL];
-        float x2 = 0.f;
+        float x2 = 0.f, xl2 = 0.f;
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
             const int q = lane + 32 * v;
             x[v] = q < d4 ? ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
             x2 = dot4(x[v], x[v], x2);
+            const float4 r = make_float4(x[v].x - __uint_as_float(__float_as_uint(x[v].x) & 0xFFFFE000u),
+                                         x[v].y - __uint_as_float(__float_as_uint(x[v].y) & 0xFFFFE000u),
+                                         x[v].z - __uint_as_float(__float_as_uint(x[v].z) & 0xFFFFE000u),
+                                         x[v].w - __uint_as_float(__float_as_uint(x[v].w) & 0xFFFFE000u));
+            xl2 = dot4(r, r, xl2);
         }
         x2 = warp_sum(x2);
+        xl2 = warp_sum(xl2);
+        ++n_rows;
         const uint2 *cr = cand + (size_t)(row - row_begin) * G;
         float lo = CUDART_INF_F;
         for (int g = lane; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
-        const float thr = lo + 2.f * screen_allowance(sqrtf(x2), cmax, cmax2, d);
+        const float thr = lo + 2.f * screen_allowance(sqrtf(x2) * 1.000001f, sqrtf(xl2) * 1.000001f, cmax, cmax2, clomax, d);
 
         float best = CUDART_INF_F;
         int bidx = 0x7fffffff;
@@ -357,6 +381,7 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                 const int kone = kbase + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
                 if ((mboth >> src) & 1u) {
                     // two of this group's centroids cannot be told from the best: score the whole group
+                    ++n_scan;
                     const int kend = min(K, kbase + GROUP);
                     for (int kb = kbase; kb < kend; kb += KC) {
                         float acc[KC];
@@ -381,6 +406,7 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                         }
                     }
                 } else if (kone < K) {
+                    ++n_single;
                     float acc = 0.f;
 #pragma unroll
                     for (int v = 0; v < VPL; ++v) {
@@ -407,6 +433,11 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
             }
         }
         if (lane == 0) assign[row] = (bidx >= 0 && bidx < K) ? bidx : 0;   // a row of NaNs still gets a valid label
+    }
+    if (counters && lane == 0) {
+        atomicAdd(&counters[0], n_rows);
+        atomicAdd(&counters[1], n_single);
+        atomicAdd(&counters[2], n_scan);
     }
 }
 
@@ -479,7 +510,8 @@ int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, co
 
 // One assignment step on the tensor-core path: labels of all N rows against `centroids` / `cn`.
 int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K,
-                     const float *centroids, const float *cn, int32_t *assign, void *cand_ws, cudaStream_t stream) {
+                     const float *centroids, const float *cn, const float *clo, int32_t *assign, void *cand_ws,
+                     cudaStream_t stream) {
     const int num_kb = (d + KBLK - 1) / KBLK;
     const int num_nt = (K + BN - 1) / BN;
     const int G = num_nt * 2;
@@ -501,10 +533,12 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
         }
         Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
         const int rgrid = (int)std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(r1 - r0, 8));
+        unsigned long long *counters =
+            ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
         if (d <= 128)
-            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cand, assign);
+            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, clo, cand, assign, counters);
         else
-            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cand, assign);
+            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, clo, cand, assign, counters);
         tm.end(1);
         launches += 2;
     }

@@ -91,6 +91,7 @@ struct KMeansPlan {
     int d, K;
     bool fused;        // centroids + per-warp sums live in shared memory, one pass per iteration
     bool tensor;       // labels come from the tcgen05 screening kernel + fp32 resolve kernel
+    bool tc_fused;     // few centroids: one tcgen05 kernel assigns and accumulates (implies tensor)
     int warps;         // warps per block of the assign kernel
     int grid;          // blocks of the assign kernel (fused: also the number of partial sums)
     int parts;         // partial-sum slabs the update kernel reduces (fused: grid; otherwise splits per cluster)
@@ -103,12 +104,26 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &plan, const float *emb, int iters,
 
 // ---- k-means on the tensor cores (kmeans_tc.cu) --------------------------------------------------
 struct TcState;                                   // tensor maps of one ep_kmeans call
+// Tensor map (128-byte swizzle) over a row-major [rows x d] fp32 matrix with boxes of box_rows x 32 floats;
+// `map` points at a CUtensorMap.
+bool tc_encode_kblock_map(void *map, const float *base, int64_t rows, int d, int box_rows);
 bool kmeans_tc_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tc_state_bytes();
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K);
 int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st);
 int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K, const float *centroids,
                      const float *cn, const float *clo, int32_t *assign, void *cand_ws, cudaStream_t stream);
+
+// ---- fused tensor-core pass for few centroids (kmeans_tc_fused.cu) --------------------------------
+struct TcFusedState;
+bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K);
+size_t kmeans_tcf_state_bytes();
+int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N);
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
+                       TcFusedState *st, cudaStream_t stream);
+int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
+                      const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
+                      cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(256) objective_finalize(const double *__restri
 }
 
 constexpr int X2_BLOCKS = 1184;
-constexpr int TENSOR_MIN_K = 64;      // from here on the tensor-core path is chosen when the shape allows it
+constexpr int TENSOR_MIN_K = 24;      // from here on the tensor-core path is chosen when the shape allows it
 constexpr int CN_PAD = 256;           // |c|^2 is padded to the tensor path's centroid tile
 
 template <typename F>
@@ -448,6 +448,7 @@ struct KMeansBuffers {
     void *cand;        // tensor path: screening keys of one row chunk
     float *ct;         // tensor path: centroids rounded to TF32
     float *clo;        // tensor path: |c_k - ct_k|
+    float2 *rownorm;   // fused tensor path: (|x_i|, |x_i - trunc(x_i)|)
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -472,10 +473,17 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
             break;
         }
     }
-    const bool tc_ok = kmeans_tc_shape_ok(ctx, d, K);
-    p.tensor = tc_ok && (ctx->opt_kmeans_path == 2 || (ctx->opt_kmeans_path == 0 && K >= TENSOR_MIN_K));
+    const bool tc_ok = kmeans_tc_shape_ok(ctx, d, K), tcf_ok = kmeans_tcf_shape_ok(ctx, d, K);
+    const bool want_tc = ctx->opt_kmeans_path == 2 || (ctx->opt_kmeans_path == 0 && K >= TENSOR_MIN_K);
+    p.tc_fused = tcf_ok && want_tc;
+    p.tensor = (tc_ok && want_tc) || p.tc_fused;
     p.fused = !p.tensor && W >= 4 && K <= 256;
-    if (p.fused) {
+    if (p.tc_fused) {
+        p.warps = 12;
+        p.smem = 0;
+        p.grid = kmeans_tcf_grid(ctx, N);
+        p.parts = p.grid;
+    } else if (p.fused) {
         p.warps = W;
         p.smem = Kpad * row_bytes + (size_t)W * K * row_bytes + Kpad * 4 + (size_t)W * K * 4;
         const int64_t step = (int64_t)W * rows_per_step(vpl);
@@ -503,14 +511,17 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
     b.pcnt = a.take<int>((size_t)p.parts * p.K);
     b.objterm = a.take<double>(p.K);
     b.x2part = a.take<double>(X2_BLOCKS);
-    if (!p.fused) {
+    if (!p.fused && !p.tc_fused) {
         b.hist = a.take<unsigned long long>(p.K);
         b.off = a.take<int64_t>(p.K + 1);
         b.order = a.take<int32_t>(p.N);
         b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
     }
     if (p.tensor) {
-        b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
+        if (p.tc_fused)
+            b.rownorm = a.take<float2>(p.N);
+        else
+            b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
         b.ct = a.take<float>((size_t)p.K * p.d);
         b.clo = a.take<float>(p.K);
     }
@@ -530,9 +541,12 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
         EP_CUDA(ctx, cudaMemcpyAsync(centroids, init, sizeof(float) * K * d, cudaMemcpyDeviceToDevice, stream));
     alignas(64) unsigned char tc_state_mem[512];
     TcState *tc_state = reinterpret_cast<TcState *>(tc_state_mem);
+    TcFusedState *tcf_state = reinterpret_cast<TcFusedState *>(tc_state_mem);
     if (p.tensor) {
-        if (kmeans_tc_state_bytes() > sizeof(tc_state_mem)) return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
-        int rc = kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
+        if (std::max(kmeans_tc_state_bytes(), kmeans_tcf_state_bytes()) > sizeof(tc_state_mem))
+            return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
+        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, b.ct, b.rownorm, tcf_state, stream)
+                            : kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
         if (rc != EP_OK) return rc;
         // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38
         EP_CUDA(ctx, cudaMemsetAsync(b.cnorm, 0x7F, sizeof(float) * (size_t)ceil_div(K, CN_PAD) * CN_PAD, stream));
@@ -549,7 +563,10 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
         int rc = dispatch_vpl(d, [&](auto vpl_c) -> int {
             constexpr int VPL = decltype(vpl_c)::value;
             constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
-            if (p.fused) {
+            if (p.tc_fused) {
+                return kmeans_tcf_assign(ctx, *tcf_state, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
+                                         b.pcnt, stream);
+            } else if (p.fused) {
                 auto kern = kmeans_assign_fused<VPL, R>;
                 EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
                 int64_t rpw = ceil_div(ceil_div(N, p.grid), p.warps);

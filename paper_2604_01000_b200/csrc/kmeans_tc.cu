@@ -14,6 +14,7 @@
 // lowest index winning ties, as on the CUDA-core path.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
+#include "tc_device.cuh"
 
 #include <cuda.h>
 #include <math_constants.h>
@@ -24,6 +25,7 @@
 namespace {
 
 using namespace epk;
+using namespace eptc;
 
 constexpr int BM = 128;                    // rows per tile = TMEM lanes
 constexpr int BN = 256;                    // centroids per accumulator
@@ -37,12 +39,8 @@ constexpr int TC_THREADS = 384;            // warp 0 TMA, warp 1 MMA, warp 2 TME
 constexpr int EPI_WARP0 = 4;
 constexpr int EPI_WARPS = 8;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s: far beyond any legitimate wait
-constexpr uint32_t KEY_INIT = 0x7F7FFFFFu;              // FLT_MAX: above every real key
-constexpr uint32_t IDX_MASK = GROUP - 1;
 
-// UMMA instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128.
-constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((BN >> 3) << 17) | ((BM >> 4) << 24);
+constexpr uint32_t IDESC = umma_idesc_tf32_m128(BN);
 
 struct TcShared {
     uint64_t x_full[MAX_KB], x_empty[MAX_KB];
@@ -51,93 +49,6 @@ struct TcShared {
     uint32_t tmem_base;
     int abort;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Waits for the phase of the given parity, but never for ever: after WAIT_LIMIT_CLOCKS, or once
-// another thread has given up, it sets the block's abort flag and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    const uint32_t addr = smem_u32(bar);
-    long long t0 = 0;
-    for (uint32_t spins = 0;; ++spins) {
-        uint32_t ok;
-        asm volatile(
-            "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-            "selp.u32 %0, 1, 0, p;\n}"
-            : "=r"(ok)
-            : "r"(addr), "r"(parity)
-            : "memory");
-        if (ok) return true;
-        if (*abort_flag) return false;
-        if (spins == 64) t0 = clock64();
-        if (spins > 64 && (spins & 63) == 0 && clock64() - t0 > WAIT_LIMIT_CLOCKS) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
-// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-           (2ull << 61);
-}
-
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
-        : "memory");
-}
-// The barrier receives one arrival when every tcgen05.mma issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// 32 consecutive accumulator columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Keeps the two smallest keys seen.  A key is a score whose low 7 mantissa bits hold the column's
-// index inside its group, compared as a float, so one min/max pair carries value and index.
-__device__ __forceinline__ void keep_two(float &b1, float &b2, float key) {
-    const float t = fmaxf(key, b1);
-    b1 = fminf(key, b1);
-    b2 = fminf(b2, t);
-}
 
 // Screening pass over the rows [row_begin, row_end): for row r and group g (centroids [128 g, 128 g + 128))
 // cand[(r - row_begin) * G + g] = the two smallest TF32 scores of the group as packed keys.
@@ -228,7 +139,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)s * C_STAGE_BYTES));
 #pragma unroll
                         for (int ks = 0; ks < KBLK / 8; ++ks)   // 8 tf32 = 32 bytes per step: +2 in 16-byte units
-                            umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks),
+                            umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), IDESC,
                                       (kb | ks) != 0 ? 1u : 0u);
                         umma_commit(&sh->c_empty[s]);
                         if (nt == num_nt - 1) umma_commit(&sh->x_empty[kb]);
@@ -288,20 +199,6 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
-}
-
-// Error allowance of a screened score s~ = |c|^2 - 2 fl(x~.c~) against the fp32 score, for a row x and
-// any centroid c.  x~ is what the tensor core makes of x (it drops the low 13 mantissa bits, or rounds:
-// either way |x - x~| <= |x - trunc(x)| element by element), c~ the TF32-rounded copy the update kernel
-// stores.  x.c - x~.c~ = (x - x~).c + x~.(c - c~), so by Cauchy-Schwarz
-//     |x.c - x~.c~| <= xlo * cmax + xnorm * clomax
-// with xlo = |x - trunc(x)|_2 measured on this very row and clomax = max_k |c_k - c~_k|_2 measured on the
-// centroids.  The products x~_j c~_j are exact in fp32; summing d of them and the final fma lose at most
-// (d + 2) 2^-23 of |x||c| each way, allowed for as d 2^-20; overwriting 7 mantissa bits with the index
-// moves a score by < 2^-16 of itself.
-__device__ __forceinline__ float screen_allowance(float xnorm, float xlo, float cmax, float cmax2, float clomax, int d) {
-    const float a = xnorm * cmax;
-    return 2.002f * (xlo * cmax + xnorm * clomax) + a * ((float)d * 9.6e-7f) + 1.6e-5f * (cmax2 + 2.f * a);
 }
 
 // Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
@@ -441,12 +338,16 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
     }
 }
 
+}  // namespace
+
+namespace ep {
+
 // ---- host ------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn encode_tiled_fn() {
+static EncodeTiledFn encode_tiled_fn() {
     static EncodeTiledFn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
@@ -460,21 +361,20 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // Map over a row-major [rows x d] fp32 matrix whose boxes are `box_rows` rows of one 128-byte k-block.
-bool encode_kblock_map(CUtensorMap *map, const float *base, int64_t rows, int d, int box_rows) {
+bool tc_encode_kblock_map(void *map_out, const float *base, int64_t rows, int d, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    CUtensorMap *map = static_cast<CUtensorMap *>(map_out);
     const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)d * sizeof(float)};
-    const cuuint32_t box[2] = {(cuuint32_t)KBLK, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)32, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
 
-namespace ep {
 
 struct TcState {
     CUtensorMap map_x, map_c;
@@ -503,7 +403,7 @@ size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K) {
 }
 
 int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st) {
-    if (!encode_kblock_map(&st->map_x, emb, N, d, BM) || !encode_kblock_map(&st->map_c, centroids, K, d, BN))
+    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, centroids, K, d, BN))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
     return EP_OK;
 }

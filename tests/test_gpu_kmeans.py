@@ -122,6 +122,29 @@ def test_tensor_core_path_ties_and_duplicates(ctx):
     assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
 
 
+def test_fused_tensor_core_pass_ties_duplicates_and_repeatability(ctx):
+    """K <= 128: the single-kernel tensor-core pass.  Duplicated centroids tie exactly, so those rows must
+    go through its fp32 queue and come out on the lowest index; two runs must agree bit for bit."""
+    rng = np.random.default_rng(6)
+    base = rng.integers(-4, 5, size=(50, 64)).astype(np.float32)
+    emb_h = np.concatenate([base, base, base[:29]] * 3)
+    init_h = np.concatenate([base[:40], base[:40], np.full((1, 64), 1e3, np.float32)])
+    emb, init = torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+    ctx.set_kmeans_path("tensor")
+    try:
+        got = ctx.kmeans(emb, 81, 2, init, objective=True)
+        w = synth.scaled(synth.WORKLOADS["cfg4"], 70_001)
+        e2, i2 = _inputs(w)
+        a = ctx.kmeans(e2, w.K, 5, i2, objective=True)
+        b = ctx.kmeans(e2, w.K, 5, i2, objective=True)
+    finally:
+        ctx.set_kmeans_path("auto")
+    ref = oracle.kmeans(emb_h, 81, 2, init_h)
+    np.testing.assert_array_equal(got.assign.cpu().numpy(), ref.assign)
+    assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
+    assert torch.equal(a.assign, b.assign) and torch.equal(a.centroids, b.centroids) and torch.equal(a.objective, b.objective)
+
+
 @pytest.mark.parametrize("N,d,K", [(1, 4, 1), (2, 8, 2), (33, 4, 3), (257, 1024, 5), (1000, 12, 1), (515, 100, 9),
                                    (64, 36, 64), (4097, 260, 17), (100, 516, 7)])
 def test_shapes_and_edges(ctx, N, d, K):

@@ -119,7 +119,7 @@ struct TcFusedState;
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tcf_state_bytes();
 int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N);
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, float2 *rownorm,
                        TcFusedState *st, cudaStream_t stream);
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
                       const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,

@@ -326,8 +326,14 @@ __device__ __forceinline__ float round_to_tf32(float x) {
     return __uint_as_float(r);
 }
 
-// |c_k|^2 of the initial centroids (fp64 sum, rounded once).  When ct is given (tensor-core path) it
-// receives the centroids rounded to TF32 and clo[k] an upper bound of |c_k - ct_k|_2.
+// What the tensor cores see of a centroid coordinate, and what they miss.  With a TF32 copy (ct given) the
+// copy holds the nearest TF32 value; without one the tensor core itself drops the low 13 mantissa bits.
+__device__ __forceinline__ float tf32_image(float c, bool rounded) {
+    return rounded ? round_to_tf32(c) : __uint_as_float(__float_as_uint(c) & 0xFFFFE000u);
+}
+
+// |c_k|^2 of the initial centroids (fp64 sum, rounded once).  Tensor-core paths also get clo[k], an upper
+// bound of |c_k - image(c_k)|_2, and, when ct is given, the TF32-rounded copy itself.
 __global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__restrict__ C, int d, float *cnorm,
                                                               float *__restrict__ ct, float *__restrict__ clo) {
     __shared__ double buf[UPD_THREADS];
@@ -337,15 +343,15 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__res
         const float cf = C[(size_t)k * d + j];
         const double c = cf;
         t += c * c;
-        if (ct) {
-            const float r = round_to_tf32(cf);
-            ct[(size_t)k * d + j] = r;
+        if (clo) {
+            const float r = tf32_image(cf, ct != nullptr);
+            if (ct) ct[(size_t)k * d + j] = r;
             const double lo = (double)cf - (double)r;
             tl += lo * lo;
         }
     }
     t = block_sum_fixed<UPD_THREADS>(t, buf);
-    if (ct) tl = block_sum_fixed<UPD_THREADS>(tl, buf);
+    if (clo) tl = block_sum_fixed<UPD_THREADS>(tl, buf);
     if (threadIdx.x == 0) {
         cnorm[k] = (float)t;
         if (clo) clo[k] = (float)(sqrt(tl) * 1.000001);
@@ -376,14 +382,14 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__re
         t_cc += (double)cold * (double)cold;
         t_nn += (double)cnew * (double)cnew;
         C[(size_t)k * d + j] = cnew;
-        if (ct) {   // tensor-core path: the TF32 copy the next screening pass multiplies with
-            const float r = round_to_tf32(cnew);
-            ct[(size_t)k * d + j] = r;
+        if (clo) {   // tensor-core paths: what the next screening pass will not see of this centroid
+            const float r = tf32_image(cnew, ct != nullptr);
+            if (ct) ct[(size_t)k * d + j] = r;
             const double lo = (double)cnew - (double)r;
             t_lo += lo * lo;
         }
     }
-    if (ct) t_lo = block_sum_fixed<UPD_THREADS>(t_lo, buf);
+    if (clo) t_lo = block_sum_fixed<UPD_THREADS>(t_lo, buf);
     t_cs = block_sum_fixed<UPD_THREADS>(t_cs, buf);
     t_cc = block_sum_fixed<UPD_THREADS>(t_cc, buf);
     t_nn = block_sum_fixed<UPD_THREADS>(t_nn, buf);
@@ -520,9 +526,10 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
     if (p.tensor) {
         if (p.tc_fused)
             b.rownorm = a.take<float2>(p.N);
-        else
+        else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
-        b.ct = a.take<float>((size_t)p.K * p.d);
+            b.ct = a.take<float>((size_t)p.K * p.d);
+        }
         b.clo = a.take<float>(p.K);
     }
     if (out) *out = b;
@@ -545,7 +552,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     if (p.tensor) {
         if (std::max(kmeans_tc_state_bytes(), kmeans_tcf_state_bytes()) > sizeof(tc_state_mem))
             return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
-        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, b.ct, b.rownorm, tcf_state, stream)
+        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, centroids, b.rownorm, tcf_state, stream)
                             : kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
         if (rc != EP_OK) return rc;
         // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38

@@ -1,20 +1,22 @@
 // Fused assign-and-accumulate pass of Lloyd K-Means (Algorithm 3, line 1) for few centroids
-// (K <= 128, d <= 128) on the tensor cores: one read of the embedding matrix per iteration.
+// (K <= 64, d <= 128) on the tensor cores: one read of the embedding matrix per iteration.
 //
 // A persistent block per SM streams 128-row tiles of X through a ring of shared-memory stages (TMA,
-// 128-byte swizzle).  All K centroids (their TF32-rounded copy) sit in shared memory for the whole
-// launch.  Per tile:
+// 128-byte swizzle).  All K centroids sit in shared memory for the whole launch, in fp32: the tensor
+// core reads their upper 19 bits, the fp32 re-scoring reads all of them.  Three groups of warps work
+// on consecutive tiles at the same time:
 //   1. one thread issues tcgen05.mma kind::tf32: scores [128 x K] into one of two TMEM accumulators;
-//   2. four warps read the accumulator back, one row per thread, and keep the two smallest packed
-//      (score | column) keys.  If the second key is farther from the first than the TF32 error bound
-//      of that row allows, the first is provably the fp32 argmin and becomes the label.  Otherwise the
-//      row is queued;
-//   3. queued rows are scored against all K centroids in fp32 (a warp per row, the row read from the
-//      shared-memory tile) with the lowest index winning ties, exactly as the CUDA-core kernels do;
-//   4. every (cluster, 16-byte column chunk) pair has one owning thread that adds up, in row order,
-//      the tile's rows carrying that label, straight from the shared-memory tile into registers.
-// The block's sums and counts go to psum[block] / pcnt[block] at the end; the order of every addition
-// is fixed by the launch shape, so results repeat bit for bit.
+//   2. the screen group (4 warps, one row per thread) reads the accumulator back and keeps the two
+//      smallest packed (score | column) keys.  If the second is farther from the first than the TF32
+//      error bound of that row allows, the first is provably the fp32 argmin.  Otherwise the thread lists
+//      the centroids within the bound, and the group re-scores those (row, centroid) pairs in fp32 from
+//      the shared-memory tiles, eight pairs per warp step, lowest index winning ties, with the same
+//      summation order as the CUDA-core kernels;
+//   3. the accumulate group (4 warps) adds every row of the tile into the per-cluster sums it keeps in
+//      registers: a warp owns rows, a lane owns columns, the label selects the register by a jump that
+//      is uniform across the warp.  No atomics: the order of every addition is fixed by the launch
+//      shape, so results repeat bit for bit.
+// At the end the accumulate group folds its row groups in order through shared memory into psum[block].
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -33,63 +35,91 @@ constexpr int KBLK = 32;                // floats in one 128-byte swizzle row
 constexpr int MAX_KB = 4;               // d <= 128
 constexpr int X_KB_BYTES = BM * 128;    // one k-block of a row tile
 constexpr int MAX_STAGES = 8;
-constexpr int THREADS = 384;            // warp 0 TMA, warp 1 MMA, warp 2 TMEM alloc, warp 3 idle, warps 4..11 consumers
-constexpr int CONS_WARP0 = 4;
-constexpr int CONS_WARPS = 8;
+constexpr int THREADS = 512;            // warp 0 TMA, 1 MMA, 2 TMEM alloc, 3 idle, 4..7 screen group, 8..15 accumulate group
+constexpr int S_WARP0 = 4;
+constexpr int A_WARP0 = 8;
+constexpr int A_WARPS = 8;
+constexpr int MAX_K = 64;
+constexpr int ROW_CANDS = 8;            // candidates listed per undecided row before it is scored against all K
+constexpr int QUEUE_CAP = BM * ROW_CANDS;
 
 struct FusedShared {
     uint64_t x_full[MAX_STAGES], x_empty[MAX_STAGES];
     uint64_t c_full;
     uint64_t t_full[2], t_empty[2];
+    uint64_t lab_full[2], lab_empty[2];
+    unsigned long long rowbest[BM];     // undecided rows: min over candidates of (ordered fp32 score << 32 | centroid)
     uint32_t tmem_base;
     int abort;
-    int stop[2];       // the abort flag as consumer thread 0 saw it before a tile's first consumer barrier
-    int qn[2];
-    int queue[2][BM];
-    int lab[2][BM];
-    float red[2][8];
+    int stop;                           // the abort flag as screen thread 0 saw it before the tile's first group barrier
+    int qn, fqn;
+    int queue[QUEUE_CAP];               // (row in tile << 8) | centroid
+    int fullq[BM];                      // rows with more than ROW_CANDS candidates
+    int order[2][BM];                   // rows of the tile grouped by label, ascending row inside a label
+    int off[2][MAX_K + 1];              // first position of each label in order[]
+    int wcnt[2][4][MAX_K + 1];          // rows per (screen warp, label); label MAX_K = rows beyond N
+    int cnt[MAX_K];
+    float cn[MAX_K];
+    float red[2][4];
 };
 
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
-// 16-byte chunk q of row r of a swizzled row tile (k-blocks of 128 rows x 128 bytes).
-__device__ __forceinline__ float4 tile_chunk(const uint8_t *xs, int r, int q) {
-    return *reinterpret_cast<const float4 *>(xs + (size_t)(q >> 3) * X_KB_BYTES + r * 128 + (((q & 7) ^ (r & 7)) << 4));
+// Byte offset of 16-byte chunk q of row r in a swizzled tile whose k-blocks are kb_bytes apart.
+__device__ __forceinline__ uint32_t chunk_off(int r, int q, int kb_bytes) {
+    return (uint32_t)((q >> 3) * kb_bytes + r * 128 + (((q & 7) ^ (r & 7)) << 4));
 }
 
-// KPW = clusters per consumer warp (K <= 8 KPW).  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|).
-template <int KPW>
+__device__ __forceinline__ unsigned long long pack_score(float sc, int k) {
+    uint32_t u = __float_as_uint(sc);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);        // unsigned order = float order
+    return ((unsigned long long)u << 32) | (uint32_t)k;
+}
+
+// KMAX = 32 or 64: upper bound of K, 8 accumulate warps each owning KMAX / 8 clusters.
+// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - trunc_tf32(c_k)|.
+template <int KMAX>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
-                const float *__restrict__ C, const float *__restrict__ cn, const float *__restrict__ clo,
-                const float2 *__restrict__ rownorm, int64_t N, int d, int K, int npad, int num_kb, int stages,
-                uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask, int32_t *__restrict__ assign,
-                float *__restrict__ psum, int *__restrict__ pcnt, unsigned long long *counters, int *status) {
+                const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
+                int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
+                int32_t *__restrict__ assign, float *__restrict__ psum, int *__restrict__ pcnt,
+                unsigned long long *counters, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int stage_bytes = num_kb * X_KB_BYTES;
+    const int c_kb_bytes = npad * 128;
     uint8_t *x_smem = smem;                                          // [stages][num_kb][128 rows][128 B]
     uint8_t *c_smem = x_smem + (size_t)stages * stage_bytes;         // [num_kb][npad rows][128 B]
-    FusedShared *sh = reinterpret_cast<FusedShared *>(c_smem + (size_t)num_kb * npad * 128);
+    FusedShared *sh = reinterpret_cast<FusedShared *>(c_smem + (size_t)num_kb * c_kb_bytes);
     volatile int *abort_flag = &sh->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int d4 = d >> 2;
     const int64_t num_tiles = (N + BM - 1) / BM;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_STAGES; ++i) {
             mbar_init(&sh->x_full[i], 1);
-            mbar_init(&sh->x_empty[i], CONS_WARPS);
+            mbar_init(&sh->x_empty[i], A_WARPS);
         }
         mbar_init(&sh->c_full, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh->t_full[i], 1);
             mbar_init(&sh->t_empty[i], 4);
+            mbar_init(&sh->lab_full[i], 4);
+            mbar_init(&sh->lab_empty[i], A_WARPS);
         }
         sh->abort = 0;
+        sh->stop = 0;
         sh->tmem_base = 0;
-        sh->qn[0] = sh->qn[1] = 0;
+        sh->qn = sh->fqn = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int k = threadIdx.x; k < 2 * 4 * (MAX_K + 1); k += blockDim.x) (&sh->wcnt[0][0][0])[k] = 0;
+    for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
+        sh->cnt[k] = 0;
+        sh->cn[k] = k < npad ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
     }
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
@@ -105,9 +135,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            mbar_expect_tx(&sh->c_full, (uint32_t)(num_kb * npad * 128));
+            mbar_expect_tx(&sh->c_full, (uint32_t)(num_kb * c_kb_bytes));
             for (int kb = 0; kb < num_kb; ++kb)
-                tma_load_2d(c_smem + (size_t)kb * npad * 128, &map_c, kb * KBLK, 0, &sh->c_full);
+                tma_load_2d(c_smem + (size_t)kb * c_kb_bytes, &map_c, kb * KBLK, 0, &sh->c_full);
             uint32_t it = 0;
             for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
@@ -132,7 +162,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)npad;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES));
-                    const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)kb * npad * 128));
+                    const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)kb * c_kb_bytes));
 #pragma unroll
                     for (int ks = 0; ks < KBLK / 8; ++ks)
                         umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), idesc,
@@ -141,15 +171,13 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&sh->t_full[buf]);
             }
         }
-    } else if (warp >= CONS_WARP0) {
-        // ---------------------------------------------------------------- consumers
-        const int cw = warp - CONS_WARP0;                  // 0..7
-        const int ctid = threadIdx.x - CONS_WARP0 * 32;    // 0..255
-        const int d4 = d >> 2;
-        // largest centroid norm and rounding residual
-        {
+    } else if (warp >= S_WARP0 && warp < A_WARP0) {
+        // ---------------------------------------------------------------- screen group: one row per thread
+        const int sw = warp - S_WARP0;                     // TMEM lanes 32 sw .. 32 sw + 31
+        const int stid = threadIdx.x - S_WARP0 * 32;       // 0..127 = row in tile
+        {   // largest centroid norm and truncation residual
             float m2 = 0.f, ml = 0.f;
-            for (int k = ctid; k < K; k += 256) {
+            for (int k = stid; k < K; k += 128) {
                 m2 = fmaxf(m2, cn[k]);
                 ml = fmaxf(ml, clo[k]);
             }
@@ -159,170 +187,247 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 ml = fmaxf(ml, __shfl_xor_sync(FULL, ml, o));
             }
             if (lane == 0) {
-                sh->red[0][cw] = m2;
-                sh->red[1][cw] = ml;
+                sh->red[0][sw] = m2;
+                sh->red[1][sw] = ml;
             }
         }
-        consumer_sync();
-        float cmax2 = sh->red[0][0], clomax = sh->red[1][0];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) {
-            cmax2 = fmaxf(cmax2, sh->red[0][w]);
-            clomax = fmaxf(clomax, sh->red[1][w]);
-        }
+        group_sync(1);
+        const float cmax2 = fmaxf(fmaxf(sh->red[0][0], sh->red[0][1]), fmaxf(sh->red[0][2], sh->red[0][3]));
+        const float clomax = fmaxf(fmaxf(sh->red[1][0], sh->red[1][1]), fmaxf(sh->red[1][2], sh->red[1][3]));
         const float cmax = sqrtf(cmax2) * 1.000001f;
-        const float4 *C4 = reinterpret_cast<const float4 *>(C);
         const int slot = lane_chunk_slot(lane);
+        unsigned long long n_rows = 0, n_undecided = 0, n_items = 0, n_full = 0;
+        mbar_wait(&sh->c_full, 0u, abort_flag);            // the fp32 re-scoring below reads the centroid tile
 
-        float4 acc[KPW];
-        int cnt[KPW];
-#pragma unroll
-        for (int i = 0; i < KPW; ++i) {
-            acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            cnt[i] = 0;
-        }
-        unsigned long long n_rows = 0, n_queued = 0;
+        float2 nr_next = make_float2(0.f, 0.f);            // this row's norms, fetched one tile ahead
+        if ((int64_t)blockIdx.x * BM + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BM + stid);
 
         uint32_t it = 0;
         for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-            const uint32_t s = it % (uint32_t)stages;
+            const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u, par = it & 1u;
             const uint8_t *xs = x_smem + (size_t)s * stage_bytes;
-            const int64_t row0 = tile * BM;
-            if (cw < 4) {
-                // ---- one row per thread: the two best screened scores, then label or queue
-                const int r = cw * 32 + lane;
-                const int64_t row = row0 + r;
-                if (mbar_wait(&sh->t_full[buf], use, abort_flag)) {
-                    tc_fence_after();
-                    const uint32_t taddr = tmem_base + ((uint32_t)(cw * 32) << 16) + buf * (uint32_t)npad;
-                    float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
-                    for (int c = 0; c < npad; c += 16) {
-                        uint32_t v[16];
-                        tmem_ld16(taddr + c, v);
+            const int64_t row = tile * BM + stid;
+            const float2 nr = nr_next;
+            {
+                const int64_t nrow = (tile + gridDim.x) * BM + stid;
+                if (nrow < N) nr_next = __ldg(rownorm + nrow);
+            }
+            // Waits that give up leave garbage behind but nothing out of bounds; the group leaves the loop
+            // together after the next barrier.
+            mbar_wait(&sh->lab_empty[par], use ^ 1u, abort_flag);
+            mbar_wait(&sh->t_full[buf], use, abort_flag);
+            mbar_wait(&sh->x_full[s], ph, abort_flag);
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(sw * 32) << 16) + buf * (uint32_t)npad;
+            float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
+            for (int c = 0; c < npad; c += 16) {
+                uint32_t v[16];
+                tmem_ld16(taddr + c, v);
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float4 n4 = __ldg(reinterpret_cast<const float4 *>(cn + c) + q);
-                            const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+                for (int j = 0; j < 16; ++j) {
+                    const float sc = fmaf(-2.f, __uint_as_float(v[j]), sh->cn[c + j]);
+                    const float key = __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + j));
+                    if (j & 1)
+                        keep_two(b1, b2, key);
+                    else
+                        keep_two(a1, a2, key);
+                }
+            }
+            const float k1 = fminf(a1, b1);
+            const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+            const float thr = k1 + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
+            const int i1 = (int)(__float_as_uint(k1) & IDX_MASK);
+            const bool live = row < N;
+            const bool decided = k2 > thr && i1 < K;       // the best screened score cannot be overtaken
+            const bool undecided = live && !decided;
+            if (__any_sync(FULL, undecided)) {
+                // list this row's centroids whose screened score is within the allowance of the best
+                int nc = 0;
+                if (undecided) sh->rowbest[stid] = ~0ull;
+                for (int c = 0; c < npad; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(taddr + c, v);
+                    if (undecided) {
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float sc = fmaf(-2.f, __uint_as_float(v[q * 4 + j]), nn[j]);
-                                const float key = __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + q * 4 + j));
-                                if (j & 1)
-                                    keep_two(b1, b2, key);
-                                else
-                                    keep_two(a1, a2, key);
+                        for (int j = 0; j < 16; ++j) {
+                            const float sc = fmaf(-2.f, __uint_as_float(v[j]), sh->cn[c + j]);
+                            if (sc <= thr && c + j < K) {
+                                if (nc < ROW_CANDS) sh->queue[atomicAdd(&sh->qn, 1)] = (stid << 8) | (c + j);
+                                ++nc;
                             }
                         }
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
-                    const float k1 = fminf(a1, b1);
-                    const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
-                    int label = -1;
-                    if (row < N) {
-                        const float2 nr = __ldg(rownorm + row);
-                        const float thr = k1 + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
-                        const int i1 = (int)(__float_as_uint(k1) & IDX_MASK);
-                        if (k2 > thr && i1 < K) {
-                            label = i1;
-                            assign[row] = i1;
-                        } else {
-                            sh->queue[par][atomicAdd(&sh->qn[par], 1)] = r;   // includes rows whose keys are NaN
-                        }
-                        ++n_rows;
-                    }
-                    sh->lab[par][r] = label;
                 }
-                if (ctid == 0) sh->stop[par] = *abort_flag;
+                if (undecided && (nc > ROW_CANDS || nc == 0)) sh->fullq[atomicAdd(&sh->fqn, 1)] = stid;   // nc == 0: NaN scores
             }
-            consumer_sync();
-            if (sh->stop[par]) break;   // one thread's reading, so all eight warps leave together
-            // ---- queued rows: exact fp32 scores against all K centroids, a warp per row
-            const int qn = sh->qn[par];
-            for (int qi = cw; qi < qn; qi += CONS_WARPS) {
-                const int r = sh->queue[par][qi];
-                const float4 x = lane < d4 ? tile_chunk(xs, r, lane) : make_float4(0.f, 0.f, 0.f, 0.f);
-                float best = CUDART_INF_F;
-                int bidx = 0x7fffffff;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
+            if (stid == 0) sh->stop = *abort_flag;
+            group_sync(1);
+            if (sh->stop) break;
+            // ---- fp32 re-scoring of the listed (row, centroid) pairs, eight per warp step
+            const int qn = min(sh->qn, QUEUE_CAP), fqn = min(sh->fqn, BM);
+            for (int base = sw * KC; base < qn; base += 4 * KC) {
+                float a[KC];
+#pragma unroll
+                for (int kk = 0; kk < KC; ++kk) {
+                    const int item = sh->queue[min(base + kk, qn - 1)];
+                    a[kk] = 0.f;
+                    if (lane < d4) {
+                        const float4 x = *reinterpret_cast<const float4 *>(xs + chunk_off(item >> 8, lane, X_KB_BYTES));
+                        const float4 cc = *reinterpret_cast<const float4 *>(c_smem + chunk_off(item & 255, lane, c_kb_bytes));
+                        a[kk] = dot4(x, cc, 0.f);
+                    }
+                }
+                const float dot = reduce8_transposed(a, lane);
+                if ((lane & 3) == 0 && base + slot < qn) {
+                    const int item = sh->queue[base + slot];
+                    float sc = fmaf(-2.f, dot, sh->cn[item & 255]);
+                    sc = (sc == sc) ? sc : CUDART_INF_F;
+                    atomicMin(&sh->rowbest[item >> 8], pack_score(sc, item & 255));
+                }
+            }
+            // ---- rows with too many candidates: all K centroids
+            for (int fi = sw; fi < fqn; fi += 4) {
+                const int r = sh->fullq[fi];
+                const float4 x = lane < d4 ? *reinterpret_cast<const float4 *>(xs + chunk_off(r, lane, X_KB_BYTES))
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                unsigned long long best = ~0ull;
                 for (int kb = 0; kb < K; kb += KC) {
                     float a[KC];
 #pragma unroll
                     for (int kk = 0; kk < KC; ++kk) {
                         a[kk] = 0.f;
-                        if (kb + kk < K && lane < d4) a[kk] = dot4(x, __ldg(C4 + (size_t)(kb + kk) * d4 + lane), 0.f);
+                        if (kb + kk < K && lane < d4)
+                            a[kk] = dot4(x, *reinterpret_cast<const float4 *>(c_smem + chunk_off(kb + kk, lane, c_kb_bytes)), 0.f);
                     }
                     const float dot = reduce8_transposed(a, lane);
                     const int k = kb + slot;
-                    float sc = k < K ? fmaf(-2.f, dot, cn[k]) : CUDART_INF_F;
-                    sc = (sc == sc) ? sc : CUDART_INF_F;
-                    if (sc < best || (sc == best && k < bidx)) {
-                        best = sc;
-                        bidx = k;
+                    if (k < K) {
+                        float sc = fmaf(-2.f, dot, sh->cn[k]);
+                        sc = (sc == sc) ? sc : CUDART_INF_F;
+                        const unsigned long long p = pack_score(sc, k);
+                        best = p < best ? p : best;
                     }
                 }
-#pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) {
-                    const float ov = __shfl_xor_sync(FULL, best, o);
-                    const int oi = __shfl_xor_sync(FULL, bidx, o);
-                    if (ov < best || (ov == best && oi < bidx)) {
-                        best = ov;
-                        bidx = oi;
-                    }
-                }
-                if (bidx < 0 || bidx >= K) bidx = 0;   // a row of NaNs still gets a valid label
-                if (lane == 0) {
-                    sh->lab[par][r] = bidx;
-                    assign[row0 + r] = bidx;
-                }
-                ++n_queued;
+                if ((lane & 3) == 0) atomicMin(&sh->rowbest[r], best);
             }
-            consumer_sync();
-            if (ctid == 0) sh->qn[par] = 0;
-            // ---- accumulate: warp cw owns clusters cw, cw + 8, ...; lane owns 16-byte chunk `lane`
-            int l[BM / 32];
+            group_sync(1);
+            // ---- final label of this thread's row
+            if (stid == 0) sh->qn = sh->fqn = 0;
+            int label = MAX_K;                             // bucket of the rows beyond N
+            if (live) {
+                label = decided ? i1 : (int)(uint32_t)(sh->rowbest[stid] & 0xffffffffull);
+                if (label < 0 || label >= K) label = 0;    // a row of NaNs still gets a valid label
+                assign[row] = label;
+                ++n_rows;
+                n_undecided += undecided ? 1 : 0;
+            }
+            n_items += (lane == 0 && sw == 0) ? (unsigned long long)qn : 0ull;
+            n_full += (lane == 0 && sw == 0) ? (unsigned long long)fqn : 0ull;
+            // ---- group the tile's rows by label for the accumulate group (a stable counting sort)
+            const unsigned peers = __match_any_sync(FULL, label);
+            if (lane == __ffs(peers) - 1) sh->wcnt[par][sw][label] = __popc(peers);
+            for (int i = stid; i < 4 * (MAX_K + 1); i += 128) (&sh->wcnt[par ^ 1u][0][0])[i] = 0;
+            group_sync(1);
+            if (sw == 0) {   // exclusive prefix over the labels: two labels per lane
+                const int k0 = 2 * lane, k1 = 2 * lane + 1;
+                const int t0 = sh->wcnt[par][0][k0] + sh->wcnt[par][1][k0] + sh->wcnt[par][2][k0] + sh->wcnt[par][3][k0];
+                const int t1 = sh->wcnt[par][0][k1] + sh->wcnt[par][1][k1] + sh->wcnt[par][2][k1] + sh->wcnt[par][3][k1];
+                int inc = t0 + t1;
 #pragma unroll
-            for (int j = 0; j < BM / 32; ++j) l[j] = sh->lab[par][j * 32 + lane];
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int u = __shfl_up_sync(FULL, inc, o);
+                    if (lane >= o) inc += u;
+                }
+                const int ex = inc - t0 - t1;
+                sh->off[par][k0] = ex;
+                sh->off[par][k1] = ex + t0;
+                if (lane == 31) sh->off[par][MAX_K] = inc;
+                sh->cnt[k0] += t0;
+                sh->cnt[k1] += t1;
+            }
+            group_sync(1);
+            if (live) {
+                int pos = sh->off[par][label] + __popc(peers & ((1u << lane) - 1u));
+                for (int w2 = 0; w2 < sw; ++w2) pos += sh->wcnt[par][w2][label];
+                sh->order[par][pos] = stid;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->lab_full[par]);
+        }
+        group_sync(1);
+        for (int k = stid; k < K; k += 128) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[k];
+        if (counters) {
 #pragma unroll
-            for (int i = 0; i < KPW; ++i) {
-                const int k = cw + CONS_WARPS * i;
+            for (int o = 16; o >= 1; o >>= 1) {
+                n_rows += __shfl_xor_sync(FULL, n_rows, o);
+                n_undecided += __shfl_xor_sync(FULL, n_undecided, o);
+            }
+            if (lane == 0) {
+                atomicAdd(&counters[0], n_rows);
+                atomicAdd(&counters[3], n_undecided);
+                atomicAdd(&counters[4], n_items);
+                atomicAdd(&counters[5], n_full);
+            }
+        }
+    } else if (warp >= A_WARP0) {
+        // ---------------------------------------------------------------- accumulate group
+        const int aw = warp - A_WARP0;                     // owns clusters aw, aw + 8, ...
+        const int atid = threadIdx.x - A_WARP0 * 32;
+        constexpr int OWN = KMAX / A_WARPS;
+        const bool has_cols = lane < d4;                   // this lane's 16-byte chunk of a row is chunk `lane`
+        float4 acc[OWN];
+#pragma unroll
+        for (int i = 0; i < OWN; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        uint32_t it = 0;
+        for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+            const uint32_t s = it % (uint32_t)stages;
+            const uint32_t par = it & 1u, use = (it >> 1) & 1u;
+            const uint8_t *xs = x_smem + (size_t)s * stage_bytes;
+            if (!mbar_wait(&sh->lab_full[par], use, abort_flag)) break;
+            if (!mbar_wait(&sh->x_full[s], (it / (uint32_t)stages) & 1u, abort_flag)) break;   // long complete: makes the tile visible here
+#pragma unroll
+            for (int i = 0; i < OWN; ++i) {
+                const int k = aw + A_WARPS * i;
                 if (k < K) {
+                    const int p1 = sh->off[par][k + 1];
+                    for (int p = sh->off[par][k]; p < p1; p += 4) {   // four rows at a time: loads first, adds in row order
+                        float4 x[4];
 #pragma unroll
-                    for (int j = 0; j < BM / 32; ++j) {
-                        unsigned m = __ballot_sync(FULL, l[j] == k);
-                        cnt[i] += __popc(m);
-                        while (m) {
-                            const int r = j * 32 + __ffs(m) - 1;
-                            m &= m - 1;
-                            if (lane < d4) {
-                                const float4 x = tile_chunk(xs, r, lane);
-                                acc[i].x += x.x;
-                                acc[i].y += x.y;
-                                acc[i].z += x.z;
-                                acc[i].w += x.w;
+                        for (int u = 0; u < 4; ++u) {
+                            const int r = sh->order[par][min(p + u, p1 - 1)];
+                            x[u] = has_cols ? *reinterpret_cast<const float4 *>(xs + chunk_off(r, lane, X_KB_BYTES))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (p + u < p1) {
+                                acc[i].x += x[u].x;
+                                acc[i].y += x[u].y;
+                                acc[i].z += x[u].z;
+                                acc[i].w += x[u].w;
                             }
                         }
                     }
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->x_empty[s]);
-        }
-        // ---- publish this block's partial sums and counts
-        float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
-#pragma unroll
-        for (int i = 0; i < KPW; ++i) {
-            const int k = cw + CONS_WARPS * i;
-            if (k < K) {
-                if (lane < d4) out[(size_t)k * d4 + lane] = acc[i];
-                if (lane == 0) pcnt[(size_t)blockIdx.x * K + k] = cnt[i];
+            if (lane == 0) {
+                mbar_arrive(&sh->x_empty[s]);
+                mbar_arrive(&sh->lab_empty[par]);
             }
         }
-        if (counters && lane == 0) {
-            atomicAdd(&counters[0], n_rows);
-            atomicAdd(&counters[3], n_queued);
+        // ---- publish this block's sums: every (cluster, chunk) has exactly one owner
+        float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
+#pragma unroll
+        for (int i = 0; i < OWN; ++i) {
+            const int k = aw + A_WARPS * i;
+            if (k < K && has_cols) out[(size_t)k * d4 + lane] = acc[i];
         }
+        (void)atid;
     }
     __syncthreads();
     if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
@@ -373,7 +478,7 @@ static size_t tcf_fixed_smem(int d, int K) {
 }
 
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K) {
-    if (d < KBLK || d > MAX_KB * KBLK || K < 1 || K > 128) return false;
+    if (d < KBLK || d > MAX_KB * KBLK || K < 1 || K > MAX_K) return false;
     const int num_kb = (d + KBLK - 1) / KBLK;
     return tcf_fixed_smem(d, K) + 2 * (size_t)num_kb * X_KB_BYTES <= (size_t)ctx->smem_optin;
 }
@@ -382,7 +487,7 @@ int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N) {
     return (int)std::max<int64_t>(1, std::min<int64_t>(ctx->sm_count, ceil_div(N, BM)));
 }
 
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, float2 *rownorm,
                        TcFusedState *st, cudaStream_t stream) {
     st->npad = tcf_npad(K);
     st->num_kb = (d + KBLK - 1) / KBLK;
@@ -394,7 +499,7 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)st->npad) cols <<= 1;
     st->tmem_cols = cols;
-    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
+    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, centroids, K, d, st->npad))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
     Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
     row_norms<<<(int)std::min<int64_t>((int64_t)ctx->sm_count * 16, ceil_div(N, 8)), 256, 0, stream>>>(emb, N, d, rownorm);
@@ -403,16 +508,16 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     return EP_OK;
 }
 
-template <int KPW>
-static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
+template <int KMAX>
+static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo,
                       const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
                       cudaStream_t stream) {
-    auto kern = kmeans_tc_fused<KPW>;
+    auto kern = kmeans_tc_fused<KMAX>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
     unsigned long long *counters =
         ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
-    kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, centroids, cn, clo, rownorm, N, d, K, st.npad, st.num_kb,
+    kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, cn, clo, rownorm, N, d, K, st.npad, st.num_kb,
                                               st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK, assign,
                                               psum, pcnt, counters, ctx->d_status);
     tm.end(1);
@@ -424,9 +529,9 @@ static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *centroid
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
                       const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
                       cudaStream_t stream) {
-    if (K <= 32) return tcf_launch<4>(ctx, st, centroids, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
-    if (K <= 64) return tcf_launch<8>(ctx, st, centroids, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
-    return tcf_launch<16>(ctx, st, centroids, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
+    (void)centroids;   // the kernel reads them through the tensor map made by kmeans_tcf_prepare
+    if (K <= 32) return tcf_launch<32>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
+    return tcf_launch<64>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
 }
 
 }  // namespace ep

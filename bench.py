@@ -363,6 +363,11 @@ def main():
              bytes_per_unit=4 * w.d + 4)
     if tensor_small:
         add_pass(f"kmeans_resolve_K{w.K}", (0, "kmeans_resolve"), w.N, "rows*iters/s", S * w.iters)
+        # the assign step as a whole: the fused kernel plus the kernel for the rows it leaves undecided
+        both = timers[(0, "kmeans_assign")][0] + timers[(0, "kmeans_resolve")][0]
+        gbs = w.N * S * w.iters * (4 * w.d + 4) / (both * 1e-3) / 1e9
+        passes[f"kmeans_assign_K{w.K}"]["roofline_with_resolve"] = {"achieved": gbs, "peak": hbm, "unit": "GB/s",
+                                                                    "frac": gbs / hbm}
     add_pass(f"kmeans_update_K{w.K}", (0, "kmeans_update"), w.N, "rows*iters/s", S * w.iters)
     if w.reorder_K:
         if tensor_large:
@@ -426,8 +431,8 @@ def main():
             "edge_cut_edges_per_s": passes.get("edge_cut", {}).get("rate"),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "passes": passes,
-            "tensor_path_resolve": ({"rows": counters[0], "single_evals_per_row": counters[1] / counters[0],
-                                     "group_scans_per_row": counters[2] / counters[0]} if counters[0] else None),
+            "tensor_path_counters": {"rows_screened": counters[0], "large_K_single_evals": counters[1],
+                                     "large_K_group_scans": counters[2], "small_K_rows_left_to_fp32_kernel": counters[3]},
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

@@ -95,8 +95,9 @@ int ep_profile_read(ep_ctx *ctx, int timer, double *total_ms, int64_t *intervals
 /* Number of kernels this context has launched since it was created. */
 int64_t ep_launch_count(const ep_ctx *ctx);
 /* Diagnostic counters kept while EP_OPT_PROFILE is 1; synchronises the device, copies the 8 counters to
- * out [host, 8 x int64] and clears them.  Tensor-core K-Means path: [0] rows resolved, [1] centroids
- * re-evaluated singly in fp32, [2] groups of 128 centroids re-evaluated whole; the rest are reserved. */
+ * out [host, 8 x int64] and clears them.  Tensor-core K-Means paths: [0] rows screened, [1] centroids the
+ * large-K path re-evaluated singly in fp32, [2] groups of 128 centroids it re-evaluated whole, [3] rows the
+ * fused small-K kernel left to the fp32 kernel; the rest are reserved. */
 int ep_debug_counters(ep_ctx *ctx, int64_t *out);
 
 /* --------------------------------------------------------------------------------------------

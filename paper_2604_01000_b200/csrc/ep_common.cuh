@@ -119,11 +119,12 @@ struct TcFusedState;
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tcf_state_bytes();
 int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N);
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, float2 *rownorm,
+int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N);
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
                        TcFusedState *st, cudaStream_t stream);
-int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
-                      const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
-                      cudaStream_t stream);
+int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
+                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
+                      int *pcnt, void *late_list, int *late_count, cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

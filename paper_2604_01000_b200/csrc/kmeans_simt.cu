@@ -455,6 +455,8 @@ struct KMeansBuffers {
     float *ct;         // tensor path: centroids rounded to TF32
     float *clo;        // tensor path: |c_k - ct_k|
     float2 *rownorm;   // fused tensor path: (|x_i|, |x_i - trunc(x_i)|)
+    void *late_list;   // fused tensor path: per screen warp, the rows the screening left undecided (16 bytes each)
+    int *late_count;
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -488,7 +490,7 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
         p.warps = 12;
         p.smem = 0;
         p.grid = kmeans_tcf_grid(ctx, N);
-        p.parts = p.grid;
+        p.parts = 2 * p.grid;   // the fused kernel's slabs, then those of the kernel for the rows it left undecided
     } else if (p.fused) {
         p.warps = W;
         p.smem = Kpad * row_bytes + (size_t)W * K * row_bytes + Kpad * 4 + (size_t)W * K * 4;
@@ -524,12 +526,14 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
     }
     if (p.tensor) {
-        if (p.tc_fused)
+        if (p.tc_fused) {
             b.rownorm = a.take<float2>(p.N);
-        else {
+            b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N) * 4 * p.grid);
+            b.late_count = a.take<int>((size_t)4 * p.grid);
+        } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
-            b.ct = a.take<float>((size_t)p.K * p.d);
         }
+        b.ct = a.take<float>((size_t)p.K * p.d);
         b.clo = a.take<float>(p.K);
     }
     if (out) *out = b;
@@ -552,7 +556,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     if (p.tensor) {
         if (std::max(kmeans_tc_state_bytes(), kmeans_tcf_state_bytes()) > sizeof(tc_state_mem))
             return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
-        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, centroids, b.rownorm, tcf_state, stream)
+        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, b.ct, b.rownorm, tcf_state, stream)
                             : kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
         if (rc != EP_OK) return rc;
         // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38
@@ -571,8 +575,8 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
             constexpr int VPL = decltype(vpl_c)::value;
             constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
             if (p.tc_fused) {
-                return kmeans_tcf_assign(ctx, *tcf_state, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
-                                         b.pcnt, stream);
+                return kmeans_tcf_assign(ctx, *tcf_state, emb, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
+                                         b.pcnt, b.late_list, b.late_count, stream);
             } else if (p.fused) {
                 auto kern = kmeans_assign_fused<VPL, R>;
                 EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));

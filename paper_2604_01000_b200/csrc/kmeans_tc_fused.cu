@@ -1,22 +1,23 @@
 // Fused assign-and-accumulate pass of Lloyd K-Means (Algorithm 3, line 1) for few centroids
 // (K <= 64, d <= 128) on the tensor cores: one read of the embedding matrix per iteration.
 //
-// A persistent block per SM streams 128-row tiles of X through a ring of shared-memory stages (TMA,
-// 128-byte swizzle).  All K centroids sit in shared memory for the whole launch, in fp32: the tensor
-// core reads their upper 19 bits, the fp32 re-scoring reads all of them.  Three groups of warps work
-// on consecutive tiles at the same time:
+// kmeans_tc_fused: a persistent block per SM streams 128-row tiles of X through a ring of shared-memory
+// stages (TMA, 128-byte swizzle).  The TF32-rounded copy of all K centroids sits in shared memory for the
+// whole launch.  Four kinds of warps work on consecutive tiles at the same time, handing tiles on through
+// mbarriers (every wait has a time limit):
 //   1. one thread issues tcgen05.mma kind::tf32: scores [128 x K] into one of two TMEM accumulators;
-//   2. the screen group (4 warps, one row per thread) reads the accumulator back and keeps the two
-//      smallest packed (score | column) keys.  If the second is farther from the first than the TF32
-//      error bound of that row allows, the first is provably the fp32 argmin.  Otherwise the thread lists
-//      the centroids within the bound, and the group re-scores those (row, centroid) pairs in fp32 from
-//      the shared-memory tiles, eight pairs per warp step, lowest index winning ties, with the same
-//      summation order as the CUDA-core kernels;
-//   3. the accumulate group (4 warps) adds every row of the tile into the per-cluster sums it keeps in
-//      registers: a warp owns rows, a lane owns columns, the label selects the register by a jump that
-//      is uniform across the warp.  No atomics: the order of every addition is fixed by the launch
-//      shape, so results repeat bit for bit.
-// At the end the accumulate group folds its row groups in order through shared memory into psum[block].
+//   2. four screen warps, one row per thread and no barrier between them, read the accumulator back and
+//      keep the two smallest packed (score | column) keys.  If the second is farther from the first than
+//      the TF32 error bound of that row allows, the first is provably the fp32 argmin and becomes the
+//      label.  Otherwise the row id goes to the warp's list of undecided rows, with the set of centroids
+//      inside the bound;
+//   3. two sorting warps (alternating tiles) group the tile's decided rows by label, stably;
+//   4. eight accumulate warps, each owning K/8 clusters with one 16-byte column chunk per lane, add the
+//      rows of their clusters, in row order, from the shared-memory tile into registers.
+// kmeans_late_rows then settles the undecided rows in fp32 (lowest index wins ties, same summation order
+// as the CUDA-core kernels) and adds them into a second set of partial sums.  No floating-point atomics
+// anywhere: the order of every addition is fixed by the launch shape and the lists, so results repeat
+// bit for bit.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -35,58 +36,64 @@ constexpr int KBLK = 32;                // floats in one 128-byte swizzle row
 constexpr int MAX_KB = 4;               // d <= 128
 constexpr int X_KB_BYTES = BM * 128;    // one k-block of a row tile
 constexpr int MAX_STAGES = 8;
-constexpr int THREADS = 512;            // warp 0 TMA, 1 MMA, 2 TMEM alloc, 3 idle, 4..7 screen group, 8..15 accumulate group
+constexpr int THREADS = 512;            // warp 0 TMA, 1 MMA, 2..3 sorting (2 also owns TMEM), 4..7 screen, 8..15 accumulate
 constexpr int S_WARP0 = 4;
 constexpr int A_WARP0 = 8;
 constexpr int A_WARPS = 8;
 constexpr int MAX_K = 64;
-constexpr int ROW_CANDS = 8;            // candidates listed per undecided row before it is scored against all K
-constexpr int QUEUE_CAP = BM * ROW_CANDS;
 
 struct FusedShared {
     uint64_t x_full[MAX_STAGES], x_empty[MAX_STAGES];
     uint64_t c_full;
     uint64_t t_full[2], t_empty[2];
     uint64_t lab_full[2], lab_empty[2];
-    unsigned long long rowbest[BM];     // undecided rows: min over candidates of (ordered fp32 score << 32 | centroid)
+    uint64_t ord_full[2], ord_empty[2];
     uint32_t tmem_base;
     int abort;
-    int stop;                           // the abort flag as screen thread 0 saw it before the tile's first group barrier
-    int qn, fqn;
-    int queue[QUEUE_CAP];               // (row in tile << 8) | centroid
-    int fullq[BM];                      // rows with more than ROW_CANDS candidates
-    int order[2][BM];                   // rows of the tile grouped by label, ascending row inside a label
-    int off[2][MAX_K + 1];              // first position of each label in order[]
-    int wcnt[2][4][MAX_K + 1];          // rows per (screen warp, label); label MAX_K = rows beyond N
+    uint8_t lab[2][BM];                 // label of each row of the tile; MAX_K = not to be accumulated here
+    uint16_t order[2][BM];              // the tile's rows grouped by label, ascending row inside a label, each as
+                                        // its byte offset inside a k-block with the swizzle term in bits 4..6
+    int goff[2][MAX_K + 1];             // first position of each label in order[]
+    int hcnt[2][MAX_K + 1];             // scratch of the two sorting warps
     int cnt[MAX_K];
-    float cn[MAX_K];
-    float red[2][4];
+    alignas(16) float cn[MAX_K];
 };
 
-__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
-
-// Byte offset of 16-byte chunk q of row r in a swizzled tile whose k-blocks are kb_bytes apart.
-__device__ __forceinline__ uint32_t chunk_off(int r, int q, int kb_bytes) {
-    return (uint32_t)((q >> 3) * kb_bytes + r * 128 + (((q & 7) ^ (r & 7)) << 4));
+// 16 accumulator columns, issued without waiting: several of these go out before one tmem_wait().
+template <int O, int VN>
+__device__ __forceinline__ void tmem_issue16(uint32_t taddr, uint32_t (&v)[VN]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[O + 0]), "=r"(v[O + 1]), "=r"(v[O + 2]), "=r"(v[O + 3]), "=r"(v[O + 4]), "=r"(v[O + 5]), "=r"(v[O + 6]),
+          "=r"(v[O + 7]), "=r"(v[O + 8]), "=r"(v[O + 9]), "=r"(v[O + 10]), "=r"(v[O + 11]), "=r"(v[O + 12]),
+          "=r"(v[O + 13]), "=r"(v[O + 14]), "=r"(v[O + 15])
+        : "r"(taddr + O)
+        : "memory");
 }
+__device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ unsigned long long pack_score(float sc, int k) {
-    uint32_t u = __float_as_uint(sc);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);        // unsigned order = float order
-    return ((unsigned long long)u << 32) | (uint32_t)k;
-}
-
-// KMAX = 32 or 64: upper bound of K, 8 accumulate warps each owning KMAX / 8 clusters.
-// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - trunc_tf32(c_k)|.
+// KMAX = 32 or 64: upper bound of K.  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - tf32(c_k)|;
+// cn = |c_k|^2 padded with a huge value.  Block b leaves the sums of the rows it decided in psum[b][K][d],
+// their counts in pcnt[b][K], and per screen warp w the undecided rows in late_list[(4 b + w) late_cap ..]
+// (x = row id, y and z = mask of the centroids within the bound), late_count[4 b + w] of them.
 template <int KMAX>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
                 const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
                 int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
                 int32_t *__restrict__ assign, float *__restrict__ psum, int *__restrict__ pcnt,
+                int4 *__restrict__ late_list, int64_t late_cap, int *__restrict__ late_count,
                 unsigned long long *counters, int *status) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // The swizzled tiles need 1024-byte alignment.  The array is used as declared (no pointer arithmetic
+    // through integers), so that every access below stays a shared-memory instruction; should a launch
+    // ever place it differently, the block reports that and leaves before touching anything.
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if ((smem_u32(smem) & 1023u) != 0u) {
+        if (threadIdx.x == 0) ep_raise(status, EP_ERR_CUDA);
+        if (threadIdx.x < 4) late_count[blockIdx.x * 4 + threadIdx.x] = 0;
+        return;
+    }
     const int stage_bytes = num_kb * X_KB_BYTES;
     const int c_kb_bytes = npad * 128;
     uint8_t *x_smem = smem;                                          // [stages][num_kb][128 rows][128 B]
@@ -106,17 +113,16 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         mbar_init(&sh->c_full, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh->t_full[i], 1);
-            mbar_init(&sh->t_empty[i], 4);
+            mbar_init(&sh->t_empty[i], 4);    // the screen warps
             mbar_init(&sh->lab_full[i], 4);
-            mbar_init(&sh->lab_empty[i], A_WARPS);
+            mbar_init(&sh->lab_empty[i], 1);  // a sorting warp
+            mbar_init(&sh->ord_full[i], 1);
+            mbar_init(&sh->ord_empty[i], A_WARPS);
         }
         sh->abort = 0;
-        sh->stop = 0;
         sh->tmem_base = 0;
-        sh->qn = sh->fqn = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int k = threadIdx.x; k < 2 * 4 * (MAX_K + 1); k += blockDim.x) (&sh->wcnt[0][0][0])[k] = 0;
     for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
         sh->cnt[k] = 0;
         sh->cn[k] = k < npad ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
@@ -171,214 +177,185 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&sh->t_full[buf]);
             }
         }
-    } else if (warp >= S_WARP0 && warp < A_WARP0) {
-        // ---------------------------------------------------------------- screen group: one row per thread
-        const int sw = warp - S_WARP0;                     // TMEM lanes 32 sw .. 32 sw + 31
-        const int stid = threadIdx.x - S_WARP0 * 32;       // 0..127 = row in tile
-        {   // largest centroid norm and truncation residual
-            float m2 = 0.f, ml = 0.f;
-            for (int k = stid; k < K; k += 128) {
-                m2 = fmaxf(m2, cn[k]);
-                ml = fmaxf(ml, clo[k]);
-            }
+    }
+    if (warp == 2 || warp == 3) {
+        // ---------------------------------------------------------------- sorting warps: warp 2 takes the
+        // block's even tiles, warp 3 the odd ones.  A stable counting sort of the tile's 128 rows by label,
+        // so that an accumulate warp finds the rows of a cluster as one run, in row order.
+        const uint32_t hw = (uint32_t)warp - 2u;
+        const unsigned lt = (1u << lane) - 1u;
+        for (uint32_t it = hw;; it += 2) {
+            const int64_t tile = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
+            if (tile >= num_tiles) break;
+            const uint32_t par = hw, use = (it >> 1) & 1u;
+            if (!mbar_wait(&sh->lab_full[par], use, abort_flag)) break;
+            int l[4];
 #pragma unroll
-            for (int o = 16; o >= 1; o >>= 1) {
-                m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
-                ml = fmaxf(ml, __shfl_xor_sync(FULL, ml, o));
+            for (int j = 0; j < 4; ++j) l[j] = sh->lab[par][j * 32 + lane];
+            for (int i = lane; i <= MAX_K; i += 32) sh->hcnt[hw][i] = 0;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->lab_empty[par]);
+            int before[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const unsigned peers = __match_any_sync(FULL, l[j]);
+                const int leader = __ffs(peers) - 1;
+                int old = 0;
+                if (lane == leader) {
+                    old = sh->hcnt[hw][l[j]];
+                    sh->hcnt[hw][l[j]] = old + __popc(peers);
+                }
+                before[j] = __shfl_sync(FULL, old, leader) + __popc(peers & lt);
+                __syncwarp();
             }
-            if (lane == 0) {
-                sh->red[0][sw] = m2;
-                sh->red[1][sw] = ml;
+            const int t0 = sh->hcnt[hw][2 * lane], t1 = sh->hcnt[hw][2 * lane + 1];
+            int inc = t0 + t1;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(FULL, inc, o);
+                if (lane >= o) inc += up;
             }
+            const int ex = inc - t0 - t1;
+            if (t0) atomicAdd(&sh->cnt[2 * lane], t0);       // integer: exact whatever the order
+            if (t1) atomicAdd(&sh->cnt[2 * lane + 1], t1);
+            if (!mbar_wait(&sh->ord_empty[par], use ^ 1u, abort_flag)) break;
+            sh->goff[par][2 * lane] = ex;
+            sh->goff[par][2 * lane + 1] = ex + t0;
+            if (lane == 31) sh->goff[par][MAX_K] = inc;
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (l[j] < MAX_K) {
+                    const int r = j * 32 + lane;
+                    sh->order[par][sh->goff[par][l[j]] + before[j]] = (uint16_t)((r << 7) | ((r & 7) << 4));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->ord_full[par]);
         }
-        group_sync(1);
-        const float cmax2 = fmaxf(fmaxf(sh->red[0][0], sh->red[0][1]), fmaxf(sh->red[0][2], sh->red[0][3]));
-        const float clomax = fmaxf(fmaxf(sh->red[1][0], sh->red[1][1]), fmaxf(sh->red[1][2], sh->red[1][3]));
+    } else if (warp >= S_WARP0 && warp < A_WARP0) {
+        // ---------------------------------------------------------------- screen warps: one row per thread,
+        // each warp on its own (no barrier between them): TMEM lanes 32 sw .. 32 sw + 31 = rows of the tile
+        const int sw = warp - S_WARP0;
+        const int stid = threadIdx.x - S_WARP0 * 32;       // row in tile
+        float m2 = 0.f, ml = 0.f;                          // largest centroid norm and rounding residual
+        for (int k = lane; k < K; k += 32) {
+            m2 = fmaxf(m2, cn[k]);
+            ml = fmaxf(ml, clo[k]);
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
+            ml = fmaxf(ml, __shfl_xor_sync(FULL, ml, o));
+        }
+        const float cmax2 = m2, clomax = ml;
         const float cmax = sqrtf(cmax2) * 1.000001f;
-        const int slot = lane_chunk_slot(lane);
-        unsigned long long n_rows = 0, n_undecided = 0, n_items = 0, n_full = 0;
-        mbar_wait(&sh->c_full, 0u, abort_flag);            // the fp32 re-scoring below reads the centroid tile
+        const unsigned lt = (1u << lane) - 1u;
+        int4 *late_rows = late_list + ((size_t)blockIdx.x * 4 + sw) * late_cap;
+        int late_n = 0;
+        unsigned n_rows = 0;
 
         float2 nr_next = make_float2(0.f, 0.f);            // this row's norms, fetched one tile ahead
         if ((int64_t)blockIdx.x * BM + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BM + stid);
 
         uint32_t it = 0;
         for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-            const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u, par = it & 1u;
-            const uint8_t *xs = x_smem + (size_t)s * stage_bytes;
             const int64_t row = tile * BM + stid;
             const float2 nr = nr_next;
             {
                 const int64_t nrow = (tile + gridDim.x) * BM + stid;
                 if (nrow < N) nr_next = __ldg(rownorm + nrow);
             }
-            // Waits that give up leave garbage behind but nothing out of bounds; the group leaves the loop
-            // together after the next barrier.
-            mbar_wait(&sh->lab_empty[par], use ^ 1u, abort_flag);
-            mbar_wait(&sh->t_full[buf], use, abort_flag);
-            mbar_wait(&sh->x_full[s], ph, abort_flag);
+            if (!mbar_wait(&sh->t_full[buf], use, abort_flag)) break;
             tc_fence_after();
+            // ---- all of this row's screened products into registers, then the accumulator is free again
             const uint32_t taddr = tmem_base + ((uint32_t)(sw * 32) << 16) + buf * (uint32_t)npad;
-            float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
-            for (int c = 0; c < npad; c += 16) {
-                uint32_t v[16];
-                tmem_ld16(taddr + c, v);
+            uint32_t v[KMAX];
+            tmem_issue16<0>(taddr, v);
+            if (npad > 16) tmem_issue16<16>(taddr, v);
+            if constexpr (KMAX > 32) {
+                if (npad > 32) tmem_issue16<32>(taddr, v);
+                if (npad > 48) tmem_issue16<48>(taddr, v);
+            }
+            tmem_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
+            float key1[4], key2[4];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float sc = fmaf(-2.f, __uint_as_float(v[j]), sh->cn[c + j]);
-                    const float key = __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + j));
-                    if (j & 1)
-                        keep_two(b1, b2, key);
-                    else
-                        keep_two(a1, a2, key);
+            for (int i = 0; i < 4; ++i) key1[i] = key2[i] = __uint_as_float(KEY_INIT);
+#pragma unroll
+            for (int c = 0; c < KMAX; c += 16) {
+                if (c < npad) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 16; j4 += 4) {
+                        const float4 n4 = *reinterpret_cast<const float4 *>(&sh->cn[c + j4]);
+                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float sc = fmaf(-2.f, __uint_as_float(v[c + j4 + j]), nn[j]);
+                            v[c + j4 + j] = __float_as_uint(sc);
+                            keep_two(key1[j], key2[j],
+                                     __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + j4 + j)));
+                        }
+                    }
                 }
             }
-            const float k1 = fminf(a1, b1);
-            const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+            const float lo01 = fminf(key1[0], key1[1]), hi01 = fminf(fmaxf(key1[0], key1[1]), fminf(key2[0], key2[1]));
+            const float lo23 = fminf(key1[2], key1[3]), hi23 = fminf(fmaxf(key1[2], key1[3]), fminf(key2[2], key2[3]));
+            const float k1 = fminf(lo01, lo23);
+            const float k2 = fminf(fmaxf(lo01, lo23), fminf(hi01, hi23));
             const float thr = k1 + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
             const int i1 = (int)(__float_as_uint(k1) & IDX_MASK);
             const bool live = row < N;
             const bool decided = k2 > thr && i1 < K;       // the best screened score cannot be overtaken
             const bool undecided = live && !decided;
-            if (__any_sync(FULL, undecided)) {
-                // list this row's centroids whose screened score is within the allowance of the best
-                int nc = 0;
-                if (undecided) sh->rowbest[stid] = ~0ull;
-                for (int c = 0; c < npad; c += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(taddr + c, v);
-                    if (undecided) {
+            const int label = (live && decided) ? i1 : MAX_K;   // MAX_K: not accumulated by this kernel
+            const unsigned todo = __ballot_sync(FULL, undecided);
+            if (todo) {
+                // Rows that the screening cannot decide are not settled here: their ids go, in row order, to
+                // this warp's list, each with the set of centroids whose screened score is within the allowance
+                // of the row's best (bit c of the two mask words); kmeans_late_rows labels and accumulates them.
+                if (undecided) {
+                    uint32_t mlo = 0u, mhi = 0u;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float sc = fmaf(-2.f, __uint_as_float(v[j]), sh->cn[c + j]);
-                            if (sc <= thr && c + j < K) {
-                                if (nc < ROW_CANDS) sh->queue[atomicAdd(&sh->qn, 1)] = (stid << 8) | (c + j);
-                                ++nc;
-                            }
-                        }
+                    for (int c = 0; c < KMAX; ++c) {
+                        const uint32_t hit = (c < K && __uint_as_float(v[c]) <= thr) ? 1u : 0u;
+                        if (c < 32)
+                            mlo |= hit << (c & 31);
+                        else
+                            mhi |= hit << (c & 31);
                     }
+                    late_rows[(size_t)late_n + __popc(todo & lt)] = make_int4((int)row, (int)mlo, (int)mhi, 0);
                 }
-                if (undecided && (nc > ROW_CANDS || nc == 0)) sh->fullq[atomicAdd(&sh->fqn, 1)] = stid;   // nc == 0: NaN scores
+                late_n += __popc(todo);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
-            if (stid == 0) sh->stop = *abort_flag;
-            group_sync(1);
-            if (sh->stop) break;
-            // ---- fp32 re-scoring of the listed (row, centroid) pairs, eight per warp step
-            const int qn = min(sh->qn, QUEUE_CAP), fqn = min(sh->fqn, BM);
-            for (int base = sw * KC; base < qn; base += 4 * KC) {
-                float a[KC];
-#pragma unroll
-                for (int kk = 0; kk < KC; ++kk) {
-                    const int item = sh->queue[min(base + kk, qn - 1)];
-                    a[kk] = 0.f;
-                    if (lane < d4) {
-                        const float4 x = *reinterpret_cast<const float4 *>(xs + chunk_off(item >> 8, lane, X_KB_BYTES));
-                        const float4 cc = *reinterpret_cast<const float4 *>(c_smem + chunk_off(item & 255, lane, c_kb_bytes));
-                        a[kk] = dot4(x, cc, 0.f);
-                    }
-                }
-                const float dot = reduce8_transposed(a, lane);
-                if ((lane & 3) == 0 && base + slot < qn) {
-                    const int item = sh->queue[base + slot];
-                    float sc = fmaf(-2.f, dot, sh->cn[item & 255]);
-                    sc = (sc == sc) ? sc : CUDART_INF_F;
-                    atomicMin(&sh->rowbest[item >> 8], pack_score(sc, item & 255));
-                }
-            }
-            // ---- rows with too many candidates: all K centroids
-            for (int fi = sw; fi < fqn; fi += 4) {
-                const int r = sh->fullq[fi];
-                const float4 x = lane < d4 ? *reinterpret_cast<const float4 *>(xs + chunk_off(r, lane, X_KB_BYTES))
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-                unsigned long long best = ~0ull;
-                for (int kb = 0; kb < K; kb += KC) {
-                    float a[KC];
-#pragma unroll
-                    for (int kk = 0; kk < KC; ++kk) {
-                        a[kk] = 0.f;
-                        if (kb + kk < K && lane < d4)
-                            a[kk] = dot4(x, *reinterpret_cast<const float4 *>(c_smem + chunk_off(kb + kk, lane, c_kb_bytes)), 0.f);
-                    }
-                    const float dot = reduce8_transposed(a, lane);
-                    const int k = kb + slot;
-                    if (k < K) {
-                        float sc = fmaf(-2.f, dot, sh->cn[k]);
-                        sc = (sc == sc) ? sc : CUDART_INF_F;
-                        const unsigned long long p = pack_score(sc, k);
-                        best = p < best ? p : best;
-                    }
-                }
-                if ((lane & 3) == 0) atomicMin(&sh->rowbest[r], best);
-            }
-            group_sync(1);
-            // ---- final label of this thread's row
-            if (stid == 0) sh->qn = sh->fqn = 0;
-            int label = MAX_K;                             // bucket of the rows beyond N
             if (live) {
-                label = decided ? i1 : (int)(uint32_t)(sh->rowbest[stid] & 0xffffffffull);
-                if (label < 0 || label >= K) label = 0;    // a row of NaNs still gets a valid label
-                assign[row] = label;
+                if (decided) assign[row] = label;
                 ++n_rows;
-                n_undecided += undecided ? 1 : 0;
             }
-            n_items += (lane == 0 && sw == 0) ? (unsigned long long)qn : 0ull;
-            n_full += (lane == 0 && sw == 0) ? (unsigned long long)fqn : 0ull;
-            // ---- group the tile's rows by label for the accumulate group (a stable counting sort)
-            const unsigned peers = __match_any_sync(FULL, label);
-            if (lane == __ffs(peers) - 1) sh->wcnt[par][sw][label] = __popc(peers);
-            for (int i = stid; i < 4 * (MAX_K + 1); i += 128) (&sh->wcnt[par ^ 1u][0][0])[i] = 0;
-            group_sync(1);
-            if (sw == 0) {   // exclusive prefix over the labels: two labels per lane
-                const int k0 = 2 * lane, k1 = 2 * lane + 1;
-                const int t0 = sh->wcnt[par][0][k0] + sh->wcnt[par][1][k0] + sh->wcnt[par][2][k0] + sh->wcnt[par][3][k0];
-                const int t1 = sh->wcnt[par][0][k1] + sh->wcnt[par][1][k1] + sh->wcnt[par][2][k1] + sh->wcnt[par][3][k1];
-                int inc = t0 + t1;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int u = __shfl_up_sync(FULL, inc, o);
-                    if (lane >= o) inc += u;
-                }
-                const int ex = inc - t0 - t1;
-                sh->off[par][k0] = ex;
-                sh->off[par][k1] = ex + t0;
-                if (lane == 31) sh->off[par][MAX_K] = inc;
-                sh->cnt[k0] += t0;
-                sh->cnt[k1] += t1;
-            }
-            group_sync(1);
-            if (live) {
-                int pos = sh->off[par][label] + __popc(peers & ((1u << lane) - 1u));
-                for (int w2 = 0; w2 < sw; ++w2) pos += sh->wcnt[par][w2][label];
-                sh->order[par][pos] = stid;
-            }
+            // ---- hand the labels to the sorting warp
+            if (!mbar_wait(&sh->lab_empty[par], use ^ 1u, abort_flag)) break;
+            sh->lab[par][stid] = (uint8_t)label;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->lab_full[par]);
         }
-        group_sync(1);
-        for (int k = stid; k < K; k += 128) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[k];
+        if (lane == 0) late_count[blockIdx.x * 4 + sw] = late_n;   // always written: the next kernel trusts it
         if (counters) {
 #pragma unroll
-            for (int o = 16; o >= 1; o >>= 1) {
-                n_rows += __shfl_xor_sync(FULL, n_rows, o);
-                n_undecided += __shfl_xor_sync(FULL, n_undecided, o);
-            }
+            for (int o = 16; o >= 1; o >>= 1) n_rows += __shfl_xor_sync(FULL, n_rows, o);
             if (lane == 0) {
-                atomicAdd(&counters[0], n_rows);
-                atomicAdd(&counters[3], n_undecided);
-                atomicAdd(&counters[4], n_items);
-                atomicAdd(&counters[5], n_full);
+                atomicAdd(&counters[0], (unsigned long long)n_rows);
+                atomicAdd(&counters[3], (unsigned long long)late_n);
             }
         }
     } else if (warp >= A_WARP0) {
-        // ---------------------------------------------------------------- accumulate group
+        // ---------------------------------------------------------------- accumulate warps
         const int aw = warp - A_WARP0;                     // owns clusters aw, aw + 8, ...
-        const int atid = threadIdx.x - A_WARP0 * 32;
         constexpr int OWN = KMAX / A_WARPS;
         const bool has_cols = lane < d4;                   // this lane's 16-byte chunk of a row is chunk `lane`
+        const uint32_t lx = (uint32_t)(lane & 7) << 4;     // its place inside a 128-byte swizzle row, before the swizzle
         float4 acc[OWN];
 #pragma unroll
         for (int i = 0; i < OWN; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -386,21 +363,20 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t s = it % (uint32_t)stages;
             const uint32_t par = it & 1u, use = (it >> 1) & 1u;
-            const uint8_t *xs = x_smem + (size_t)s * stage_bytes;
-            if (!mbar_wait(&sh->lab_full[par], use, abort_flag)) break;
+            const uint8_t *xl = x_smem + (size_t)s * stage_bytes + (size_t)(lane >> 3) * X_KB_BYTES;   // this lane's k-block
+            if (!mbar_wait(&sh->ord_full[par], use, abort_flag)) break;
             if (!mbar_wait(&sh->x_full[s], (it / (uint32_t)stages) & 1u, abort_flag)) break;   // long complete: makes the tile visible here
 #pragma unroll
             for (int i = 0; i < OWN; ++i) {
                 const int k = aw + A_WARPS * i;
                 if (k < K) {
-                    const int p1 = sh->off[par][k + 1];
-                    for (int p = sh->off[par][k]; p < p1; p += 4) {   // four rows at a time: loads first, adds in row order
+                    const int p1 = sh->goff[par][k + 1];
+                    for (int p = sh->goff[par][k]; p < p1; p += 4) {   // four rows at a time: loads first, adds in row order
                         float4 x[4];
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            const int r = sh->order[par][min(p + u, p1 - 1)];
-                            x[u] = has_cols ? *reinterpret_cast<const float4 *>(xs + chunk_off(r, lane, X_KB_BYTES))
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                            const uint32_t o = sh->order[par][min(p + u, p1 - 1)];
+                            x[u] = has_cols ? *reinterpret_cast<const float4 *>(xl + (o ^ lx)) : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
@@ -417,7 +393,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(&sh->x_empty[s]);
-                mbar_arrive(&sh->lab_empty[par]);
+                mbar_arrive(&sh->ord_empty[par]);
             }
         }
         // ---- publish this block's sums: every (cluster, chunk) has exactly one owner
@@ -427,14 +403,200 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const int k = aw + A_WARPS * i;
             if (k < K && has_cols) out[(size_t)k * d4 + lane] = acc[i];
         }
-        (void)atid;
     }
     __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[k];
     if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
     if (warp == 2) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
+}
+
+// The rows the fused kernel left undecided.  Block b serves fused-kernel block b and its four lists.
+//   1. All 16 warps, 32 consecutive entries per coalesced load: fp32 scores of each row against the
+//      centroids its mask names (all K if the mask is empty, which NaN scores cause), eight per reduction,
+//      lowest index winning ties, with the same summation order as the other kernels; the label goes to
+//      assign[].
+//   2. Warps 0..3: warp w adds the rows of list w, in list order, into its own sum table.
+//   3. The block folds the four tables in warp order into psum[b] / pcnt[b].
+// Every addition happens in an order fixed by the lists, so results repeat bit for bit.
+constexpr int LATE_THREADS = 512;
+constexpr int LATE_LABELS = 4096;
+
+__global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__restrict__ emb, int64_t N, int d, int K,
+                                                                 int kpad, const float *__restrict__ C,
+                                                                 const float *__restrict__ cn,
+                                                                 const int4 *__restrict__ late_list, int64_t late_cap,
+                                                                 const int *__restrict__ late_count,
+                                                                 int32_t *__restrict__ assign, float *__restrict__ psum,
+                                                                 int *__restrict__ pcnt) {
+    extern __shared__ float4 late_smem[];
+    __shared__ int cum[5];
+    __shared__ int ncount[4];
+    __shared__ uint8_t lab_s[LATE_LABELS];                   // labels of the block's first LATE_LABELS listed rows
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
+    const int nwarps = blockDim.x >> 5;
+    float4 *cs = late_smem;                                  // [kpad][32] centroids, zero padded
+    float4 *tab = cs + (size_t)kpad * 32;                    // [4][K][32] per-list sums
+    float *cns = reinterpret_cast<float *>(tab + (size_t)4 * K * 32);   // [kpad]
+    int *cw = reinterpret_cast<int *>(cns + kpad);           // [4][K]
+    for (int i = threadIdx.x; i < kpad * 32; i += blockDim.x) {
+        const int k = i >> 5, q = i & 31;
+        cs[i] = (k < K && q < d4) ? __ldg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int i = threadIdx.x; i < 4 * K * 32; i += blockDim.x) tab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = threadIdx.x; i < kpad; i += blockDim.x) cns[i] = i < K ? cn[i] : CUDART_INF_F;
+    for (int i = threadIdx.x; i < 4 * K; i += blockDim.x) cw[i] = 0;
+    if (threadIdx.x < 4) ncount[threadIdx.x] = (int)min((int64_t)max(late_count[blockIdx.x * 4 + threadIdx.x], 0), late_cap);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int w = 0; w < 4; ++w) {
+            cum[w] = run;
+            run += ncount[w];
+        }
+        cum[4] = run;
+    }
+    __syncthreads();
+    const int4 *lists = late_list + (size_t)blockIdx.x * 4 * late_cap;
+    const int slot = lane_chunk_slot(lane);
+    // ---- 1. labels, the rows' data fetched four ahead
+    constexpr int AHEAD1 = 4;
+    for (int p0 = warp * 32; p0 < cum[4]; p0 += nwarps * 32) {
+        const int cnt = min(32, cum[4] - p0);
+        int4 e = make_int4(-1, 0, 0, 0);
+        if (lane < cnt) {
+            const int p = p0 + lane;
+            const int w = (p >= cum[1]) + (p >= cum[2]) + (p >= cum[3]);
+            e = lists[(size_t)w * late_cap + (p - cum[w])];
+            if (e.x < 0 || e.x >= N) e.x = -1;               // never index outside the matrix, whatever the list holds
+        }
+        float4 xq[AHEAD1];
+#pragma unroll
+        for (int u = 0; u < AHEAD1; ++u) {
+            const int r = __shfl_sync(FULL, e.x, u);
+            xq[u] = (r >= 0 && lane < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int i0 = 0; i0 < cnt; i0 += AHEAD1) {
+#pragma unroll
+            for (int u = 0; u < AHEAD1; ++u) {
+                const int i = i0 + u;
+                const float4 x = xq[u];
+                const int row = __shfl_sync(FULL, e.x, i & 31);
+                const uint32_t mlo = (uint32_t)__shfl_sync(FULL, e.y, i & 31), mhi = (uint32_t)__shfl_sync(FULL, e.z, i & 31);
+                const int rn = __shfl_sync(FULL, e.x, (i + AHEAD1) & 31);
+                xq[u] = (i + AHEAD1 < cnt && rn >= 0 && lane < d4)
+                            ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)rn * d4 + lane)
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i >= cnt || row < 0) continue;
+                unsigned long long m = ((unsigned long long)mhi << 32) | mlo;
+                if (K < 64) m &= (1ull << K) - 1ull;
+                if (m == 0ull) m = K < 64 ? (1ull << K) - 1ull : ~0ull;
+                float best = CUDART_INF_F;
+                int bidx = 0x7fffffff;
+                while (m) {
+                    float a[KC];
+                    int myk = -1;
+#pragma unroll
+                    for (int kk = 0; kk < KC; ++kk) {        // the next eight named centroids (fewer at the end)
+                        a[kk] = 0.f;
+                        if (m) {
+                            const int k = __ffsll((long long)m) - 1;
+                            m &= m - 1;
+                            if (kk == slot) myk = k;
+                            a[kk] = dot4(x, cs[k * 32 + lane], 0.f);
+                        }
+                    }
+                    const float dot = reduce8_transposed(a, lane);
+                    if (myk >= 0) {
+                        float sc = fmaf(-2.f, dot, cns[myk]);
+                        sc = (sc == sc) ? sc : CUDART_INF_F;
+                        if (sc < best || (sc == best && myk < bidx)) {
+                            best = sc;
+                            bidx = myk;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o >= 4; o >>= 1) {          // the eight slots differ in lane bits 4, 3, 2
+                    const float ov = __shfl_xor_sync(FULL, best, o);
+                    const int oi = __shfl_xor_sync(FULL, bidx, o);
+                    if (ov < best || (ov == best && oi < bidx)) {
+                        best = ov;
+                        bidx = oi;
+                    }
+                }
+                if (bidx < 0 || bidx >= K) bidx = 0;         // a row of NaNs still gets a valid label
+                if (lane == 0) {
+                    assign[row] = bidx;
+                    if (p0 + i < LATE_LABELS) lab_s[p0 + i] = (uint8_t)bidx;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // ---- 2. sums: warp w walks list w in order, 32 entries per coalesced load, row data fetched eight ahead
+    if (warp < 4) {
+        const int n = cum[warp + 1] - cum[warp];
+        const int4 *rows = lists + (size_t)warp * late_cap;
+        float4 *mytab = tab + (size_t)warp * K * 32;
+        constexpr int AHEAD = 8;
+        for (int j0 = 0; j0 < n; j0 += 32) {
+            const int cnt = min(32, n - j0);
+            int row_l = -1, lab_l = -1;
+            if (lane < cnt) {
+                row_l = rows[j0 + lane].x;
+                if (row_l < 0 || row_l >= N) row_l = -1;
+                if (row_l >= 0) lab_l = cum[warp] + j0 + lane < LATE_LABELS ? (int)lab_s[cum[warp] + j0 + lane] : assign[row_l];
+            }
+            float4 xq[AHEAD];
+#pragma unroll
+            for (int u = 0; u < AHEAD; ++u) {
+                const int r = __shfl_sync(FULL, row_l, u);
+                xq[u] = (r >= 0 && lane < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            for (int i0 = 0; i0 < cnt; i0 += AHEAD) {
+#pragma unroll
+                for (int u = 0; u < AHEAD; ++u) {
+                    const int i = i0 + u;
+                    const float4 x = xq[u];
+                    const int a = __shfl_sync(FULL, lab_l, i & 31);
+                    const int rn = __shfl_sync(FULL, row_l, (i + AHEAD) & 31);
+                    xq[u] = (i + AHEAD < cnt && rn >= 0 && lane < d4)
+                                ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)rn * d4 + lane)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i < cnt && a >= 0 && a < K) {
+                        float4 t = mytab[a * 32 + lane];
+                        t.x += x.x;
+                        t.y += x.y;
+                        t.z += x.z;
+                        t.w += x.w;
+                        mytab[a * 32 + lane] = t;
+                        if (lane == 0) cw[warp * K + a] += 1;
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // ---- 3. fold
+    float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
+    for (int i = threadIdx.x; i < K * d4; i += blockDim.x) {
+        const int k = i / d4, q = i - k * d4;
+        float4 t = tab[k * 32 + q];
+        for (int w = 1; w < 4; ++w) {
+            const float4 u = tab[((size_t)w * K + k) * 32 + q];
+            t.x += u.x;
+            t.y += u.y;
+            t.z += u.z;
+            t.w += u.w;
+        }
+        out[i] = t;
+    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = cw[k] + cw[K + k] + cw[2 * K + k] + cw[3 * K + k];
 }
 
 // rownorm[i] = (|x_i|_2, |x_i - trunc_tf32(x_i)|_2), both rounded up a little; one warp per row.
@@ -464,6 +626,7 @@ namespace ep {
 struct TcFusedState {
     CUtensorMap map_x, map_c;
     int npad, num_kb, stages, grid;
+    int64_t late_cap;
     size_t smem;
     uint32_t tmem_cols;
 };
@@ -474,7 +637,7 @@ static inline int tcf_npad(int K) { return std::max(16, (K + 15) / 16 * 16); }
 
 static size_t tcf_fixed_smem(int d, int K) {
     const int num_kb = (d + KBLK - 1) / KBLK;
-    return (size_t)num_kb * tcf_npad(K) * 128 + sizeof(FusedShared) + 1024;
+    return (size_t)num_kb * tcf_npad(K) * 128 + sizeof(FusedShared);
 }
 
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K) {
@@ -487,7 +650,12 @@ int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N) {
     return (int)std::max<int64_t>(1, std::min<int64_t>(ctx->sm_count, ceil_div(N, BM)));
 }
 
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, float2 *rownorm,
+// Entries of one screen warp's list of undecided rows: every row it can ever see.
+int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N) {
+    return ceil_div(ceil_div(N, BM), kmeans_tcf_grid(ctx, N)) * 32;
+}
+
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
                        TcFusedState *st, cudaStream_t stream) {
     st->npad = tcf_npad(K);
     st->num_kb = (d + KBLK - 1) / KBLK;
@@ -496,10 +664,11 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     st->stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / stage);
     st->smem = fixed + (size_t)st->stages * stage;
     st->grid = kmeans_tcf_grid(ctx, N);
+    st->late_cap = kmeans_tcf_late_cap(ctx, N);
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)st->npad) cols <<= 1;
     st->tmem_cols = cols;
-    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, centroids, K, d, st->npad))
+    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
     Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
     row_norms<<<(int)std::min<int64_t>((int64_t)ctx->sm_count * 16, ceil_div(N, 8)), 256, 0, stream>>>(emb, N, d, rownorm);
@@ -509,8 +678,8 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
 }
 
 template <int KMAX>
-static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo,
-                      const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
+static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo, const float2 *rownorm,
+                      int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, int4 *late_list, int *late_count,
                       cudaStream_t stream) {
     auto kern = kmeans_tc_fused<KMAX>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
@@ -519,19 +688,31 @@ static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, cons
     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
     kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, cn, clo, rownorm, N, d, K, st.npad, st.num_kb,
                                               st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK, assign,
-                                              psum, pcnt, counters, ctx->d_status);
+                                              psum, pcnt, late_list, st.late_cap, late_count, counters, ctx->d_status);
     tm.end(1);
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;
 }
 
-// One Lloyd assignment + accumulation pass; block b leaves its sums in psum[b][K][d], counts in pcnt[b][K].
-int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *centroids, const float *cn, const float *clo,
-                      const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
-                      cudaStream_t stream) {
-    (void)centroids;   // the kernel reads them through the tensor map made by kmeans_tcf_prepare
-    if (K <= 32) return tcf_launch<32>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
-    return tcf_launch<64>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, stream);
+// One Lloyd assignment + accumulation pass.  The fused kernel's block b leaves its sums in psum[b][K][d] and
+// counts in pcnt[b][K]; the kernel for the rows it left undecided adds the slabs grid .. 2 grid - 1.
+int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
+                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
+                      int *pcnt, void *late_list_ws, int *late_count, cudaStream_t stream) {
+    int4 *late_list = static_cast<int4 *>(late_list_ws);
+    int rc = K <= 32 ? tcf_launch<32>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
+                     : tcf_launch<64>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream);
+    if (rc != EP_OK) return rc;
+    const int kpad = (K + KC - 1) / KC * KC;
+    const size_t smem = (size_t)kpad * 512 + (size_t)4 * K * 512 + (size_t)kpad * 4 + (size_t)4 * K * 4;
+    EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_late_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
+    kmeans_late_rows<<<st.grid, LATE_THREADS, smem, stream>>>(emb, N, d, K, kpad, centroids, cn, late_list, st.late_cap,
+                                                              late_count, assign, psum + (size_t)st.grid * K * d,
+                                                              pcnt + (size_t)st.grid * K);
+    tm.end(1);
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
 }
 
 }  // namespace ep

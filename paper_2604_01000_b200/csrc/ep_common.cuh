@@ -112,7 +112,8 @@ size_t kmeans_tc_state_bytes();
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K);
 int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st);
 int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K, const float *centroids,
-                     const float *cn, const float *clo, int32_t *assign, void *cand_ws, cudaStream_t stream);
+                     const float *cn, const float *clo, float *cmaxima, const float2 *rownorm, int32_t *assign,
+                     void *cand_ws, cudaStream_t stream);
 
 // ---- fused tensor-core pass for few centroids (kmeans_tc_fused.cu) --------------------------------
 struct TcFusedState;
@@ -120,8 +121,8 @@ bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tcf_state_bytes();
 int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N);
 int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N);
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
-                       TcFusedState *st, cudaStream_t stream);
+int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *rownorm, cudaStream_t stream);
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st);
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
                       const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
                       int *pcnt, void *late_list, int *late_count, cudaStream_t stream);

@@ -454,7 +454,8 @@ struct KMeansBuffers {
     void *cand;        // tensor path: screening keys of one row chunk
     float *ct;         // tensor path: centroids rounded to TF32
     float *clo;        // tensor path: |c_k - ct_k|
-    float2 *rownorm;   // fused tensor path: (|x_i|, |x_i - trunc(x_i)|)
+    float2 *rownorm;   // tensor paths: (|x_i|, |x_i - trunc(x_i)|)
+    float *cmaxima;    // large-K tensor path: max |c|^2 and max rounding residual of this iteration
     void *late_list;   // fused tensor path: per screen warp, the rows the screening left undecided (16 bytes each)
     int *late_count;
 };
@@ -526,12 +527,13 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.sort_ws = a.take<char>(reorder_workspace_bytes(p.N, p.K));
     }
     if (p.tensor) {
+        b.rownorm = a.take<float2>(p.N);
         if (p.tc_fused) {
-            b.rownorm = a.take<float2>(p.N);
             b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N) * 4 * p.grid);
             b.late_count = a.take<int>((size_t)4 * p.grid);
         } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
+            b.cmaxima = a.take<float>(2);
         }
         b.ct = a.take<float>((size_t)p.K * p.d);
         b.clo = a.take<float>(p.K);
@@ -556,8 +558,10 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     if (p.tensor) {
         if (std::max(kmeans_tc_state_bytes(), kmeans_tcf_state_bytes()) > sizeof(tc_state_mem))
             return fail(ctx, EP_ERR_CUDA, "tensor map state too large");
-        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, b.ct, b.rownorm, tcf_state, stream)
+        int rc = p.tc_fused ? kmeans_tcf_prepare(ctx, emb, N, d, K, b.ct, tcf_state)
                             : kmeans_tc_prepare(ctx, emb, N, d, K, b.ct, tc_state);
+        if (rc != EP_OK) return rc;
+        rc = kmeans_row_norms(ctx, emb, N, d, b.rownorm, stream);
         if (rc != EP_OK) return rc;
         // the padding of |c|^2 must never win: every byte 0x7F makes each float 3.39e38
         EP_CUDA(ctx, cudaMemsetAsync(b.cnorm, 0x7F, sizeof(float) * (size_t)ceil_div(K, CN_PAD) * CN_PAD, stream));
@@ -589,7 +593,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
                 tm.end(1);
             } else {
                 if (p.tensor) {
-                    int r1 = kmeans_tc_assign(ctx, *tc_state, emb, N, d, K, centroids, b.cnorm, b.clo, assign, b.cand, stream);
+                    int r1 = kmeans_tc_assign(ctx, *tc_state, emb, N, d, K, centroids, b.cnorm, b.clo, b.cmaxima, b.rownorm, assign, b.cand, stream);
                     if (r1 != EP_OK) return r1;
                 } else {
                     auto kern = kmeans_assign_chunked<VPL, R>;

@@ -201,18 +201,11 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
 }
 
-// Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
-// lane l holds the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.
-template <int VPL>
-__global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin,
-                                                         int64_t row_end, int d, int K, int G,
-                                                         const float *__restrict__ C, const float *__restrict__ cn,
-                                                         const float *__restrict__ clo,
-                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign,
-                                                         unsigned long long *counters) {
-    __shared__ float red[2][8];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
-    // largest centroid norm and largest rounding residual (every block recomputes them: 2 K loads)
+// out[0] = max_k cn[k], out[1] = max_k clo[k] (one block).
+__global__ void __launch_bounds__(1024) centroid_maxima(const float *__restrict__ cn, const float *__restrict__ clo, int K,
+                                                        float *__restrict__ out) {
+    __shared__ float red[2][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float m2 = 0.f, ml = 0.f;
     for (int k = threadIdx.x; k < K; k += blockDim.x) {
         m2 = fmaxf(m2, cn[k]);
@@ -228,94 +221,181 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
         red[1][warp] = ml;
     }
     __syncthreads();
-    float cmax2 = red[0][0], clomax = red[1][0];
+    if (warp == 0) {
+        m2 = red[0][lane];
+        ml = red[1][lane];
 #pragma unroll
-    for (int w = 1; w < 8; ++w) {
-        cmax2 = fmaxf(cmax2, red[0][w]);
-        clomax = fmaxf(clomax, red[1][w]);
+        for (int o = 16; o >= 1; o >>= 1) {
+            m2 = fmaxf(m2, __shfl_xor_sync(FULL, m2, o));
+            ml = fmaxf(ml, __shfl_xor_sync(FULL, ml, o));
+        }
+        if (lane == 0) {
+            out[0] = m2;
+            out[1] = ml;
+        }
     }
+}
+
+// Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
+// lane l holds the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.
+// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|), computed once per call.
+template <int VPL>
+__global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin,
+                                                         int64_t row_end, int d, int K, int G,
+                                                         const float *__restrict__ C, const float *__restrict__ cn,
+                                                         const float *__restrict__ cmaxima,
+                                                         const float2 *__restrict__ rownorm,
+                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign,
+                                                         unsigned long long *counters) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
+    const float cmax2 = cmaxima[0], clomax = cmaxima[1];   // largest |c_k|^2 and largest rounding residual
     const float cmax = sqrtf(cmax2) * 1.000001f;
     unsigned long long n_single = 0, n_scan = 0, n_rows = 0;
     const float4 *C4 = reinterpret_cast<const float4 *>(C);
     const int slot = lane_chunk_slot(lane);
 
-    for (int64_t row = row_begin + (int64_t)blockIdx.x * 8 + warp; row < row_end; row += (int64_t)gridDim.x * 8) {
-        float4 x[VPL];
-        float x2 = 0.f, xl2 = 0.f;
+    // Each warp fetches its next row (keys, norms, the row itself) while it works on the current one.
+    const int64_t stride = (int64_t)gridDim.x * 8;
+    uint2 key_n = make_uint2(KEY_INIT, KEY_INIT);
+    float2 nr_n = make_float2(0.f, 0.f);
+    float4 x_n[VPL];
+    auto fetch = [&](int64_t r) {
+        if (r < row_end) {
+            if (lane < G) key_n = cand[(size_t)(r - row_begin) * G + lane];
+            nr_n = __ldg(rownorm + r);
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-            const int q = lane + 32 * v;
-            x[v] = q < d4 ? ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-            x2 = dot4(x[v], x[v], x2);
-            const float4 r = make_float4(x[v].x - __uint_as_float(__float_as_uint(x[v].x) & 0xFFFFE000u),
-                                         x[v].y - __uint_as_float(__float_as_uint(x[v].y) & 0xFFFFE000u),
-                                         x[v].z - __uint_as_float(__float_as_uint(x[v].z) & 0xFFFFE000u),
-                                         x[v].w - __uint_as_float(__float_as_uint(x[v].w) & 0xFFFFE000u));
-            xl2 = dot4(r, r, xl2);
+            for (int v = 0; v < VPL; ++v) {
+                const int q = lane + 32 * v;
+                x_n[v] = q < d4 ? ldg_stream(reinterpret_cast<const float4 *>(emb) + r * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
-        x2 = warp_sum(x2);
-        xl2 = warp_sum(xl2);
+    };
+    fetch(row_begin + (int64_t)blockIdx.x * 8 + warp);
+    for (int64_t row = row_begin + (int64_t)blockIdx.x * 8 + warp; row < row_end; row += stride) {
         ++n_rows;
         const uint2 *cr = cand + (size_t)(row - row_begin) * G;
-        float lo = CUDART_INF_F;
-        for (int g = lane; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
+        const float2 nr = nr_n;
+        const uint2 key0 = lane < G ? key_n : make_uint2(KEY_INIT, KEY_INIT);   // this lane's group of the first 32
+        float4 x[VPL];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) x[v] = x_n[v];
+        fetch(row + stride);
+        float lo = __uint_as_float(key0.x);
+        for (int g = lane + 32; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
-        const float thr = lo + 2.f * screen_allowance(sqrtf(x2) * 1.000001f, sqrtf(xl2) * 1.000001f, cmax, cmax2, clomax, d);
+        const float thr = lo + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
 
+        if (G <= 32) {
+            // One centroid within the allowance and its group's second best outside: it is the fp32 argmin.
+            const unsigned m1 = __ballot_sync(FULL, __uint_as_float(key0.x) <= thr);
+            const unsigned mboth = __ballot_sync(FULL, __uint_as_float(key0.y) <= thr);
+            if (__popc(m1) == 1 && mboth == 0u) {
+                const int src = __ffs(m1) - 1;
+                const int kone = src * GROUP + (int)(__shfl_sync(FULL, key0.x, src) & IDX_MASK);
+                if (kone < K) {
+                    if (lane == 0) assign[row] = kone;
+                    continue;
+                }
+            }
+        }
         float best = CUDART_INF_F;
         int bidx = 0x7fffffff;
         for (int g0 = 0; g0 < G; g0 += 32) {
             const int g = g0 + lane;
-            uint2 key = make_uint2(KEY_INIT, KEY_INIT);
-            if (g < G) key = cr[g];
-            unsigned m1 = __ballot_sync(FULL, __uint_as_float(key.x) <= thr);
+            uint2 key = key0;
+            if (g0 > 0) key = g < G ? cr[g] : make_uint2(KEY_INIT, KEY_INIT);
+            const unsigned m1 = __ballot_sync(FULL, __uint_as_float(key.x) <= thr);
             const unsigned mboth = __ballot_sync(FULL, __uint_as_float(key.y) <= thr);
-            while (m1) {
-                const int src = __ffs(m1) - 1;
-                m1 &= m1 - 1;
-                const int kbase = (g0 + src) * GROUP;
-                const int kone = kbase + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
-                if ((mboth >> src) & 1u) {
-                    // two of this group's centroids cannot be told from the best: score the whole group
-                    ++n_scan;
-                    const int kend = min(K, kbase + GROUP);
-                    for (int kb = kbase; kb < kend; kb += KC) {
-                        float acc[KC];
+            // groups with one centroid inside the allowance: score those centroids (one or two of them is the
+            // usual case: a plain warp sum each; more go eight per reduction)
+            unsigned ms = m1 & ~mboth;
+            if (__popc(ms) <= 2) {
+                while (ms) {
+                    const int src = __ffs(ms) - 1;
+                    ms &= ms - 1;
+                    const int kone = (g0 + src) * GROUP + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
+                    if (kone < K) {
+                        ++n_single;
+                        const float cnk = __ldg(cn + kone);
+                        float acc = 0.f;
 #pragma unroll
-                        for (int kk = 0; kk < KC; ++kk) {
-                            acc[kk] = 0.f;
-                            if (kb + kk < kend) {
+                        for (int v = 0; v < VPL; ++v) {
+                            const int q = lane + 32 * v;
+                            if (q < d4) acc = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc);
+                        }
+                        float s = fmaf(-2.f, warp_sum(acc), cnk);
+                        s = (s == s) ? s : CUDART_INF_F;
+                        if (s < best || (s == best && kone < bidx)) {
+                            best = s;
+                            bidx = kone;
+                        }
+                    }
+                }
+            }
+            while (ms) {
+                float acc[KC];
+                int myk = -1;
+                float mycn = 0.f;
 #pragma unroll
-                                for (int v = 0; v < VPL; ++v) {
-                                    const int q = lane + 32 * v;
-                                    if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
-                                }
+                for (int kk = 0; kk < KC; ++kk) {
+                    acc[kk] = 0.f;
+                    if (ms) {
+                        const int src = __ffs(ms) - 1;
+                        ms &= ms - 1;
+                        const int kone = (g0 + src) * GROUP + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
+                        if (kone < K) {
+                            ++n_single;
+                            if (kk == slot) {
+                                myk = kone;
+                                mycn = __ldg(cn + kone);
+                            }
+#pragma unroll
+                            for (int v = 0; v < VPL; ++v) {
+                                const int q = lane + 32 * v;
+                                if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc[kk]);
                             }
                         }
-                        const float dot = reduce8_transposed(acc, lane);
-                        const int k = kb + slot;
-                        float s = k < kend ? fmaf(-2.f, dot, cn[k]) : CUDART_INF_F;
-                        s = (s == s) ? s : CUDART_INF_F;
-                        if (s < best || (s == best && k < bidx)) {
-                            best = s;
-                            bidx = k;
+                    }
+                }
+                const float dot = reduce8_transposed(acc, lane);
+                if (myk >= 0) {
+                    float s = fmaf(-2.f, dot, mycn);
+                    s = (s == s) ? s : CUDART_INF_F;
+                    if (s < best || (s == best && myk < bidx)) {
+                        best = s;
+                        bidx = myk;
+                    }
+                }
+            }
+            // groups with two inside: a third may hide behind them, so the whole group is scored
+            unsigned mscan = m1 & mboth;
+            while (mscan) {
+                const int src = __ffs(mscan) - 1;
+                mscan &= mscan - 1;
+                ++n_scan;
+                const int kbase = (g0 + src) * GROUP;
+                const int kend = min(K, kbase + GROUP);
+                for (int kb = kbase; kb < kend; kb += KC) {
+                    float acc[KC];
+#pragma unroll
+                    for (int kk = 0; kk < KC; ++kk) {
+                        acc[kk] = 0.f;
+                        if (kb + kk < kend) {
+#pragma unroll
+                            for (int v = 0; v < VPL; ++v) {
+                                const int q = lane + 32 * v;
+                                if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
+                            }
                         }
                     }
-                } else if (kone < K) {
-                    ++n_single;
-                    float acc = 0.f;
-#pragma unroll
-                    for (int v = 0; v < VPL; ++v) {
-                        const int q = lane + 32 * v;
-                        if (q < d4) acc = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc);
-                    }
-                    const float dot = warp_sum(acc);
-                    float s = fmaf(-2.f, dot, cn[kone]);
+                    const float dot = reduce8_transposed(acc, lane);
+                    const int k = kb + slot;
+                    float s = k < kend ? fmaf(-2.f, dot, cn[k]) : CUDART_INF_F;
                     s = (s == s) ? s : CUDART_INF_F;
-                    if (s < best || (s == best && kone < bidx)) {
+                    if (s < best || (s == best && k < bidx)) {
                         best = s;
-                        bidx = kone;
+                        bidx = k;
                     }
                 }
             }
@@ -410,8 +490,8 @@ int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, co
 
 // One assignment step on the tensor-core path: labels of all N rows against `centroids` / `cn`.
 int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N, int d, int K,
-                     const float *centroids, const float *cn, const float *clo, int32_t *assign, void *cand_ws,
-                     cudaStream_t stream) {
+                     const float *centroids, const float *cn, const float *clo, float *cmaxima, const float2 *rownorm,
+                     int32_t *assign, void *cand_ws, cudaStream_t stream) {
     const int num_kb = (d + KBLK - 1) / KBLK;
     const int num_nt = (K + BN - 1) / BN;
     const int G = num_nt * 2;
@@ -420,6 +500,11 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
     const size_t smem = fixed + (size_t)stages * C_STAGE_BYTES;
     EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_tc_screen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     uint2 *cand = static_cast<uint2 *>(cand_ws);
+    {
+        Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
+        centroid_maxima<<<1, 1024, 0, stream>>>(cn, clo, K, cmaxima);
+        tm.end(1);
+    }
     const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
     int launches = 0;
     for (int64_t r0 = 0; r0 < N; r0 += chunk) {
@@ -436,9 +521,9 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
         unsigned long long *counters =
             ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
         if (d <= 128)
-            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, clo, cand, assign, counters);
+            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cmaxima, rownorm, cand, assign, counters);
         else
-            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, clo, cand, assign, counters);
+            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cmaxima, rownorm, cand, assign, counters);
         tm.end(1);
         launches += 2;
     }

@@ -655,8 +655,16 @@ int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N) {
     return ceil_div(ceil_div(N, BM), kmeans_tcf_grid(ctx, N)) * 32;
 }
 
-int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, float2 *rownorm,
-                       TcFusedState *st, cudaStream_t stream) {
+// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|): what the error bound of both tensor-core paths needs of a row.
+int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *rownorm, cudaStream_t stream) {
+    Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
+    row_norms<<<(int)std::min<int64_t>((int64_t)ctx->sm_count * 16, ceil_div(N, 8)), 256, 0, stream>>>(emb, N, d, rownorm);
+    tm.end(1);
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
+}
+
+int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st) {
     st->npad = tcf_npad(K);
     st->num_kb = (d + KBLK - 1) / KBLK;
     const size_t fixed = tcf_fixed_smem(d, K);
@@ -670,10 +678,6 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     st->tmem_cols = cols;
     if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
-    Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
-    row_norms<<<(int)std::min<int64_t>((int64_t)ctx->sm_count * 16, ceil_div(N, 8)), 256, 0, stream>>>(emb, N, d, rownorm);
-    tm.end(1);
-    EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;
 }
 

@@ -29,6 +29,14 @@ import torch  # noqa: E402
 
 import synth  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries under profiles/;
+# the key carries the launch the capture covers.  Set an entry to None when its kernel changes.
+NCU_TRAFFIC = {
+    ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 163_525_376, "launch": "one row chunk of 246,272 rows",
+                                      "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
+    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_287_798_552, "launch": "all rows, one iteration",
+                                    "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
+}
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio used to derive the TF32 roof from the bf16 one
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -386,6 +394,10 @@ def main():
     dominant_name = [k for k, v in passes.items() if v is dominant][0]
     roofline = dict(dominant["roofline"])
     roofline["kernel"] = dominant_name
+    t = NCU_TRAFFIC.get((dominant_name, w.name))
+    if t and args.kmeans_path == "auto":
+        roofline["traffic"] = t["bytes_per_launch"]
+        roofline["traffic_note"] = f"{t['launch']}; {t['source']}"
     roofline["ms_per_launch"] = dominant["ms_per_launch"]
     roofline["ms_per_pass"] = dominant["ms_per_pass"]
 

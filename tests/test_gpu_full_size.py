@@ -1,0 +1,108 @@
+"""GPU parity at the benchmark's full sizes (cfg4: N = 2,449,029, d = 128, nnz ~ 123.5 M), in the launch
+configuration bench.py times.  The oracle cannot run whole Lloyd iterations at this size in seconds, so:
+labels are compared on a seeded row sample against the oracle's assignment step from the GPU's own
+C_{T-1}; centroids against an independent fp64 mean of the rows carrying each label; the rest through
+properties that hold at any size.  The graph passes are integer and are compared in full."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from parity import assert_labels_match, CENTROID_RTOL, rms_row_norm
+
+pytestmark = pytest.mark.gpu
+
+SAMPLE = 20_000
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2604_01000_b200 as ep
+    c = ep.Context(0)
+    yield c
+    c.check()
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def cfg4():
+    w = synth.WORKLOADS["cfg4"]
+    emb = synth.embeddings(w, device="cuda")
+    rows = synth.init_centroid_rows(w, max(w.K, w.reorder_K), device="cuda")
+    return w, emb, rows
+
+
+class _Step:
+    def __init__(self, assign, best1, best2):
+        self.assign, self.best1, self.best2 = assign, best1, best2
+
+
+def _check_run(ctx, emb, init, K, T, w):
+    prev = ctx.kmeans(emb, K, T - 1, init, objective=True)
+    last = ctx.kmeans(emb, K, T, init, objective=True)
+    torch.cuda.synchronize()
+    ctx.check()
+    N = emb.shape[0]
+    a = last.assign
+    assert int(a.min()) >= 0 and int(a.max()) < K
+    # the first T-1 iterations of the longer run are the shorter run, bit for bit
+    assert torch.equal(last.objective[: T - 1], prev.objective)
+    assert bool(torch.all(last.objective[1:] <= last.objective[:-1] * (1 + 1e-7)))
+    # resuming from C_{T-1} gives the same last iteration
+    step = ctx.kmeans(emb, K, 1, prev.centroids)
+    assert torch.equal(step.assign, a) and torch.equal(step.centroids, last.centroids)
+    # labels on a row sample: the oracle's assignment step against the GPU's C_{T-1}
+    s = synth.subsample_rows(w, SAMPLE, device="cuda")
+    xs = emb[s].cpu().numpy()
+    c_prev = prev.centroids.cpu().numpy().astype(np.float64)
+    ra, b1, b2 = oracle.assign_step(xs, c_prev)
+    flips = assert_labels_match(a[s].cpu().numpy(), _Step(ra, b1, b2), xs, c_prev)
+    assert flips <= SAMPLE // 1000
+    # every non-empty centroid is the mean of its rows (independent fp64 sums on the device)
+    sums = torch.zeros((K, emb.shape[1]), dtype=torch.float64, device="cuda")
+    chunk = 1 << 19
+    for r0 in range(0, N, chunk):
+        sums.index_add_(0, a[r0:r0 + chunk].long(), emb[r0:r0 + chunk].double())
+    cnt = torch.bincount(a.long(), minlength=K)
+    assert int(cnt.sum()) == N
+    mean = sums / cnt.clamp(min=1).double()[:, None]
+    got = last.centroids.double()
+    keep = cnt == 0
+    assert torch.equal(got[keep].float(), prev.centroids[keep])          # empty clusters keep their centroid
+    err = (got - mean).norm(dim=1)[~keep]
+    scale = torch.clamp(mean.norm(dim=1)[~keep], min=1e-3 * rms_row_norm(xs))
+    assert bool(torch.all(err <= CENTROID_RTOL * scale)), float((err / scale).max())
+    # the objective of the last iteration, recomputed in fp64 on the sample's share: J >= sum over the sample
+    d_s = ((torch.from_numpy(xs).double() - torch.from_numpy(c_prev)[torch.from_numpy(ra).long()]) ** 2).sum()
+    assert float(last.objective[-1]) >= float(d_s) * (1 - 1e-6)
+
+
+def test_cfg4_partition_run_full_size(ctx, cfg4):
+    w, emb, rows = cfg4
+    _check_run(ctx, emb, emb[rows[: w.K]].contiguous(), w.K, 4, w)
+
+
+def test_cfg4_reordering_run_full_size(ctx, cfg4):
+    w, emb, rows = cfg4
+    _check_run(ctx, emb, emb[rows[: w.reorder_K]].contiguous(), w.reorder_K, 2, w)
+
+
+def test_cfg4_graph_passes_full_size(ctx, cfg4):
+    w, emb, rows = cfg4
+    rowptr, colidx = synth.graph(w, device="cuda")
+    km = ctx.kmeans(emb, w.K, 3, emb[rows[: w.K]].contiguous())
+    q = ctx.partition_quality(rowptr, colidx, km.assign, w.K)
+    fine = ctx.kmeans(emb, w.reorder_K, 1, emb[rows[: w.reorder_K]].contiguous())
+    r = ctx.reorder(fine.assign, w.reorder_K)
+    torch.cuda.synchronize()
+    ctx.check()
+    a = km.assign.cpu().numpy()
+    ref = oracle.partition_quality(rowptr.cpu().numpy(), colidx.cpu().numpy(), a, w.K)
+    assert int(q.edge_cut.item()) == ref.edge_cut and ref.edge_cut % 2 == 0
+    np.testing.assert_array_equal(q.part_vertices.cpu().numpy(), ref.part_vertices)
+    np.testing.assert_array_equal(q.part_edges.cpu().numpy(), ref.part_edges)
+    assert int(ref.part_edges.sum()) == colidx.numel() and int(ref.part_vertices.sum()) == w.N
+    perm, inv = oracle.reorder(fine.assign.cpu().numpy(), w.reorder_K)
+    np.testing.assert_array_equal(r.perm.cpu().numpy(), perm)
+    np.testing.assert_array_equal(r.inv_perm.cpu().numpy(), inv)

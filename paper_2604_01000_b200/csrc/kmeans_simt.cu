@@ -426,7 +426,8 @@ __global__ void __launch_bounds__(256) objective_finalize(const double *__restri
 }
 
 constexpr int X2_BLOCKS = 1184;
-constexpr int TENSOR_MIN_K = 24;      // from here on the tensor-core path is chosen when the shape allows it
+constexpr int FUSED_TC_MIN_K = 2;     // auto: the fused tensor-core kernel from here on, when the shape allows it
+constexpr int LARGE_TC_MIN_K = 65;    // auto: screening + resolve from here on (below, d > 128 stays on the CUDA cores)
 constexpr int CN_PAD = 256;           // |c|^2 is padded to the tensor path's centroid tile
 
 template <typename F>
@@ -483,9 +484,9 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
         }
     }
     const bool tc_ok = kmeans_tc_shape_ok(ctx, d, K), tcf_ok = kmeans_tcf_shape_ok(ctx, d, K);
-    const bool want_tc = ctx->opt_kmeans_path == 2 || (ctx->opt_kmeans_path == 0 && K >= TENSOR_MIN_K);
-    p.tc_fused = tcf_ok && want_tc;
-    p.tensor = (tc_ok && want_tc) || p.tc_fused;
+    const bool forced = ctx->opt_kmeans_path == 2, autop = ctx->opt_kmeans_path == 0;
+    p.tc_fused = tcf_ok && (forced || (autop && K >= FUSED_TC_MIN_K));
+    p.tensor = p.tc_fused || (tc_ok && (forced || (autop && K >= LARGE_TC_MIN_K)));
     p.fused = !p.tensor && W >= 4 && K <= 256;
     if (p.tc_fused) {
         p.warps = 12;

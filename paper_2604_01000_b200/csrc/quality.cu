@@ -92,7 +92,12 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
 // set a bit at that position and park their label there; an entry's source label is the label at the
 // nearest set bit at or before it (or, before the first set bit, the label of the row that straddles
 // the tile start).
-template <typename RowT, typename LabT>
+//
+// PACK = 0: the label of an entry's target comes from the repacked label array in global memory (L2).
+// PACK = 8 / 4: every block first copies all labels into shared memory, one byte / one nibble each (K <= 256 /
+// K <= 16, and N small enough to fit), so that the per-entry gather never leaves the SM and the pass becomes a
+// plain stream of the column ids.
+template <typename RowT, typename LabT, int PACK>
 __global__ void __launch_bounds__(QT_THREADS) edge_cut_tiles(const RowT *__restrict__ rowptr,
                                                              const int32_t *__restrict__ colidx, int64_t nnz,
                                                              const LabT *__restrict__ lab, int64_t N,
@@ -103,9 +108,22 @@ __global__ void __launch_bounds__(QT_THREADS) edge_cut_tiles(const RowT *__restr
     __shared__ LabT headlab[QT_EDGES];
     __shared__ int warp_max[QT_THREADS / 32];
     __shared__ unsigned long long block_cut;
+    extern __shared__ __align__(16) uint8_t lab_tab[];       // PACK != 0: all labels, packed
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) block_cut = 0ull;
     unsigned long long my_cut = 0ull;
+    if (PACK == 8) {
+        for (int64_t v = tid * 4; v < N; v += QT_THREADS * 4) {      // N bytes; the array is padded to a multiple of 4
+            *reinterpret_cast<uint32_t *>(lab_tab + v) = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
+        }
+    } else if (PACK == 4) {
+        for (int64_t v = tid * 4; v < N; v += QT_THREADS * 4) {      // four labels in, two bytes out
+            const uint32_t w4 = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
+            *reinterpret_cast<uint16_t *>(lab_tab + (v >> 1)) =
+                (uint16_t)((w4 & 15u) | ((w4 >> 4) & 0xF0u) | ((w4 >> 8) & 0xF00u) | ((w4 >> 12) & 0xF000u));
+        }
+    }
+    if (PACK != 0) __syncthreads();
 
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int64_t e0 = tile * QT_EDGES;
@@ -172,10 +190,18 @@ __global__ void __launch_bounds__(QT_THREADS) edge_cut_tiles(const RowT *__restr
                     if (j > 0 && ((bits >> (b + j)) & 1u)) cur = headlab[q + j];
                     if (q + j < ne) {
                         const int col = cols[j];
-                        if ((unsigned)col < (unsigned)N)
-                            cut += (__ldg(lab + col) != cur) ? 1u : 0u;
-                        else
+                        if ((unsigned)col < (unsigned)N) {
+                            unsigned tgt;
+                            if (PACK == 8)
+                                tgt = lab_tab[col];
+                            else if (PACK == 4)
+                                tgt = (lab_tab[col >> 1] >> ((col & 1) << 2)) & 15u;
+                            else
+                                tgt = (unsigned)__ldg(lab + col);
+                            cut += (tgt != (unsigned)cur) ? 1u : 0u;
+                        } else {
                             ep_raise(status, EP_ERR_BAD_INDEX);
+                        }
                     }
                 }
             }
@@ -207,7 +233,7 @@ struct QualityBuffers {
 static size_t quality_layout(int64_t N, int64_t nnz, int K, void *ws, QualityBuffers *out) {
     Arena a(ws);
     QualityBuffers b{};
-    b.lab = a.take<char>((size_t)N * label_width(K));
+    b.lab = a.take<char>(((size_t)N + 4) * label_width(K));
     b.tile_row = a.take<int32_t>(ceil_div(nnz, QT_EDGES) + 1);
     if (out) *out = b;
     return a.used;
@@ -231,9 +257,30 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
     }
     if (ntiles > 0) {
         Timed tm(ctx, stream, EP_TIMER_EDGE_CUT);
-        const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
-        edge_cut_tiles<RowT, LabT><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
-                                                                   edge_cut, ctx->d_status);
+        // labels in shared memory when they fit beside the kernel's ~11 KB of static shared memory
+        const size_t room = (size_t)ctx->smem_optin - 12 * 1024;
+        const size_t tab4 = ((size_t)N + 7) / 8 * 4 + 16, tab8 = ((size_t)N + 3) / 4 * 4 + 16;
+        const int pack = sizeof(LabT) != 1 ? 0 : (K <= 16 && tab4 <= room) ? 4 : (tab8 <= room) ? 8 : 0;
+        // worth it only when the copy (N bytes per block) is small beside the block's share of the entries
+        const bool use_tab = pack != 0 && (int64_t)N * ctx->sm_count <= nnz * 2;
+        if (use_tab) {
+            const size_t tab = pack == 4 ? tab4 : tab8;
+            const int per_sm = 2 * (tab + 12 * 1024) <= (size_t)ctx->smem_optin ? 2 : 1;
+            const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * per_sm);
+            if (pack == 4) {
+                auto kern = edge_cut_tiles<RowT, LabT, 4>;
+                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));
+                kern<<<grid, QT_THREADS, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status);
+            } else {
+                auto kern = edge_cut_tiles<RowT, LabT, 8>;
+                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));
+                kern<<<grid, QT_THREADS, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status);
+            }
+        } else {
+            const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
+            edge_cut_tiles<RowT, LabT, 0><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
+                                                                         edge_cut, ctx->d_status);
+        }
         tm.end(1);
     }
     EP_CUDA(ctx, cudaGetLastError());

@@ -53,6 +53,16 @@ def test_scaled_configs(ctx, name, N):
     _quality_matches(ctx, rowptr, colidx, _random_labels(N, w.K, 2), w.K)
 
 
+@pytest.mark.parametrize("N,K", [(6_007, 2), (6_007, 16), (6_007, 17), (6_007, 200), (9_001, 256), (5_003, 300)])
+def test_dense_graph_label_tables_in_shared_memory(ctx, N, K):
+    """Dense graphs with few vertices: the kernel variants that keep all labels in shared memory, as nibbles
+    (K <= 16) or bytes (K <= 256), and the global-memory gather beyond."""
+    w = synth.scaled(synth.WORKLOADS["cfg3"], N)
+    rowptr, colidx = synth.graph(w, device="cuda")
+    _quality_matches(ctx, rowptr, colidx, _random_labels(N, K, N + K), K)
+    _quality_matches(ctx, rowptr.to(torch.int64), colidx, _random_labels(N, K, N + K + 1), K)
+
+
 @pytest.mark.parametrize("K", [1, 2, 255, 256, 257, 5000, 70_000])
 def test_label_widths(ctx, K):
     N = 80_000

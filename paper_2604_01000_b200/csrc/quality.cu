@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
 // K <= 16, and N small enough to fit), so that the per-entry gather never leaves the SM and the pass becomes a
 // plain stream of the column ids.
 template <typename RowT, typename LabT, int PACK>
-__global__ void __launch_bounds__(QT_THREADS) edge_cut_tiles(const RowT *__restrict__ rowptr,
+__global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__restrict__ rowptr,
                                                              const int32_t *__restrict__ colidx, int64_t nnz,
                                                              const LabT *__restrict__ lab, int64_t N,
                                                              const int32_t *__restrict__ tile_row, int64_t ntiles,
@@ -258,14 +258,15 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
     if (ntiles > 0) {
         Timed tm(ctx, stream, EP_TIMER_EDGE_CUT);
         // labels in shared memory when they fit beside the kernel's ~11 KB of static shared memory
-        const size_t room = (size_t)ctx->smem_optin - 12 * 1024;
+        // (two blocks per SM must fit: one block alone has too few warps to hide the stream's latency)
+        const size_t room = (size_t)ctx->smem_optin / 2 - 12 * 1024;
         const size_t tab4 = ((size_t)N + 7) / 8 * 4 + 16, tab8 = ((size_t)N + 3) / 4 * 4 + 16;
         const int pack = sizeof(LabT) != 1 ? 0 : (K <= 16 && tab4 <= room) ? 4 : (tab8 <= room) ? 8 : 0;
         // worth it only when the copy (N bytes per block) is small beside the block's share of the entries
         const bool use_tab = pack != 0 && (int64_t)N * ctx->sm_count <= nnz * 2;
         if (use_tab) {
             const size_t tab = pack == 4 ? tab4 : tab8;
-            const int per_sm = 2 * (tab + 12 * 1024) <= (size_t)ctx->smem_optin ? 2 : 1;
+            const int per_sm = (int)std::min<size_t>(4, (size_t)ctx->smem_optin / (tab + 12 * 1024));
             const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * per_sm);
             if (pack == 4) {
                 auto kern = edge_cut_tiles<RowT, LabT, 4>;

@@ -256,6 +256,21 @@ def run_reference(args, w, rank):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------------------ ranks
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's device time: what a whole-job rate has to be divided by."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, units_per_rank_per_step: int, steps: int, ms: float) -> float:
+    """Units all ranks processed (every rank runs its own replica of the workload) per second."""
+    return world * units_per_rank_per_step * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -328,13 +343,10 @@ def main():
     counters = ctx.debug_counters()
     timers = {(g, t): ctx.profile_read(t, g) for g in (0, 1) for t in ep.binding.TIMERS}
     ctx.check()
-    if dist is not None:
-        tms = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
+    ms = max_over_ranks(ms, dist, device)
 
     row_iters = w.N * (w.iters + w.reorder_iters)
-    value = world * row_iters * args.steps / (ms * 1e-3)
+    value = whole_job_rate(world, row_iters, args.steps, ms)
 
     # ---- per-pass rates and rooflines from the library's event timers -----------------------------------
     hbm = peaks["hbm_gbs"]
@@ -419,12 +431,9 @@ def main():
         stop.record()
         barrier()
         ems = start.elapsed_time(stop)
-        if dist is not None:
-            tms = torch.tensor([ems], dtype=torch.float64, device=device)
-            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-            ems = float(tms.item())
+        ems = max_over_ranks(ems, dist, device)
         ctx.check()
-        e2e = {"value": world * row_iters * e_steps / (ems * 1e-3), "unit": "rows*iters/s",
+        e2e = {"value": whole_job_rate(world, row_iters, e_steps, ems), "unit": "rows*iters/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ems / e_steps, "steps": e_steps,
                "api": "ep_kmeans_host / ep_partition_quality_host / ep_reorder_host with page-locked host buffers"}
 

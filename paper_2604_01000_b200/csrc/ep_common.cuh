@@ -119,8 +119,8 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
 struct TcFusedState;
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tcf_state_bytes();
-int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N);
-int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N);
+int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N, int d);
+int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N, int d);
 int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *rownorm, cudaStream_t stream);
 int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st);
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,

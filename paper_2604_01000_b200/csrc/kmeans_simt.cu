@@ -362,7 +362,7 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_norms(const float *__res
 // c_k <- S_k / n_k when n_k > 0, else unchanged; also |c_k|^2 of the new centroid and this
 // cluster's share of the objective, n_k |c|^2 - 2 c.S_k with c the centroid the rows were assigned
 // against (the rows' own sum of |x|^2 is added once by objective_finalize).
-__global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__restrict__ psum,
+__global__ void __launch_bounds__(UPD_THREADS) centroid_update_few(const float *__restrict__ psum,
                                                                const int *__restrict__ pcnt, int parts, int K, int d,
                                                                float *C, float *cnorm, double *objterm,
                                                                int keep_centroids, float *__restrict__ ct,
@@ -393,6 +393,76 @@ __global__ void __launch_bounds__(UPD_THREADS) centroid_update(const float *__re
     t_cs = block_sum_fixed<UPD_THREADS>(t_cs, buf);
     t_cc = block_sum_fixed<UPD_THREADS>(t_cc, buf);
     t_nn = block_sum_fixed<UPD_THREADS>(t_nn, buf);
+    if (threadIdx.x == 0) {
+        cnorm[k] = (float)t_nn;
+        objterm[k] = (double)n * t_cc - 2.0 * t_cs;
+        if (clo) clo[k] = (float)(sqrt(t_lo) * 1.000001);
+    }
+}
+
+// The same update for many slabs (the fused kernels leave one or two per SM), one block of 1024 per cluster.  S_k = sum over the partial slabs in fp64: with
+// G = UPD2_THREADS / dpad thread groups, group g adds its contiguous share of the slabs in slab order and the
+// group sums are then added in group order (a fixed tree: results repeat).  c_k <- S_k / n_k when n_k > 0,
+// else unchanged; also |c_k|^2 of the new centroid and this cluster's share of the objective,
+// n_k |c|^2 - 2 c.S_k with c the centroid the rows were assigned against (the rows' own sum of |x|^2 is
+// added once by objective_finalize).
+constexpr int UPD2_THREADS = 1024;
+
+__global__ void __launch_bounds__(UPD2_THREADS) centroid_update_many(const float *__restrict__ psum,
+                                                                const int *__restrict__ pcnt, int parts, int K, int d,
+                                                                float *C, float *cnorm, double *objterm,
+                                                                int keep_centroids, float *__restrict__ ct,
+                                                                float *__restrict__ clo) {
+    __shared__ double buf[UPD2_THREADS];
+    __shared__ long long n_s;
+    const int k = blockIdx.x;
+    const int dpad = (d + 31) / 32 * 32;
+    const int G = max(1, UPD2_THREADS / dpad);            // dpad <= 1024
+    const int g = threadIdx.x / dpad, j = threadIdx.x - g * dpad;
+    const bool mine = g < G && j < d;
+    {   // n_k: integer, any order
+        long long n = 0;
+        for (int p = threadIdx.x; p < parts; p += UPD2_THREADS) n += pcnt[(size_t)p * K + k];
+        buf[threadIdx.x] = (double)n;                     // counts are far below 2^53: exact
+        __syncthreads();
+        for (int s2 = UPD2_THREADS / 2; s2 > 0; s2 >>= 1) {
+            if ((int)threadIdx.x < s2) buf[threadIdx.x] += buf[threadIdx.x + s2];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) n_s = (long long)buf[0];
+        __syncthreads();
+    }
+    const long long n = n_s;
+    double part = 0.0;
+    if (mine) {
+        const int p0 = (int)((long long)parts * g / G), p1 = (int)((long long)parts * (g + 1) / G);
+        for (int p = p0; p < p1; ++p) part += (double)psum[((size_t)p * K + k) * d + j];
+    }
+    buf[threadIdx.x] = part;
+    __syncthreads();
+    double t_cs = 0.0, t_cc = 0.0, t_nn = 0.0, t_lo = 0.0;
+    if (g == 0 && j < d) {
+        double S = buf[j];
+        for (int gg = 1; gg < G; ++gg) S += buf[gg * dpad + j];
+        const float cold = C[(size_t)k * d + j];
+        float cnew = cold;
+        if (n > 0 && !keep_centroids) cnew = (float)(S / (double)n);
+        t_cs = (double)cold * S;
+        t_cc = (double)cold * (double)cold;
+        t_nn = (double)cnew * (double)cnew;
+        C[(size_t)k * d + j] = cnew;
+        if (clo) {   // tensor-core paths: what the next screening pass will not see of this centroid
+            const float r = tf32_image(cnew, ct != nullptr);
+            if (ct) ct[(size_t)k * d + j] = r;
+            const double lo = (double)cnew - (double)r;
+            t_lo = lo * lo;
+        }
+    }
+    __syncthreads();
+    if (clo) t_lo = block_sum_fixed<UPD2_THREADS>(t_lo, buf);
+    t_cs = block_sum_fixed<UPD2_THREADS>(t_cs, buf);
+    t_cc = block_sum_fixed<UPD2_THREADS>(t_cc, buf);
+    t_nn = block_sum_fixed<UPD2_THREADS>(t_nn, buf);
     if (threadIdx.x == 0) {
         cnorm[k] = (float)t_nn;
         objterm[k] = (double)n * t_cc - 2.0 * t_cs;
@@ -491,7 +561,7 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
     if (p.tc_fused) {
         p.warps = 12;
         p.smem = 0;
-        p.grid = kmeans_tcf_grid(ctx, N);
+        p.grid = kmeans_tcf_grid(ctx, N, d);
         p.parts = 2 * p.grid;   // the fused kernel's slabs, then those of the kernel for the rows it left undecided
     } else if (p.fused) {
         p.warps = W;
@@ -530,7 +600,7 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
     if (p.tensor) {
         b.rownorm = a.take<float2>(p.N);
         if (p.tc_fused) {
-            b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N) * 4 * p.grid);
+            b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N, p.d) * 4 * p.grid);
             b.late_count = a.take<int>((size_t)4 * p.grid);
         } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
@@ -619,7 +689,11 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
         });
         if (rc != EP_OK) return rc;
         Timed tm(ctx, stream, EP_TIMER_KMEANS_UPDATE);
-        centroid_update<<<K, UPD_THREADS, 0, stream>>>(b.psum, b.pcnt, p.parts, K, d, centroids, b.cnorm, b.objterm,
+        if (p.parts >= 32 && d <= 512)
+            centroid_update_many<<<K, UPD2_THREADS, 0, stream>>>(b.psum, b.pcnt, p.parts, K, d, centroids, b.cnorm, b.objterm,
+                                                         iters == 0 ? 1 : 0, b.ct, b.clo);
+        else
+            centroid_update_few<<<K, UPD_THREADS, 0, stream>>>(b.psum, b.pcnt, p.parts, K, d, centroids, b.cnorm, b.objterm,
                                                        iters == 0 ? 1 : 0, b.ct, b.clo);
         if (objective) objective_finalize<<<1, 256, 0, stream>>>(b.x2part, X2_BLOCKS, b.objterm, K, objective + t);
         tm.end(objective ? 2 : 1);

@@ -33,14 +33,34 @@ using namespace eptc;
 
 constexpr int BM = 128;                 // rows per tile = TMEM lanes
 constexpr int KBLK = 32;                // floats in one 128-byte swizzle row
-constexpr int MAX_KB = 4;               // d <= 128
-constexpr int X_KB_BYTES = BM * 128;    // one k-block of a row tile
+constexpr int MAX_KB = 8;               // d <= 256
 constexpr int MAX_STAGES = 8;
 constexpr int THREADS = 512;            // warp 0 TMA, 1 MMA, 2..3 sorting (2 also owns TMEM), 4..7 screen, 8..15 accumulate
 constexpr int S_WARP0 = 4;
 constexpr int A_WARP0 = 8;
 constexpr int A_WARPS = 8;
 constexpr int MAX_K = 64;
+
+// Phase clocks for tuning (compiled in with -DEP_PHASE_CLOCKS only): thread 0 of a warp set adds up how long
+// it waited and how long it worked, into the diagnostic counters.
+#ifdef EP_PHASE_CLOCKS
+#define EP_CLK_DECL long long pc_wait = 0, pc_work = 0, pc_t = clock64();
+#define EP_CLK(var)                        \
+    {                                      \
+        const long long now_ = clock64();  \
+        var += now_ - pc_t;                \
+        pc_t = now_;                       \
+    }
+#define EP_CLK_OUT(cond, iw, ik)                                      \
+    if (counters && (cond)) {                                         \
+        atomicAdd(&counters[iw], (unsigned long long)pc_wait);        \
+        atomicAdd(&counters[ik], (unsigned long long)pc_work);        \
+    }
+#else
+#define EP_CLK_DECL
+#define EP_CLK(var)
+#define EP_CLK_OUT(cond, iw, ik)
+#endif
 
 struct FusedShared {
     uint64_t x_full[MAX_STAGES], x_empty[MAX_STAGES];
@@ -73,11 +93,13 @@ __device__ __forceinline__ void tmem_issue16(uint32_t taddr, uint32_t (&v)[VN]) 
 }
 __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// KMAX = 32 or 64: upper bound of K.  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - tf32(c_k)|;
+// KMAX = 32 or 64: upper bound of K.  VPL = 16-byte chunks of a row per lane: 1 for d <= 128 with tiles of 128
+// rows, 2 for d <= 256 with tiles of 64 rows (the stage stays 64 KB; the MMA still spans 128 TMEM lanes, the upper
+// 64 of which then hold scores of whatever follows the tile in shared memory and are never read).  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - tf32(c_k)|;
 // cn = |c_k|^2 padded with a huge value.  Block b leaves the sums of the rows it decided in psum[b][K][d],
 // their counts in pcnt[b][K], and per screen warp w the undecided rows in late_list[(4 b + w) late_cap ..]
 // (x = row id, y and z = mask of the centroids within the bound), late_count[4 b + w] of them.
-template <int KMAX>
+template <int KMAX, int VPL>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
                 const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
@@ -94,6 +116,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (threadIdx.x < 4) late_count[blockIdx.x * 4 + threadIdx.x] = 0;
         return;
     }
+    constexpr int BMR = BM / VPL;                      // rows per tile
+    constexpr int SWARPS = BMR / 32;                   // screen warps with rows
+    constexpr int X_KB_BYTES = BMR * 128;              // one k-block of a row tile
     const int stage_bytes = num_kb * X_KB_BYTES;
     const int c_kb_bytes = npad * 128;
     uint8_t *x_smem = smem;                                          // [stages][num_kb][128 rows][128 B]
@@ -103,7 +128,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int d4 = d >> 2;
-    const int64_t num_tiles = (N + BM - 1) / BM;
+    const int64_t num_tiles = (N + BMR - 1) / BMR;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_STAGES; ++i) {
@@ -113,8 +138,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         mbar_init(&sh->c_full, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh->t_full[i], 1);
-            mbar_init(&sh->t_empty[i], 4);    // the screen warps
-            mbar_init(&sh->lab_full[i], 4);
+            mbar_init(&sh->t_empty[i], SWARPS);   // the screen warps
+            mbar_init(&sh->lab_full[i], SWARPS);
             mbar_init(&sh->lab_empty[i], 1);  // a sorting warp
             mbar_init(&sh->ord_full[i], 1);
             mbar_init(&sh->ord_empty[i], A_WARPS);
@@ -151,7 +176,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 mbar_expect_tx(&sh->x_full[s], (uint32_t)stage_bytes);
                 for (int kb = 0; kb < num_kb; ++kb)
                     tma_load_2d(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK,
-                                (int)(tile * BM), &sh->x_full[s]);
+                                (int)(tile * BMR), &sh->x_full[s]);
             }
         }
     } else if (warp == 1) {
@@ -184,14 +209,17 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // so that an accumulate warp finds the rows of a cluster as one run, in row order.
         const uint32_t hw = (uint32_t)warp - 2u;
         const unsigned lt = (1u << lane) - 1u;
+        EP_CLK_DECL
         for (uint32_t it = hw;; it += 2) {
             const int64_t tile = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
             if (tile >= num_tiles) break;
             const uint32_t par = hw, use = (it >> 1) & 1u;
+            EP_CLK(pc_work)
             if (!mbar_wait(&sh->lab_full[par], use, abort_flag)) break;
+            EP_CLK(pc_wait)
             int l[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) l[j] = sh->lab[par][j * 32 + lane];
+            for (int j = 0; j < 4; ++j) l[j] = j < SWARPS ? (int)sh->lab[par][j * 32 + lane] : MAX_K;
             for (int i = lane; i <= MAX_K; i += 32) sh->hcnt[hw][i] = 0;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->lab_empty[par]);
@@ -218,7 +246,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const int ex = inc - t0 - t1;
             if (t0) atomicAdd(&sh->cnt[2 * lane], t0);       // integer: exact whatever the order
             if (t1) atomicAdd(&sh->cnt[2 * lane + 1], t1);
+            EP_CLK(pc_work)
             if (!mbar_wait(&sh->ord_empty[par], use ^ 1u, abort_flag)) break;
+            EP_CLK(pc_wait)
             sh->goff[par][2 * lane] = ex;
             sh->goff[par][2 * lane + 1] = ex + t0;
             if (lane == 31) sh->goff[par][MAX_K] = inc;
@@ -233,6 +263,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->ord_full[par]);
         }
+        EP_CLK_OUT(warp == 2 && lane == 0, 4, 5)
     } else if (warp >= S_WARP0 && warp < A_WARP0) {
         // ---------------------------------------------------------------- screen warps: one row per thread,
         // each warp on its own (no barrier between them): TMEM lanes 32 sw .. 32 sw + 31 = rows of the tile
@@ -254,20 +285,23 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         int4 *late_rows = late_list + ((size_t)blockIdx.x * 4 + sw) * late_cap;
         int late_n = 0;
         unsigned n_rows = 0;
+        EP_CLK_DECL
 
         float2 nr_next = make_float2(0.f, 0.f);            // this row's norms, fetched one tile ahead
-        if ((int64_t)blockIdx.x * BM + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BM + stid);
+        if (sw < SWARPS && (int64_t)blockIdx.x * BMR + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BMR + stid);
 
         uint32_t it = 0;
-        for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+        for (int64_t tile = blockIdx.x; sw < SWARPS && tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u, par = it & 1u;
-            const int64_t row = tile * BM + stid;
+            const int64_t row = tile * BMR + stid;
             const float2 nr = nr_next;
             {
-                const int64_t nrow = (tile + gridDim.x) * BM + stid;
+                const int64_t nrow = (tile + gridDim.x) * BMR + stid;
                 if (nrow < N) nr_next = __ldg(rownorm + nrow);
             }
+            EP_CLK(pc_work)
             if (!mbar_wait(&sh->t_full[buf], use, abort_flag)) break;
+            EP_CLK(pc_wait)
             tc_fence_after();
             // ---- all of this row's screened products into registers, then the accumulator is free again
             const uint32_t taddr = tmem_base + ((uint32_t)(sw * 32) << 16) + buf * (uint32_t)npad;
@@ -336,11 +370,14 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 ++n_rows;
             }
             // ---- hand the labels to the sorting warp
+            EP_CLK(pc_work)
             if (!mbar_wait(&sh->lab_empty[par], use ^ 1u, abort_flag)) break;
+            EP_CLK(pc_wait)
             sh->lab[par][stid] = (uint8_t)label;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->lab_full[par]);
         }
+        EP_CLK_OUT(stid == 0, 1, 2)
         if (lane == 0) late_count[blockIdx.x * 4 + sw] = late_n;   // always written: the next kernel trusts it
         if (counters) {
 #pragma unroll
@@ -354,37 +391,52 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---------------------------------------------------------------- accumulate warps
         const int aw = warp - A_WARP0;                     // owns clusters aw, aw + 8, ...
         constexpr int OWN = KMAX / A_WARPS;
-        const bool has_cols = lane < d4;                   // this lane's 16-byte chunk of a row is chunk `lane`
-        const uint32_t lx = (uint32_t)(lane & 7) << 4;     // its place inside a 128-byte swizzle row, before the swizzle
-        float4 acc[OWN];
+        const uint32_t lx = (uint32_t)(lane & 7) << 4;     // a lane's place inside a 128-byte swizzle row, before the swizzle
+        float4 acc[OWN][VPL];                              // this lane's 16-byte chunks of a row are lane, lane + 32
 #pragma unroll
-        for (int i = 0; i < OWN; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < OWN; ++i)
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) acc[i][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        EP_CLK_DECL
         uint32_t it = 0;
         for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t s = it % (uint32_t)stages;
             const uint32_t par = it & 1u, use = (it >> 1) & 1u;
-            const uint8_t *xl = x_smem + (size_t)s * stage_bytes + (size_t)(lane >> 3) * X_KB_BYTES;   // this lane's k-block
+            const uint8_t *xl = x_smem + (size_t)s * stage_bytes + (size_t)(lane >> 3) * X_KB_BYTES;   // this lane's first k-block
+            EP_CLK(pc_work)
             if (!mbar_wait(&sh->ord_full[par], use, abort_flag)) break;
             if (!mbar_wait(&sh->x_full[s], (it / (uint32_t)stages) & 1u, abort_flag)) break;   // long complete: makes the tile visible here
+            EP_CLK(pc_wait)
+            int q0[OWN], q1[OWN];                          // the runs of this warp's clusters in order[]
 #pragma unroll
             for (int i = 0; i < OWN; ++i) {
-                const int k = aw + A_WARPS * i;
-                if (k < K) {
-                    const int p1 = sh->goff[par][k + 1];
-                    for (int p = sh->goff[par][k]; p < p1; p += 4) {   // four rows at a time: loads first, adds in row order
-                        float4 x[4];
+                const int k = min(aw + A_WARPS * i, K - 1);
+                q0[i] = sh->goff[par][k];
+                q1[i] = aw + A_WARPS * i < K ? sh->goff[par][k + 1] : q0[i];
+            }
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const uint32_t o = sh->order[par][min(p + u, p1 - 1)];
-                            x[u] = has_cols ? *reinterpret_cast<const float4 *>(xl + (o ^ lx)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
+            for (int i = 0; i < OWN; ++i) {
+                const int p1 = q1[i];
+                for (int p = q0[i]; p < p1; p += 4) {       // four rows at a time: loads first, adds in row order
+                    float4 x[4][VPL];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (p + u < p1) {
-                                acc[i].x += x[u].x;
-                                acc[i].y += x[u].y;
-                                acc[i].z += x[u].z;
-                                acc[i].w += x[u].w;
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t o = sh->order[par][min(p + u, p1 - 1)];
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v)
+                            x[u][v] = lane + 32 * v < d4
+                                          ? *reinterpret_cast<const float4 *>(xl + (size_t)(4 * v) * X_KB_BYTES + (o ^ lx))
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (p + u < p1) {
+#pragma unroll
+                            for (int v = 0; v < VPL; ++v) {
+                                acc[i][v].x += x[u][v].x;
+                                acc[i][v].y += x[u][v].y;
+                                acc[i][v].z += x[u][v].z;
+                                acc[i][v].w += x[u][v].w;
                             }
                         }
                     }
@@ -396,12 +448,17 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 mbar_arrive(&sh->ord_empty[par]);
             }
         }
+        EP_CLK_OUT(aw == 0 && lane == 0, 6, 7)
         // ---- publish this block's sums: every (cluster, chunk) has exactly one owner
         float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
 #pragma unroll
         for (int i = 0; i < OWN; ++i) {
             const int k = aw + A_WARPS * i;
-            if (k < K && has_cols) out[(size_t)k * d4 + lane] = acc[i];
+            if (k < K) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v)
+                    if (lane + 32 * v < d4) out[(size_t)k * d4 + lane + 32 * v] = acc[i][v];
+            }
         }
     }
     __syncthreads();
@@ -424,6 +481,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 constexpr int LATE_THREADS = 512;
 constexpr int LATE_LABELS = 4096;
 
+template <int VPL>
 __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__restrict__ emb, int64_t N, int d, int K,
                                                                  int kpad, const float *__restrict__ C,
                                                                  const float *__restrict__ cn,
@@ -437,15 +495,16 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
     __shared__ uint8_t lab_s[LATE_LABELS];                   // labels of the block's first LATE_LABELS listed rows
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
     const int nwarps = blockDim.x >> 5;
-    float4 *cs = late_smem;                                  // [kpad][32] centroids, zero padded
-    float4 *tab = cs + (size_t)kpad * 32;                    // [4][K][32] per-list sums
-    float *cns = reinterpret_cast<float *>(tab + (size_t)4 * K * 32);   // [kpad]
+    constexpr int RP = 32 * VPL;                             // 16-byte chunks per (padded) row
+    float4 *cs = late_smem;                                  // [kpad][RP] centroids, zero padded
+    float4 *tab = cs + (size_t)kpad * RP;                    // [4][K][RP] per-list sums
+    float *cns = reinterpret_cast<float *>(tab + (size_t)4 * K * RP);   // [kpad]
     int *cw = reinterpret_cast<int *>(cns + kpad);           // [4][K]
-    for (int i = threadIdx.x; i < kpad * 32; i += blockDim.x) {
-        const int k = i >> 5, q = i & 31;
+    for (int i = threadIdx.x; i < kpad * RP; i += blockDim.x) {
+        const int k = i / RP, q = i - k * RP;
         cs[i] = (k < K && q < d4) ? __ldg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    for (int i = threadIdx.x; i < 4 * K * 32; i += blockDim.x) tab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = threadIdx.x; i < 4 * K * RP; i += blockDim.x) tab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = threadIdx.x; i < kpad; i += blockDim.x) cns[i] = i < K ? cn[i] : CUDART_INF_F;
     for (int i = threadIdx.x; i < 4 * K; i += blockDim.x) cw[i] = 0;
     if (threadIdx.x < 4) ncount[threadIdx.x] = (int)min((int64_t)max(late_count[blockIdx.x * 4 + threadIdx.x], 0), late_cap);
@@ -461,6 +520,13 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
     __syncthreads();
     const int4 *lists = late_list + (size_t)blockIdx.x * 4 * late_cap;
     const int slot = lane_chunk_slot(lane);
+    // this lane's 16-byte chunks (lane, lane + 32) of row r; zeros for r < 0
+    auto load_row = [&](float4 (&x)[VPL], int r) {
+#pragma unroll
+        for (int v = 0; v < VPL; ++v)
+            x[v] = (r >= 0 && lane + 32 * v < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane + 32 * v)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
     // ---- 1. labels, the rows' data fetched four ahead
     constexpr int AHEAD1 = 4;
     for (int p0 = warp * 32; p0 < cum[4]; p0 += nwarps * 32) {
@@ -472,24 +538,20 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
             e = lists[(size_t)w * late_cap + (p - cum[w])];
             if (e.x < 0 || e.x >= N) e.x = -1;               // never index outside the matrix, whatever the list holds
         }
-        float4 xq[AHEAD1];
+        float4 xq[AHEAD1][VPL];
 #pragma unroll
-        for (int u = 0; u < AHEAD1; ++u) {
-            const int r = __shfl_sync(FULL, e.x, u);
-            xq[u] = (r >= 0 && lane < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane)
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        for (int u = 0; u < AHEAD1; ++u) load_row(xq[u], __shfl_sync(FULL, e.x, u));
         for (int i0 = 0; i0 < cnt; i0 += AHEAD1) {
 #pragma unroll
             for (int u = 0; u < AHEAD1; ++u) {
                 const int i = i0 + u;
-                const float4 x = xq[u];
+                float4 x[VPL];
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) x[v] = xq[u][v];
                 const int row = __shfl_sync(FULL, e.x, i & 31);
                 const uint32_t mlo = (uint32_t)__shfl_sync(FULL, e.y, i & 31), mhi = (uint32_t)__shfl_sync(FULL, e.z, i & 31);
                 const int rn = __shfl_sync(FULL, e.x, (i + AHEAD1) & 31);
-                xq[u] = (i + AHEAD1 < cnt && rn >= 0 && lane < d4)
-                            ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)rn * d4 + lane)
-                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                load_row(xq[u], i + AHEAD1 < cnt ? rn : -1);
                 if (i >= cnt || row < 0) continue;
                 unsigned long long m = ((unsigned long long)mhi << 32) | mlo;
                 if (K < 64) m &= (1ull << K) - 1ull;
@@ -506,7 +568,8 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
                             const int k = __ffsll((long long)m) - 1;
                             m &= m - 1;
                             if (kk == slot) myk = k;
-                            a[kk] = dot4(x, cs[k * 32 + lane], 0.f);
+#pragma unroll
+                            for (int v = 0; v < VPL; ++v) a[kk] = dot4(x[v], cs[k * RP + lane + 32 * v], a[kk]);
                         }
                     }
                     const float dot = reduce8_transposed(a, lane);
@@ -541,8 +604,8 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
     if (warp < 4) {
         const int n = cum[warp + 1] - cum[warp];
         const int4 *rows = lists + (size_t)warp * late_cap;
-        float4 *mytab = tab + (size_t)warp * K * 32;
-        constexpr int AHEAD = 8;
+        float4 *mytab = tab + (size_t)warp * K * RP;
+        constexpr int AHEAD = 8 / VPL;
         for (int j0 = 0; j0 < n; j0 += 32) {
             const int cnt = min(32, n - j0);
             int row_l = -1, lab_l = -1;
@@ -551,30 +614,29 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
                 if (row_l < 0 || row_l >= N) row_l = -1;
                 if (row_l >= 0) lab_l = cum[warp] + j0 + lane < LATE_LABELS ? (int)lab_s[cum[warp] + j0 + lane] : assign[row_l];
             }
-            float4 xq[AHEAD];
+            float4 xq[AHEAD][VPL];
 #pragma unroll
-            for (int u = 0; u < AHEAD; ++u) {
-                const int r = __shfl_sync(FULL, row_l, u);
-                xq[u] = (r >= 0 && lane < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane)
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int u = 0; u < AHEAD; ++u) load_row(xq[u], __shfl_sync(FULL, row_l, u));
             for (int i0 = 0; i0 < cnt; i0 += AHEAD) {
 #pragma unroll
                 for (int u = 0; u < AHEAD; ++u) {
                     const int i = i0 + u;
-                    const float4 x = xq[u];
+                    float4 x[VPL];
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) x[v] = xq[u][v];
                     const int a = __shfl_sync(FULL, lab_l, i & 31);
                     const int rn = __shfl_sync(FULL, row_l, (i + AHEAD) & 31);
-                    xq[u] = (i + AHEAD < cnt && rn >= 0 && lane < d4)
-                                ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)rn * d4 + lane)
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    load_row(xq[u], i + AHEAD < cnt ? rn : -1);
                     if (i < cnt && a >= 0 && a < K) {
-                        float4 t = mytab[a * 32 + lane];
-                        t.x += x.x;
-                        t.y += x.y;
-                        t.z += x.z;
-                        t.w += x.w;
-                        mytab[a * 32 + lane] = t;
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            float4 t = mytab[a * RP + lane + 32 * v];
+                            t.x += x[v].x;
+                            t.y += x[v].y;
+                            t.z += x[v].z;
+                            t.w += x[v].w;
+                            mytab[a * RP + lane + 32 * v] = t;
+                        }
                         if (lane == 0) cw[warp * K + a] += 1;
                     }
                 }
@@ -586,9 +648,9 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
     float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
     for (int i = threadIdx.x; i < K * d4; i += blockDim.x) {
         const int k = i / d4, q = i - k * d4;
-        float4 t = tab[k * 32 + q];
+        float4 t = tab[k * RP + q];
         for (int w = 1; w < 4; ++w) {
-            const float4 u = tab[((size_t)w * K + k) * 32 + q];
+            const float4 u = tab[((size_t)w * K + k) * RP + q];
             t.x += u.x;
             t.y += u.y;
             t.z += u.z;
@@ -635,6 +697,8 @@ size_t kmeans_tcf_state_bytes() { return sizeof(TcFusedState); }
 
 static inline int tcf_npad(int K) { return std::max(16, (K + 15) / 16 * 16); }
 
+static inline int tcf_tile_rows(int d) { return d <= 128 ? BM : BM / 2; }
+
 static size_t tcf_fixed_smem(int d, int K) {
     const int num_kb = (d + KBLK - 1) / KBLK;
     return (size_t)num_kb * tcf_npad(K) * 128 + sizeof(FusedShared);
@@ -642,17 +706,18 @@ static size_t tcf_fixed_smem(int d, int K) {
 
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K) {
     if (d < KBLK || d > MAX_KB * KBLK || K < 1 || K > MAX_K) return false;
+    if (d > 128 && K > 32) return false;   // the fp32 kernel's sum tables must fit in shared memory
     const int num_kb = (d + KBLK - 1) / KBLK;
-    return tcf_fixed_smem(d, K) + 2 * (size_t)num_kb * X_KB_BYTES <= (size_t)ctx->smem_optin;
+    return tcf_fixed_smem(d, K) + 2 * (size_t)num_kb * tcf_tile_rows(d) * 128 <= (size_t)ctx->smem_optin;
 }
 
-int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N) {
-    return (int)std::max<int64_t>(1, std::min<int64_t>(ctx->sm_count, ceil_div(N, BM)));
+int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N, int d) {
+    return (int)std::max<int64_t>(1, std::min<int64_t>(ctx->sm_count, ceil_div(N, tcf_tile_rows(d))));
 }
 
 // Entries of one screen warp's list of undecided rows: every row it can ever see.
-int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N) {
-    return ceil_div(ceil_div(N, BM), kmeans_tcf_grid(ctx, N)) * 32;
+int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N, int d) {
+    return ceil_div(ceil_div(N, tcf_tile_rows(d)), kmeans_tcf_grid(ctx, N, d)) * 32;
 }
 
 // rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|): what the error bound of both tensor-core paths needs of a row.
@@ -668,24 +733,24 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     st->npad = tcf_npad(K);
     st->num_kb = (d + KBLK - 1) / KBLK;
     const size_t fixed = tcf_fixed_smem(d, K);
-    const size_t stage = (size_t)st->num_kb * X_KB_BYTES;
+    const size_t stage = (size_t)st->num_kb * tcf_tile_rows(d) * 128;
     st->stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / stage);
     st->smem = fixed + (size_t)st->stages * stage;
-    st->grid = kmeans_tcf_grid(ctx, N);
-    st->late_cap = kmeans_tcf_late_cap(ctx, N);
+    st->grid = kmeans_tcf_grid(ctx, N, d);
+    st->late_cap = kmeans_tcf_late_cap(ctx, N, d);
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)st->npad) cols <<= 1;
     st->tmem_cols = cols;
-    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, BM) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
+    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, tcf_tile_rows(d)) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
     return EP_OK;
 }
 
-template <int KMAX>
+template <int KMAX, int VPL>
 static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo, const float2 *rownorm,
                       int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, int4 *late_list, int *late_count,
                       cudaStream_t stream) {
-    auto kern = kmeans_tc_fused<KMAX>;
+    auto kern = kmeans_tc_fused<KMAX, VPL>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
     unsigned long long *counters =
         ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
@@ -704,16 +769,19 @@ int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, con
                       const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
                       int *pcnt, void *late_list_ws, int *late_count, cudaStream_t stream) {
     int4 *late_list = static_cast<int4 *>(late_list_ws);
-    int rc = K <= 32 ? tcf_launch<32>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
-                     : tcf_launch<64>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream);
+    const int vpl = d <= 128 ? 1 : 2;
+    int rc = vpl == 2 ? tcf_launch<32, 2>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
+             : K <= 32 ? tcf_launch<32, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
+                       : tcf_launch<64, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream);
     if (rc != EP_OK) return rc;
     const int kpad = (K + KC - 1) / KC * KC;
-    const size_t smem = (size_t)kpad * 512 + (size_t)4 * K * 512 + (size_t)kpad * 4 + (size_t)4 * K * 4;
-    EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_late_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t row = 512 * (size_t)vpl;
+    const size_t smem = (size_t)kpad * row + (size_t)4 * K * row + (size_t)kpad * 4 + (size_t)4 * K * 4;
+    auto late = vpl == 1 ? kmeans_late_rows<1> : kmeans_late_rows<2>;
+    EP_CUDA(ctx, cudaFuncSetAttribute(late, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
-    kmeans_late_rows<<<st.grid, LATE_THREADS, smem, stream>>>(emb, N, d, K, kpad, centroids, cn, late_list, st.late_cap,
-                                                              late_count, assign, psum + (size_t)st.grid * K * d,
-                                                              pcnt + (size_t)st.grid * K);
+    late<<<st.grid, LATE_THREADS, smem, stream>>>(emb, N, d, K, kpad, centroids, cn, late_list, st.late_cap, late_count, assign,
+                                                  psum + (size_t)st.grid * K * d, pcnt + (size_t)st.grid * K);
     tm.end(1);
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;

@@ -77,7 +77,8 @@ def test_large_k_label_only_path(ctx, K, N, d, iters):
 @pytest.mark.parametrize("K,N,d,iters", [(2, 1_000, 32, 3), (5, 129, 64, 2), (32, 30_011, 128, 4), (64, 25_013, 128, 3),
                                          (100, 7_001, 100, 2), (256, 9_973, 256, 2), (257, 6_007, 36, 2),
                                          (300, 12_007, 128, 3), (1024, 9_001, 64, 2), (4096, 20_003, 128, 2),
-                                         (700, 3_001, 224, 2)])
+                                         (700, 3_001, 224, 2), (16, 9_973, 256, 3), (32, 5_003, 200, 2), (5, 700, 132, 2),
+                                         (1, 300, 256, 2)])
 def test_tensor_core_path(ctx, K, N, d, iters):
     """The tcgen05 screening + fp32 resolve path, forced for every shape it accepts: labels must be the
     exact fp32 argmin, so the same tolerances apply as on the CUDA-core path."""

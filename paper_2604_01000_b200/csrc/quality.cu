@@ -174,38 +174,44 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
             lasthead[tid] = excl;
         }
         __syncthreads();
-        unsigned cut = 0;
+        unsigned cut = 0, bad = 0;
+        // one vector of four entries: their source label from the bitmap, their targets' labels gathered
+        auto vec = [&](int q, const int4 &cv, bool full) {
+            const int wd = q >> 5, b = q & 31;
+            const unsigned bits = bitmap[wd];
+            const unsigned upto = bits & (0xffffffffu >> (31 - b));
+            const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
+            LabT cur = head >= 0 ? headlab[head] : carry;
+            const int cols[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-        for (int i = 0; i < QT_VEC; ++i) {
-            const int q = (i * QT_THREADS + tid) * 4;
-            if (q < ne) {
-                const int wd = q >> 5, b = q & 31;
-                const unsigned bits = bitmap[wd];
-                const unsigned upto = bits & (0xffffffffu >> (31 - b));
-                const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
-                LabT cur = head >= 0 ? headlab[head] : carry;
-                const int cols[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+            for (int j = 0; j < 4; ++j) {
+                if (j > 0 && ((bits >> (b + j)) & 1u)) cur = headlab[q + j];
+                const bool live = full || q + j < ne;
+                const int col = cols[j];
+                const bool in = (unsigned)col < (unsigned)N;
+                const int cc = in ? col : 0;                 // an index outside [0, N) is reported, never followed
+                unsigned tgt;
+                if (PACK == 8)
+                    tgt = lab_tab[cc];
+                else if (PACK == 4)
+                    tgt = (lab_tab[cc >> 1] >> ((cc & 1) << 2)) & 15u;
+                else
+                    tgt = (unsigned)__ldg(lab + cc);
+                cut += (live && in && tgt != (unsigned)cur) ? 1u : 0u;
+                bad |= (live && !in) ? 1u : 0u;
+            }
+        };
+        if (ne == QT_EDGES) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (j > 0 && ((bits >> (b + j)) & 1u)) cur = headlab[q + j];
-                    if (q + j < ne) {
-                        const int col = cols[j];
-                        if ((unsigned)col < (unsigned)N) {
-                            unsigned tgt;
-                            if (PACK == 8)
-                                tgt = lab_tab[col];
-                            else if (PACK == 4)
-                                tgt = (lab_tab[col >> 1] >> ((col & 1) << 2)) & 15u;
-                            else
-                                tgt = (unsigned)__ldg(lab + col);
-                            cut += (tgt != (unsigned)cur) ? 1u : 0u;
-                        } else {
-                            ep_raise(status, EP_ERR_BAD_INDEX);
-                        }
-                    }
-                }
+            for (int i = 0; i < QT_VEC; ++i) vec((i * QT_THREADS + tid) * 4, c[i], true);
+        } else {
+#pragma unroll
+            for (int i = 0; i < QT_VEC; ++i) {
+                const int q = (i * QT_THREADS + tid) * 4;
+                if (q < ne) vec(q, c[i], false);
             }
         }
+        if (bad) ep_raise(status, EP_ERR_BAD_INDEX);
         my_cut += cut;
     }
 #pragma unroll

@@ -141,7 +141,8 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) digit_scatter(const int32_t *
                                                                   int32_t *__restrict__ vals_out,
                                                                   int32_t *__restrict__ inv_out) {
     __shared__ int cnt[SORT_WARPS][RADIX];
-    __shared__ int gbase[RADIX];
+    __shared__ int gbase[RADIX], dstart[RADIX], wtot[SORT_WARPS];
+    __shared__ int sval[SORT_TILE], skey[SORT_TILE];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < SORT_WARPS * RADIX; i += blockDim.x) (&cnt[0][0])[i] = 0;
     gbase[threadIdx.x] = offsets[(size_t)threadIdx.x * ntiles + blockIdx.x];
@@ -168,7 +169,8 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) digit_scatter(const int32_t *
         __syncwarp();
     }
     __syncthreads();
-    {   // per digit: turn the warps' counts into exclusive offsets inside the tile
+    {   // per digit: turn the warps' counts into exclusive offsets inside the tile, and the digits' totals
+        // into the place where each digit's run starts in the tile's sorted order
         const int dg = threadIdx.x;
         int run = 0;
 #pragma unroll
@@ -177,19 +179,41 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) digit_scatter(const int32_t *
             cnt[w][dg] = run;
             run += c;
         }
+        int inc = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(FULL, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) wtot[warp] = inc;
+        __syncthreads();
+        int add = 0;
+        for (int w = 0; w < warp; ++w) add += wtot[w];
+        dstart[dg] = add + inc - run;
     }
     __syncthreads();
+    // stage the tile in sorted order, so that the global writes below go out as contiguous runs per digit
 #pragma unroll
     for (int i = 0; i < SORT_ITEMS; ++i) {
         const int64_t idx = base + i * 32 + lane;
         if (idx < N) {
             const int dg = (key[i] >> shift) & (RADIX - 1);
-            const int dst = gbase[dg] + cnt[warp][dg] + rank[i];
+            const int within = cnt[warp][dg] + rank[i];
             const int val = vals_in ? vals_in[idx] : (int)idx;
-            vals_out[dst] = val;
-            if (keys_out) keys_out[dst] = key[i];
-            if (inv_out) inv_out[val] = dst;
+            const int lp = dstart[dg] + within;
+            sval[lp] = val;
+            skey[lp] = key[i];
+            if (inv_out) inv_out[val] = gbase[dg] + within;
         }
+    }
+    __syncthreads();
+    const int ntile = (int)min((int64_t)SORT_TILE, N - (int64_t)blockIdx.x * SORT_TILE);
+    for (int q = threadIdx.x; q < ntile; q += blockDim.x) {
+        const int k = skey[q];
+        const int dg = (k >> shift) & (RADIX - 1);
+        const int dst = gbase[dg] + (q - dstart[dg]);
+        vals_out[dst] = sval[q];
+        if (keys_out) keys_out[dst] = k;
     }
 }
 

@@ -97,27 +97,41 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
 // PACK = 8 / 4: every block first copies all labels into shared memory, one byte / one nibble each (K <= 256 /
 // K <= 16, and N small enough to fit), so that the per-entry gather never leaves the SM and the pass becomes a
 // plain stream of the column ids.
-template <typename RowT, typename LabT, int PACK>
-__global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__restrict__ rowptr,
-                                                             const int32_t *__restrict__ colidx, int64_t nnz,
-                                                             const LabT *__restrict__ lab, int64_t N,
-                                                             const int32_t *__restrict__ tile_row, int64_t ntiles,
-                                                             unsigned long long *edge_cut, int *status) {
-    __shared__ unsigned bitmap[QT_WORDS];
-    __shared__ int lasthead[QT_WORDS];
-    __shared__ LabT headlab[QT_EDGES];
-    __shared__ int warp_max[QT_THREADS / 32];
+//
+// GROUPS = 1: a block is one group of QT_THREADS threads.  GROUPS = 4: a block of 1024 threads holds four such
+// groups, each with its own tile, bitmap and named barrier, sharing one copy of the label table: the form for a
+// table so large that only one block fits on an SM, which still needs 32 warps to hide the stream's latency.
+template <typename RowT, typename LabT, int PACK, int GROUPS>
+__global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
+    edge_cut_tiles(const RowT *__restrict__ rowptr, const int32_t *__restrict__ colidx, int64_t nnz,
+                   const LabT *__restrict__ lab, int64_t N, const int32_t *__restrict__ tile_row, int64_t ntiles,
+                   unsigned long long *edge_cut, int *status) {
+    __shared__ unsigned bitmap_[GROUPS][QT_WORDS];
+    __shared__ int lasthead_[GROUPS][QT_WORDS];
+    __shared__ LabT headlab_[GROUPS][QT_EDGES];
+    __shared__ int warp_max_[GROUPS][QT_THREADS / 32];
     __shared__ unsigned long long block_cut;
     extern __shared__ __align__(16) uint8_t lab_tab[];       // PACK != 0: all labels, packed
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) block_cut = 0ull;
+    const int grp = GROUPS == 1 ? 0 : (int)(threadIdx.x / QT_THREADS);
+    unsigned *bitmap = bitmap_[grp];
+    int *lasthead = lasthead_[grp];
+    LabT *headlab = headlab_[grp];
+    int *warp_max = warp_max_[grp];
+    auto group_sync = [&]() {
+        if (GROUPS == 1)
+            __syncthreads();
+        else
+            asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(QT_THREADS) : "memory");
+    };
+    const int tid = threadIdx.x % QT_THREADS, lane = tid & 31, warp = tid >> 5;
+    if (threadIdx.x == 0) block_cut = 0ull;
     unsigned long long my_cut = 0ull;
     if (PACK == 8) {
-        for (int64_t v = tid * 4; v < N; v += QT_THREADS * 4) {      // N bytes; the array is padded to a multiple of 4
+        for (int64_t v = threadIdx.x * 4; v < N; v += QT_THREADS * GROUPS * 4) {   // N bytes; the array is padded to a multiple of 4
             *reinterpret_cast<uint32_t *>(lab_tab + v) = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
         }
     } else if (PACK == 4) {
-        for (int64_t v = tid * 4; v < N; v += QT_THREADS * 4) {      // four labels in, two bytes out
+        for (int64_t v = threadIdx.x * 4; v < N; v += QT_THREADS * GROUPS * 4) {   // four labels in, two bytes out
             const uint32_t w4 = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
             *reinterpret_cast<uint16_t *>(lab_tab + (v >> 1)) =
                 (uint16_t)((w4 & 15u) | ((w4 >> 4) & 0xF0u) | ((w4 >> 8) & 0xF00u) | ((w4 >> 12) & 0xF000u));
@@ -125,7 +139,7 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
     }
     if (PACK != 0) __syncthreads();
 
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    for (int64_t tile = (int64_t)blockIdx.x * GROUPS + grp; tile < ntiles; tile += (int64_t)gridDim.x * GROUPS) {
         const int64_t e0 = tile * QT_EDGES;
         const int ne = (int)min((int64_t)QT_EDGES, nnz - e0);
         const int4 *src = reinterpret_cast<const int4 *>(colidx + e0);
@@ -143,9 +157,9 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
                 c[i].w = -1;
             }
         }
-        __syncthreads();                                    // previous tile fully consumed
+        group_sync();                                    // previous tile fully consumed
         bitmap[tid] = 0u;
-        __syncthreads();
+        group_sync();
         const int64_t r_lo = tile_row[tile], r_hi = tile_row[tile + 1];
         const LabT carry = lab[r_lo];
         for (int64_t r = r_lo + tid; r <= r_hi; r += QT_THREADS) {
@@ -156,7 +170,7 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
                 headlab[h] = lab[r];
             }
         }
-        __syncthreads();
+        group_sync();
         {   // lasthead[w] = position of the last set bit in words < w, or -1
             const unsigned wbits = bitmap[tid];
             const int mine = wbits ? tid * 32 + 31 - __clz(wbits) : -1;
@@ -169,11 +183,11 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
             if (lane == 31) warp_max[warp] = inc;
             int excl = __shfl_up_sync(FULL, inc, 1);
             if (lane == 0) excl = -1;
-            __syncthreads();
+            group_sync();
             for (int w = 0; w < warp; ++w) excl = max(excl, warp_max[w]);
             lasthead[tid] = excl;
         }
-        __syncthreads();
+        group_sync();
         unsigned cut = 0, bad = 0;
         // one vector of four entries: their source label from the bitmap, their targets' labels gathered
         auto vec = [&](int q, const int4 &cv, bool full) {
@@ -219,7 +233,7 @@ __global__ void __launch_bounds__(QT_THREADS, 4) edge_cut_tiles(const RowT *__re
     __syncthreads();
     if (lane == 0 && my_cut) atomicAdd(&block_cut, my_cut);
     __syncthreads();
-    if (tid == 0 && block_cut) atomicAdd(edge_cut, block_cut);
+    if (threadIdx.x == 0 && block_cut) atomicAdd(edge_cut, block_cut);
 }
 
 template <typename LabT>
@@ -263,30 +277,37 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
     }
     if (ntiles > 0) {
         Timed tm(ctx, stream, EP_TIMER_EDGE_CUT);
-        // labels in shared memory when they fit beside the kernel's ~11 KB of static shared memory
-        // (two blocks per SM must fit: one block alone has too few warps to hide the stream's latency)
-        const size_t room = (size_t)ctx->smem_optin / 2 - 12 * 1024;
+        // labels in shared memory when they fit beside the kernel's static shared memory (about 10.3 KB per group)
+        const size_t stat1 = 12 * 1024, stat4 = 44 * 1024;
         const size_t tab4 = ((size_t)N + 7) / 8 * 4 + 16, tab8 = ((size_t)N + 3) / 4 * 4 + 16;
+        const size_t room = (size_t)ctx->smem_optin - stat4;
         const int pack = sizeof(LabT) != 1 ? 0 : (K <= 16 && tab4 <= room) ? 4 : (tab8 <= room) ? 8 : 0;
         // worth it only when the copy (N bytes per block) is small beside the block's share of the entries
         const bool use_tab = pack != 0 && (int64_t)N * ctx->sm_count <= nnz * 2;
-        if (use_tab) {
+        bool launched = false;
+        if constexpr (sizeof(LabT) == 1) if (use_tab) {
+            launched = true;
             const size_t tab = pack == 4 ? tab4 : tab8;
-            const int per_sm = (int)std::min<size_t>(4, (size_t)ctx->smem_optin / (tab + 12 * 1024));
-            const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * per_sm);
-            if (pack == 4) {
-                auto kern = edge_cut_tiles<RowT, LabT, 4>;
-                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));
-                kern<<<grid, QT_THREADS, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status);
-            } else {
-                auto kern = edge_cut_tiles<RowT, LabT, 8>;
-                EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));
-                kern<<<grid, QT_THREADS, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status);
-            }
-        } else {
+            // four small blocks per SM while four copies of the table fit, else one block of four groups
+            const bool small = (tab + stat1) * 4 <= (size_t)ctx->smem_optin;
+#define EP_EC(P, G)                                                                                                  \
+    do {                                                                                                             \
+        auto kern = edge_cut_tiles<RowT, LabT, P, G>;                                                                \
+        EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));             \
+        const int grid = (int)std::min<int64_t>(ceil_div(ntiles, (int64_t)G), (int64_t)ctx->sm_count * (G == 1 ? 4 : 1)); \
+        kern<<<grid, QT_THREADS * G, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut,       \
+                                                    ctx->d_status);                                                  \
+    } while (0)
+            if (pack == 4 && small) EP_EC(4, 1);
+            else if (pack == 4) EP_EC(4, 4);
+            else if (small) EP_EC(8, 1);
+            else EP_EC(8, 4);
+#undef EP_EC
+        }
+        if (!launched) {
             const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
-            edge_cut_tiles<RowT, LabT, 0><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
-                                                                         edge_cut, ctx->d_status);
+            edge_cut_tiles<RowT, LabT, 0, 1><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
+                                                                            edge_cut, ctx->d_status);
         }
         tm.end(1);
     }

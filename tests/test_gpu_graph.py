@@ -53,10 +53,12 @@ def test_scaled_configs(ctx, name, N):
     _quality_matches(ctx, rowptr, colidx, _random_labels(N, w.K, 2), w.K)
 
 
-@pytest.mark.parametrize("N,K", [(6_007, 2), (6_007, 16), (6_007, 17), (6_007, 200), (9_001, 256), (5_003, 300)])
+@pytest.mark.parametrize("N,K", [(6_007, 2), (6_007, 16), (6_007, 17), (6_007, 200), (9_001, 256), (5_003, 300),
+                                 (100_003, 16), (60_013, 200), (180_001, 9)])
 def test_dense_graph_label_tables_in_shared_memory(ctx, N, K):
     """Dense graphs with few vertices: the kernel variants that keep all labels in shared memory, as nibbles
-    (K <= 16) or bytes (K <= 256), and the global-memory gather beyond."""
+    (K <= 16) or bytes (K <= 256), and the global-memory gather beyond.  The larger N are tables of which only one
+    copy fits on an SM: the 1024-thread form whose four thread groups share it."""
     w = synth.scaled(synth.WORKLOADS["cfg3"], N)
     rowptr, colidx = synth.graph(w, device="cuda")
     _quality_matches(ctx, rowptr, colidx, _random_labels(N, K, N + K), K)
@@ -85,6 +87,24 @@ def test_odd_csr_shapes(ctx):
     for dtype in (torch.int32, torch.int64):
         rp = torch.from_numpy(rowptr).to(dtype).cuda()
         for K in (3, 300):
+            _quality_matches(ctx, rp, torch.from_numpy(colidx).cuda(), _random_labels(N, K, 4), K)
+
+
+def test_odd_csr_shapes_one_table_per_sm(ctx):
+    """Long rows, empty runs and unsorted entries through the 1024-thread form (table too large for two blocks)."""
+    rng = np.random.default_rng(19)
+    N = 110_000
+    deg = rng.integers(0, 200, size=N)
+    deg[rng.integers(0, N, size=40)] = rng.integers(5_000, 40_000, size=40)
+    deg[2000:30_000] = 0
+    deg[-3:] = 0
+    rowptr = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+    nnz = int(rowptr[-1])
+    assert nnz * 2 >= N * 148
+    colidx = rng.integers(0, N, size=nnz).astype(np.int32)
+    for dtype in (torch.int32, torch.int64):
+        rp = torch.from_numpy(rowptr).to(dtype).cuda()
+        for K in (5, 130):
             _quality_matches(ctx, rp, torch.from_numpy(colidx).cuda(), _random_labels(N, K, 4), K)
 
 

@@ -32,10 +32,6 @@ import synth  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries under profiles/;
 # the key carries the launch the capture covers.  Set an entry to None when its kernel changes.
 NCU_TRAFFIC = {
-    ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 163_525_376, "launch": "one row chunk of 246,272 rows",
-                                      "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
-    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_287_798_552, "launch": "all rows, one iteration",
-                                    "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
 }
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio used to derive the TF32 roof from the bf16 one
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -453,7 +449,8 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "passes": passes,
             "tensor_path_counters": {"rows_screened": counters[0], "large_K_single_evals": counters[1],
-                                     "large_K_group_scans": counters[2], "small_K_rows_left_to_fp32_kernel": counters[3]},
+                                     "large_K_group_scans": counters[2], "small_K_rows_left_to_fp32_kernel": counters[3],
+                                     "large_K_rows_left_to_fp32_kernel": counters[4]},
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

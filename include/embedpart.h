@@ -54,9 +54,10 @@ enum {
                                (read with ep_profile_read); 0 = off (default) */
     EP_OPT_TIMER_GROUP = 3, /* 0..3: calls made while group g is selected log into timers
                                g * EP_TIMER_COUNT + timer, so a caller can tell two calls apart */
-    EP_OPT_KMEANS_CAND_MB = 4 /* 1..4096 (default 64): upper bound in MiB of the candidate-key buffer the
-                               tensor-core path keeps in the workspace; rows are processed in chunks that
-                               fit it (never less than one pass of the grid).  Set it before the workspace
+    EP_OPT_KMEANS_CAND_MB = 4 /* 1..32768 (default 1024): upper bound in MiB of the candidate-key buffer the
+                               tensor-core path keeps in the workspace (64 bytes per row and 1024 centroids);
+                               rows are processed in chunks that fit it (never less than one pass of the
+                               grid), and fewer, longer chunks run faster.  Set it before the workspace
                                query: it changes the answer */
 };
 
@@ -97,7 +98,8 @@ int64_t ep_launch_count(const ep_ctx *ctx);
 /* Diagnostic counters kept while EP_OPT_PROFILE is 1; synchronises the device, copies the 8 counters to
  * out [host, 8 x int64] and clears them.  Tensor-core K-Means paths: [0] rows screened, [1] centroids the
  * large-K path re-evaluated singly in fp32, [2] groups of 128 centroids it re-evaluated whole, [3] rows the
- * fused small-K kernel left to the fp32 kernel; the rest are reserved. */
+ * fused small-K kernel left to the fp32 kernel, [4] rows the large-K screening kernel left to the fp32
+ * kernel; the rest are reserved. */
 int ep_debug_counters(ep_ctx *ctx, int64_t *out);
 
 /* --------------------------------------------------------------------------------------------

@@ -87,7 +87,7 @@ int ep_create(ep_ctx **out, int device) {
     ctx->opt_kmeans_path = 0;
     ctx->opt_profile = 0;
     ctx->opt_timer_group = 0;
-    ctx->opt_cand_mb = 64;
+    ctx->opt_cand_mb = 1024;
     ctx->launches = 0;
     ctx->last_error[0] = 0;
     DeviceGuard g(device);
@@ -138,7 +138,7 @@ int ep_set_option(ep_ctx *ctx, int option, int value) {
         ctx->opt_timer_group = value;
         return EP_OK;
     }
-    if (option == EP_OPT_KMEANS_CAND_MB && value >= 1 && value <= 4096) {
+    if (option == EP_OPT_KMEANS_CAND_MB && value >= 1 && value <= 32768) {
         ctx->opt_cand_mb = value;
         return EP_OK;
     }

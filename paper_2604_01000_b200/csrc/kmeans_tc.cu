@@ -6,12 +6,14 @@
 //   - centroid tiles of 256 rows stream through a ring of shared-memory stages (TMA, L2-resident);
 //   - one thread issues tcgen05.mma kind::tf32 into one of two 256-column TMEM accumulators;
 //   - eight epilogue warps read the other accumulator back (tcgen05.ld) and keep, per row and per group
-//     of 128 centroids, the two smallest scores with the column index packed into the low mantissa bits.
-// TF32 keeps 10 mantissa bits of each operand, so these scores only screen.  kmeans_tc_resolve then
-// re-evaluates in fp32 every centroid that the TF32 error bound cannot exclude: the best of each group
-// whose best is within the bound of the row's overall best, and a whole group when its second best is
-// within the bound as well (its hidden third might be).  The label is the exact fp32 argmin with the
-// lowest index winning ties, as on the CUDA-core path.
+//     of 128 centroids, the two smallest scores with the column index packed into the low mantissa bits,
+//     and the two smallest of the whole row.
+// TF32 keeps 10 mantissa bits of each operand, so these scores only screen.  A row whose second smallest
+// score lies outside the TF32 error bound of its smallest has its label at once: the screen kernel writes
+// it.  The other rows go on a list, and kmeans_tc_resolve re-evaluates in fp32 every centroid that the
+// bound cannot exclude: the best of each group whose best is within the bound of the row's overall best,
+// and a whole group when its second best is within the bound as well (its hidden third might be).  The
+// label is the exact fp32 argmin with the lowest index winning ties, as on the CUDA-core path.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -48,6 +50,9 @@ struct TcShared {
     uint64_t t_full[2], t_empty[2];
     uint32_t tmem_base;
     int abort;
+    uint64_t h_full[4][4];                 // [tile & 3][32-row quarter]: the warp of columns 128..255 has left its result
+    float4 other_half[4][BM];              // (smallest key, second smallest, group of the smallest) per row; four tiles
+                                           // deep, which is further than the two accumulators let one warp run ahead
 };
 
 // Screening pass over the rows [row_begin, row_end): for row r and group g (centroids [128 g, 128 g + 128))
@@ -55,10 +60,16 @@ struct TcShared {
 // cn holds |c_k|^2 for k < K and a huge finite value up to the next multiple of 256.  key_mask is
 // ~(GROUP - 1); it arrives as an argument so that clearing the index bits and inserting the (compile-
 // time) index stay one three-input logic operation instead of two with an immediate each.
+// A row with a single centroid inside the allowance (see screen_allowance) gets assign[r] here; every
+// other row is appended to slow_list (row numbers, any order) and counted in *slow_count, which the caller
+// has zeroed.  counters, when given, receives the number of rows screened in word 0.
 __global__ void __launch_bounds__(TC_THREADS, 1)
 kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
                  const float *__restrict__ cn, int64_t row_begin, int64_t row_end, int num_kb, int num_nt, int stages,
-                 int G, uint32_t key_mask, uint2 *__restrict__ cand, int *status) {
+                 int G, uint32_t key_mask, int d, int K, const float *__restrict__ cmaxima,
+                 const float2 *__restrict__ rownorm, uint2 *__restrict__ cand, int32_t *__restrict__ assign,
+                 int32_t *__restrict__ slow_list, int *__restrict__ slow_count, unsigned long long *counters,
+                 int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *x_smem = smem;                                         // [num_kb][128 rows][128 B]
@@ -82,6 +93,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             mbar_init(&sh->t_full[i], 1);
             mbar_init(&sh->t_empty[i], EPI_WARPS);
         }
+        for (int i = 0; i < 16; ++i) mbar_init(&sh->h_full[i >> 2][i & 3], 1);
         sh->abort = 0;
         sh->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -152,10 +164,16 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // ---------------------------------------------------------------- epilogue
         const int quad = warp & 3;                         // TMEM lanes 32 quad .. 32 quad + 31 belong to this warp
         const int half = (warp - EPI_WARP0) >> 2;          // which 128 of the accumulator's 256 columns
-        uint32_t acc = 0;
+        const float cmax2 = cmaxima[0], clomax = cmaxima[1];   // largest |c_k|^2 and largest rounding residual
+        const float cmax = sqrtf(cmax2) * 1.000001f;
+        uint32_t acc = 0, n_live = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
             const int64_t row = row_begin + tile * BM + quad * 32 + lane;
+            float2 nr = make_float2(0.f, 0.f);
+            if (half == 0 && row < row_end) nr = __ldg(rownorm + row);
+            float run1 = __uint_as_float(KEY_INIT), run2 = run1;   // the row's two smallest keys over this half's groups
+            int rung = 0;                                          // group of run1
             for (int nt = 0; ok && nt < num_nt; ++nt, ++acc) {
                 const uint32_t buf = acc & 1u, use = (acc >> 1) & 1u;
                 if (!(ok = mbar_wait(&sh->t_full[buf], use, abort_flag))) break;
@@ -188,9 +206,46 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
                 const float k1 = fminf(a1, b1);
                 const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
+                const int g = nt * 2 + half;
                 if (row < row_end)
-                    cand[(size_t)(row - row_begin) * G + (nt * 2 + half)] = make_uint2(__float_as_uint(k1), __float_as_uint(k2));
+                    cand[(size_t)(row - row_begin) * G + g] = make_uint2(__float_as_uint(k1), __float_as_uint(k2));
+                rung = k1 < run1 ? g : rung;
+                run2 = fminf(fmaxf(run1, k1), fminf(run2, k2));
+                run1 = fminf(run1, k1);
             }
+            if (!ok) break;
+            // the two warps that own these 32 rows meet
+            float4 *slot = &sh->other_half[lt & 3][quad * 32 + lane];
+            if (half == 1) {
+                *slot = make_float4(run1, run2, __int_as_float(rung), 0.f);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->h_full[lt & 3][quad]);
+            } else {
+                if (!(ok = mbar_wait(&sh->h_full[lt & 3][quad], (uint32_t)((lt >> 2) & 1), abort_flag))) break;
+                const float4 o = *slot;
+                const float lo = fminf(run1, o.x);
+                const float second = fminf(fmaxf(run1, o.x), fminf(run2, o.y));
+                const int glo = o.x < run1 ? __float_as_int(o.z) : rung;
+                const int kone = glo * GROUP + (int)(__float_as_uint(lo) & IDX_MASK);
+                const float thr = lo + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
+                const bool live = row < row_end;
+                // one centroid inside the allowance, every other one outside: it is the fp32 argmin
+                const bool fast = live && second > thr && kone < K;
+                if (fast) assign[row] = kone;
+                n_live += live ? 1u : 0u;
+                const unsigned slow = __ballot_sync(FULL, live && !fast);
+                if (slow) {
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(slow_count, __popc(slow));
+                    base = __shfl_sync(FULL, base, 0);
+                    if (live && !fast) slow_list[base + __popc(slow & ((1u << lane) - 1u))] = (int32_t)(row - row_begin);
+                }
+            }
+        }
+        if (counters && half == 0) {
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) n_live += __shfl_xor_sync(FULL, n_live, o);
+            if (lane == 0 && n_live) atomicAdd(&counters[0], (unsigned long long)n_live);
         }
     }
     __syncthreads();
@@ -236,32 +291,38 @@ __global__ void __launch_bounds__(1024) centroid_maxima(const float *__restrict_
     }
 }
 
-// Exact fp32 decision for the rows [row_begin, row_end) from the screening keys.  One warp per row;
-// lane l holds the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.
-// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|), computed once per call.
+// Exact fp32 decision for the rows the screening pass listed (slow_list holds row numbers relative to
+// row_begin, *slow_count of them).  One warp per row; lane l holds the 16-byte slices l, l+32, ... of the
+// row, as in the CUDA-core kernels.  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|), computed once per call.
 template <int VPL>
-__global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin,
-                                                         int64_t row_end, int d, int K, int G,
-                                                         const float *__restrict__ C, const float *__restrict__ cn,
+__global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin, int rows, int d, int K,
+                                                         int G, const float *__restrict__ C,
+                                                         const float *__restrict__ cn,
                                                          const float *__restrict__ cmaxima,
                                                          const float2 *__restrict__ rownorm,
-                                                         const uint2 *__restrict__ cand, int32_t *__restrict__ assign,
-                                                         unsigned long long *counters) {
+                                                         const uint2 *__restrict__ cand,
+                                                         const int32_t *__restrict__ slow_list,
+                                                         const int *__restrict__ slow_count,
+                                                         int32_t *__restrict__ assign, unsigned long long *counters) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
     const float cmax2 = cmaxima[0], clomax = cmaxima[1];   // largest |c_k|^2 and largest rounding residual
     const float cmax = sqrtf(cmax2) * 1.000001f;
     unsigned long long n_single = 0, n_scan = 0, n_rows = 0;
     const float4 *C4 = reinterpret_cast<const float4 *>(C);
     const int slot = lane_chunk_slot(lane);
+    const int n_slow = min(*slow_count, rows);            // the list never holds more than the chunk's rows
+    auto entry = [&](int64_t i) { return i < n_slow ? min(max(slow_list[i], 0), rows - 1) : -1; };
 
-    // Each warp fetches its next row (keys, norms, the row itself) while it works on the current one.
-    const int64_t stride = (int64_t)gridDim.x * 8;
+    // Each warp fetches its next row (keys, norms, the row itself) while it works on the current one, and
+    // the list entry after that.
+    const int stride = (int)gridDim.x * 8;
     uint2 key_n = make_uint2(KEY_INIT, KEY_INIT);
     float2 nr_n = make_float2(0.f, 0.f);
     float4 x_n[VPL];
-    auto fetch = [&](int64_t r) {
-        if (r < row_end) {
-            if (lane < G) key_n = cand[(size_t)(r - row_begin) * G + lane];
+    auto fetch = [&](int rel) {
+        if (rel >= 0) {
+            const int64_t r = row_begin + rel;
+            if (lane < G) key_n = cand[(size_t)rel * G + lane];
             nr_n = __ldg(rownorm + r);
 #pragma unroll
             for (int v = 0; v < VPL; ++v) {
@@ -270,37 +331,31 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
             }
         }
     };
-    fetch(row_begin + (int64_t)blockIdx.x * 8 + warp);
-    for (int64_t row = row_begin + (int64_t)blockIdx.x * 8 + warp; row < row_end; row += stride) {
+    const int first = (int)blockIdx.x * 8 + warp;
+    int rel = entry(first);
+    int rel_n = entry((int64_t)first + stride);
+    fetch(rel);
+    for (int i = first; i < n_slow; i += stride) {
         ++n_rows;
-        const uint2 *cr = cand + (size_t)(row - row_begin) * G;
+        const int64_t row = row_begin + rel;
+        const uint2 *cr = cand + (size_t)rel * G;
         const float2 nr = nr_n;
         const uint2 key0 = lane < G ? key_n : make_uint2(KEY_INIT, KEY_INIT);   // this lane's group of the first 32
         float4 x[VPL];
 #pragma unroll
         for (int v = 0; v < VPL; ++v) x[v] = x_n[v];
-        fetch(row + stride);
+        rel = rel_n;
+        rel_n = entry((int64_t)i + 2 * (int64_t)stride);
+        fetch(rel);
         float lo = __uint_as_float(key0.x);
         for (int g = lane + 32; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
         const float thr = lo + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
 
-        if (G <= 32) {
-            // One centroid within the allowance and its group's second best outside: it is the fp32 argmin.
-            const unsigned m1 = __ballot_sync(FULL, __uint_as_float(key0.x) <= thr);
-            const unsigned mboth = __ballot_sync(FULL, __uint_as_float(key0.y) <= thr);
-            if (__popc(m1) == 1 && mboth == 0u) {
-                const int src = __ffs(m1) - 1;
-                const int kone = src * GROUP + (int)(__shfl_sync(FULL, key0.x, src) & IDX_MASK);
-                if (kone < K) {
-                    if (lane == 0) assign[row] = kone;
-                    continue;
-                }
-            }
-        }
         float best = CUDART_INF_F;
         int bidx = 0x7fffffff;
+        bool lanes_differ = false;                 // set once a lane holds a score the others do not
         for (int g0 = 0; g0 < G; g0 += 32) {
             const int g = g0 + lane;
             uint2 key = key0;
@@ -310,29 +365,48 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
             // groups with one centroid inside the allowance: score those centroids (one or two of them is the
             // usual case: a plain warp sum each; more go eight per reduction)
             unsigned ms = m1 & ~mboth;
-            if (__popc(ms) <= 2) {
-                while (ms) {
-                    const int src = __ffs(ms) - 1;
+            if (__popc(ms) <= 4) {
+                while (ms) {   // two at a time: their loads and their reductions overlap
+                    const int src0 = __ffs(ms) - 1;
                     ms &= ms - 1;
-                    const int kone = (g0 + src) * GROUP + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
-                    if (kone < K) {
-                        ++n_single;
-                        const float cnk = __ldg(cn + kone);
-                        float acc = 0.f;
+                    const bool two = ms != 0u;
+                    const int src1 = two ? __ffs(ms) - 1 : src0;
+                    ms &= ms - 1;
+                    const int k0 = (g0 + src0) * GROUP + (int)(__shfl_sync(FULL, key.x, src0) & IDX_MASK);
+                    const int k1 = (g0 + src1) * GROUP + (int)(__shfl_sync(FULL, key.x, src1) & IDX_MASK);
+                    const bool use0 = k0 < K, use1 = two && k1 < K;
+                    const int kk0 = use0 ? k0 : 0, kk1 = use1 ? k1 : 0;
+                    const float cn0 = __ldg(cn + kk0), cn1 = __ldg(cn + kk1);
+                    float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                        for (int v = 0; v < VPL; ++v) {
-                            const int q = lane + 32 * v;
-                            if (q < d4) acc = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc);
+                    for (int v = 0; v < VPL; ++v) {
+                        const int q = lane + 32 * v;
+                        if (q < d4) {
+                            const float4 c0 = __ldg(C4 + (size_t)kk0 * d4 + q), c1 = __ldg(C4 + (size_t)kk1 * d4 + q);
+                            acc0 = dot4(x[v], c0, acc0);
+                            acc1 = dot4(x[v], c1, acc1);
                         }
-                        float s = fmaf(-2.f, warp_sum(acc), cnk);
-                        s = (s == s) ? s : CUDART_INF_F;
-                        if (s < best || (s == best && kone < bidx)) {
-                            best = s;
-                            bidx = kone;
-                        }
+                    }
+#pragma unroll
+                    for (int m = 16; m >= 1; m >>= 1) {   // two warp_sum trees side by side
+                        acc0 += __shfl_xor_sync(FULL, acc0, m);
+                        acc1 += __shfl_xor_sync(FULL, acc1, m);
+                    }
+                    float s0 = fmaf(-2.f, acc0, cn0), s1 = fmaf(-2.f, acc1, cn1);
+                    s0 = (s0 == s0) ? s0 : CUDART_INF_F;
+                    s1 = (s1 == s1) ? s1 : CUDART_INF_F;
+                    n_single += (use0 ? 1 : 0) + (use1 ? 1 : 0);
+                    if (use0 && (s0 < best || (s0 == best && k0 < bidx))) {
+                        best = s0;
+                        bidx = k0;
+                    }
+                    if (use1 && (s1 < best || (s1 == best && k1 < bidx))) {
+                        best = s1;
+                        bidx = k1;
                     }
                 }
             }
+            lanes_differ |= (ms | (m1 & mboth)) != 0u;
             while (ms) {
                 float acc[KC];
                 int myk = -1;
@@ -400,19 +474,21 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                 }
             }
         }
+        if (lanes_differ) {
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            const float ov = __shfl_xor_sync(FULL, best, o);
-            const int oi = __shfl_xor_sync(FULL, bidx, o);
-            if (ov < best || (ov == best && oi < bidx)) {
-                best = ov;
-                bidx = oi;
+            for (int o = 16; o >= 1; o >>= 1) {
+                const float ov = __shfl_xor_sync(FULL, best, o);
+                const int oi = __shfl_xor_sync(FULL, bidx, o);
+                if (ov < best || (ov == best && oi < bidx)) {
+                    best = ov;
+                    bidx = oi;
+                }
             }
         }
         if (lane == 0) assign[row] = (bidx >= 0 && bidx < K) ? bidx : 0;   // a row of NaNs still gets a valid label
     }
     if (counters && lane == 0) {
-        atomicAdd(&counters[0], n_rows);
+        atomicAdd(&counters[4], n_rows);
         atomicAdd(&counters[1], n_single);
         atomicAdd(&counters[2], n_scan);
     }
@@ -478,8 +554,11 @@ int64_t kmeans_tc_chunk_rows(const ep_ctx *ctx, int64_t N, int K) {
     return std::min<int64_t>(rows, ceil_div(N, BM) * BM);
 }
 
+// Candidate keys of one chunk of rows, the chunk's list of undecided rows, and one list length per chunk.
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K) {
-    return (size_t)kmeans_tc_chunk_rows(ctx, N, K) * kmeans_tc_groups(K) * sizeof(uint2);
+    const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
+    return (size_t)chunk * kmeans_tc_groups(K) * sizeof(uint2) + (size_t)chunk * sizeof(int32_t) +
+           (size_t)ceil_div(N, chunk) * sizeof(int);
 }
 
 int kmeans_tc_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *centroids, TcState *st) {
@@ -499,31 +578,38 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
     const int stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / C_STAGE_BYTES);
     const size_t smem = fixed + (size_t)stages * C_STAGE_BYTES;
     EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_tc_screen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
+    const int64_t nchunks = ceil_div(N, chunk);
     uint2 *cand = static_cast<uint2 *>(cand_ws);
+    int32_t *slow_list = reinterpret_cast<int32_t *>(cand + (size_t)chunk * G);
+    int *slow_count = slow_list + chunk;                                // one counter per chunk
+    unsigned long long *counters =
+        ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
     {
         Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
+        EP_CUDA(ctx, cudaMemsetAsync(slow_count, 0, sizeof(int) * (size_t)nchunks, stream));
         centroid_maxima<<<1, 1024, 0, stream>>>(cn, clo, K, cmaxima);
         tm.end(1);
     }
-    const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
     int launches = 0;
-    for (int64_t r0 = 0; r0 < N; r0 += chunk) {
+    for (int64_t r0 = 0, c = 0; r0 < N; r0 += chunk, ++c) {
         const int64_t r1 = std::min(N, r0 + chunk);
         const int grid = (int)std::min<int64_t>(ctx->sm_count, ceil_div(r1 - r0, BM));
         {
             Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
             kmeans_tc_screen<<<grid, TC_THREADS, smem, stream>>>(st.map_x, st.map_c, cn, r0, r1, num_kb, num_nt, stages, G,
-                                                               ~IDX_MASK, cand, ctx->d_status);
+                                                               ~IDX_MASK, d, K, cmaxima, rownorm, cand, assign, slow_list,
+                                                               slow_count + c, counters, ctx->d_status);
             tm.end(1);
         }
         Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
         const int rgrid = (int)std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(r1 - r0, 8));
-        unsigned long long *counters =
-            ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
         if (d <= 128)
-            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cmaxima, rownorm, cand, assign, counters);
+            kmeans_tc_resolve<1><<<rgrid, 256, 0, stream>>>(emb, r0, (int)(r1 - r0), d, K, G, centroids, cn, cmaxima, rownorm, cand, slow_list,
+                                                           slow_count + c, assign, counters);
         else
-            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, r1, d, K, G, centroids, cn, cmaxima, rownorm, cand, assign, counters);
+            kmeans_tc_resolve<2><<<rgrid, 256, 0, stream>>>(emb, r0, (int)(r1 - r0), d, K, G, centroids, cn, cmaxima, rownorm, cand, slow_list,
+                                                           slow_count + c, assign, counters);
         tm.end(1);
         launches += 2;
     }

@@ -97,7 +97,7 @@ def test_tensor_core_path_in_row_chunks(ctx):
     try:
         parts = ctx.kmeans(emb, w.K, 2, init, objective=True)
     finally:
-        ctx.set_kmeans_cand_mb(64)
+        ctx.set_kmeans_cand_mb(1024)
         ctx.set_kmeans_path("auto")
     assert torch.equal(whole.assign, parts.assign) and torch.equal(whole.centroids, parts.centroids)
     ref = oracle.kmeans(emb.cpu().numpy(), w.K, 2, init.cpu().numpy())

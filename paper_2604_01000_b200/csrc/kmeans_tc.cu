@@ -63,6 +63,8 @@ struct TcShared {
 // A row with a single centroid inside the allowance (see screen_allowance) gets assign[r] here; every
 // other row is appended to slow_list (row numbers, any order) and counted in *slow_count, which the caller
 // has zeroed.  counters, when given, receives the number of rows screened in word 0.
+// CN_SMEM: all of cn is first copied behind the barriers in shared memory (the host checks that it fits).
+template <bool CN_SMEM>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
                  const float *__restrict__ cn, int64_t row_begin, int64_t row_end, int num_kb, int num_nt, int stages,
@@ -75,7 +77,10 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     uint8_t *x_smem = smem;                                         // [num_kb][128 rows][128 B]
     uint8_t *c_smem = x_smem + (size_t)num_kb * X_KB_BYTES;         // [stages][256 rows][128 B]
     TcShared *sh = reinterpret_cast<TcShared *>(c_smem + (size_t)stages * C_STAGE_BYTES);
+    float *cn_s = reinterpret_cast<float *>(sh + 1);                // [num_nt * BN] when CN_SMEM
     volatile int *abort_flag = &sh->abort;
+    if (CN_SMEM)
+        for (int i = threadIdx.x; i < num_nt * BN; i += TC_THREADS) cn_s[i] = cn[i];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t num_tiles = (row_end - row_begin + BM - 1) / BM;
@@ -181,13 +186,15 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + half * GROUP;
                 const float *cn_grp = cn + (size_t)nt * BN + half * GROUP;
                 float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
-#pragma unroll
-                for (int c = 0; c < GROUP / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + c * 32, v);
+                // 32 columns at a time; the next 32 are on their way from TMEM while these are ranked
+                auto rank32 = [&](const uint32_t (&v)[32], int c) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
-                        const float4 n4 = __ldg(reinterpret_cast<const float4 *>(cn_grp + c * 32) + q);
+                        float4 n4;
+                        if (CN_SMEM)
+                            n4 = *(reinterpret_cast<const float4 *>(cn_s + nt * BN + half * GROUP + c * 32) + q);
+                        else
+                            n4 = __ldg(reinterpret_cast<const float4 *>(cn_grp + c * 32) + q);
                         const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -200,10 +207,22 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                                 keep_two(a1, a2, key);
                         }
                     }
-                }
-                tc_fence_before();
+                };
+                uint32_t va[32], vb[32];
+                tmem_ld32_issue(taddr, va);
+                tmem_ld_wait(va);
+                tmem_ld32_issue(taddr + 32, vb);
+                rank32(va, 0);
+                tmem_ld_wait(vb);
+                tmem_ld32_issue(taddr + 64, va);
+                rank32(vb, 1);
+                tmem_ld_wait(va);
+                tmem_ld32_issue(taddr + 96, vb);
+                rank32(va, 2);
+                tc_fence_before();                          // every column is in registers: the accumulator is free
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
+                rank32(vb, 3);
                 const float k1 = fminf(a1, b1);
                 const float k2 = fminf(fmaxf(a1, b1), fminf(a2, b2));
                 const int g = nt * 2 + half;
@@ -574,10 +593,22 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
     const int num_kb = (d + KBLK - 1) / KBLK;
     const int num_nt = (K + BN - 1) / BN;
     const int G = num_nt * 2;
-    const size_t fixed = (size_t)num_kb * X_KB_BYTES + sizeof(TcShared) + 1024;
-    const int stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / C_STAGE_BYTES);
+    size_t fixed = (size_t)num_kb * X_KB_BYTES + sizeof(TcShared) + 1024;
+    int stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / C_STAGE_BYTES);
+    // |c|^2 of every centroid in shared memory too, unless that would cost the ring more than one stage
+    const size_t cn_bytes = (size_t)num_nt * BN * sizeof(float);
+    bool cn_smem = false;
+    if (fixed + cn_bytes + 2 * (size_t)C_STAGE_BYTES <= (size_t)ctx->smem_optin) {
+        const int with = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed - cn_bytes) / C_STAGE_BYTES);
+        if (with >= std::min(stages, 3)) {
+            cn_smem = true;
+            stages = with;
+            fixed += cn_bytes;
+        }
+    }
     const size_t smem = fixed + (size_t)stages * C_STAGE_BYTES;
-    EP_CUDA(ctx, cudaFuncSetAttribute(kmeans_tc_screen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    auto screen = cn_smem ? kmeans_tc_screen<true> : kmeans_tc_screen<false>;
+    EP_CUDA(ctx, cudaFuncSetAttribute(screen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
     const int64_t nchunks = ceil_div(N, chunk);
     uint2 *cand = static_cast<uint2 *>(cand_ws);
@@ -597,7 +628,7 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
         const int grid = (int)std::min<int64_t>(ctx->sm_count, ceil_div(r1 - r0, BM));
         {
             Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
-            kmeans_tc_screen<<<grid, TC_THREADS, smem, stream>>>(st.map_x, st.map_c, cn, r0, r1, num_kb, num_nt, stages, G,
+            screen<<<grid, TC_THREADS, smem, stream>>>(st.map_x, st.map_c, cn, r0, r1, num_kb, num_nt, stages, G,
                                                                ~IDX_MASK, d, K, cmaxima, rownorm, cand, assign, slow_list,
                                                                slow_count + c, counters, ctx->d_status);
             tm.end(1);

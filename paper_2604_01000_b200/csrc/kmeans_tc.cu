@@ -176,9 +176,11 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
             const int64_t row = row_begin + tile * BM + quad * 32 + lane;
             float2 nr = make_float2(0.f, 0.f);
-            if (half == 0 && row < row_end) nr = __ldg(rownorm + row);
+            if (row < row_end) nr = __ldg(rownorm + row);
+            const float allow2 = 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
             float run1 = __uint_as_float(KEY_INIT), run2 = run1;   // the row's two smallest keys over this half's groups
             int rung = 0;                                          // group of run1
+            float cut = run1;                                      // scores above it are out of the race
             for (int nt = 0; ok && nt < num_nt; ++nt, ++acc) {
                 const uint32_t buf = acc & 1u, use = (acc >> 1) & 1u;
                 if (!(ok = mbar_wait(&sh->t_full[buf], use, abort_flag))) break;
@@ -187,24 +189,37 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const float *cn_grp = cn + (size_t)nt * BN + half * GROUP;
                 float a1 = __uint_as_float(KEY_INIT), a2 = a1, b1 = a1, b2 = a1;
                 // 32 columns at a time; the next 32 are on their way from TMEM while these are ranked
+                // A score above cut = (smallest key this warp has seen for the row) + twice the allowance can
+                // never be the row's fp32 argmin nor tie with it, and the final threshold is no larger than any
+                // earlier cut: such scores are dropped eight at a time, before they are packed and ranked.
                 auto rank32 = [&](const uint32_t (&v)[32], int c) {
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        float4 n4;
-                        if (CN_SMEM)
-                            n4 = *(reinterpret_cast<const float4 *>(cn_s + nt * BN + half * GROUP + c * 32) + q);
-                        else
-                            n4 = __ldg(reinterpret_cast<const float4 *>(cn_grp + c * 32) + q);
-                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+                    for (int h = 0; h < 4; ++h) {
+                        float s[8];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float s = fmaf(-2.f, __uint_as_float(v[q * 4 + j]), nn[j]);
-                            const float key =
-                                __uint_as_float((__float_as_uint(s) & key_mask) | (uint32_t)(c * 32 + q * 4 + j));
-                            if (j & 1)
-                                keep_two(b1, b2, key);
+                        for (int q = 0; q < 2; ++q) {
+                            float4 n4;
+                            if (CN_SMEM)
+                                n4 = *(reinterpret_cast<const float4 *>(cn_s + nt * BN + half * GROUP + c * 32 + h * 8) + q);
                             else
-                                keep_two(a1, a2, key);
+                                n4 = __ldg(reinterpret_cast<const float4 *>(cn_grp + c * 32 + h * 8) + q);
+                            s[q * 4 + 0] = fmaf(-2.f, __uint_as_float(v[h * 8 + q * 4 + 0]), n4.x);
+                            s[q * 4 + 1] = fmaf(-2.f, __uint_as_float(v[h * 8 + q * 4 + 1]), n4.y);
+                            s[q * 4 + 2] = fmaf(-2.f, __uint_as_float(v[h * 8 + q * 4 + 2]), n4.z);
+                            s[q * 4 + 3] = fmaf(-2.f, __uint_as_float(v[h * 8 + q * 4 + 3]), n4.w);
+                        }
+                        const float m = fmin3(fmin3(s[0], s[1], s[2]), fmin3(s[3], s[4], s[5]), fminf(s[6], s[7]));
+                        if (m <= cut) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float key =
+                                    __uint_as_float((__float_as_uint(s[j]) & key_mask) | (uint32_t)(c * 32 + h * 8 + j));
+                                if (j & 1)
+                                    keep_two(b1, b2, key);
+                                else
+                                    keep_two(a1, a2, key);
+                            }
+                            cut = fminf(cut, fminf(a1, b1) + allow2);
                         }
                     }
                 };
@@ -219,6 +234,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tmem_ld_wait(va);
                 tmem_ld32_issue(taddr + 96, vb);
                 rank32(va, 2);
+                tmem_ld_wait(vb);
                 tc_fence_before();                          // every column is in registers: the accumulator is free
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh->t_empty[buf]);
@@ -246,7 +262,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const float second = fminf(fmaxf(run1, o.x), fminf(run2, o.y));
                 const int glo = o.x < run1 ? __float_as_int(o.z) : rung;
                 const int kone = glo * GROUP + (int)(__float_as_uint(lo) & IDX_MASK);
-                const float thr = lo + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
+                const float thr = lo + allow2;
                 const bool live = row < row_end;
                 // one centroid inside the allowance, every other one outside: it is the fp32 argmin
                 const bool fast = live && second > thr && kone < K;

@@ -122,6 +122,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Smallest of three (one instruction on sm_100).
+__device__ __forceinline__ float fmin3(float a, float b, float c) {
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // Keeps the two smallest keys seen.  A key is a score whose low 7 mantissa bits hold the column's
 // index inside its group, compared as a float, so one min/max pair carries value and index.
 __device__ __forceinline__ void keep_two(float &b1, float &b2, float key) {

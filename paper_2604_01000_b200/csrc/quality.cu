@@ -215,7 +215,39 @@ __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
                 bad |= (live && !in) ? 1u : 0u;
             }
         };
-        if (ne == QT_EDGES) {
+        // The usual vector: a full tile, every index of this thread inside [0, N).  No per-entry range or length
+        // test, and one source label for all four entries unless a row starts among the last three.
+        auto differs = [&](int col, unsigned cur) -> unsigned {
+            if (PACK == 8) return lab_tab[col] != cur ? 1u : 0u;
+            if (PACK == 4)   // cur fills both nibbles: compare the nibble of col in place
+                return ((lab_tab[col >> 1] ^ cur) & (0xFu << ((col << 2) & 4))) != 0u ? 1u : 0u;
+            return (unsigned)__ldg(lab + col) != cur ? 1u : 0u;
+        };
+        auto vec_clean = [&](int q, const int4 &cv) {
+            const int wd = q >> 5, b = q & 31;
+            const unsigned bits = bitmap[wd];
+            const unsigned upto = bits & (0xffffffffu >> (31 - b));
+            const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
+            const unsigned cur = head >= 0 ? (unsigned)headlab[head] : (unsigned)carry;
+            const unsigned rep = PACK == 4 ? 0x11u : 1u;
+            if (((bits >> b) & 0xEu) == 0u) {
+                const unsigned cw = cur * rep;
+                cut += differs(cv.x, cw) + differs(cv.y, cw) + differs(cv.z, cw) + differs(cv.w, cw);
+            } else {
+                const unsigned c1 = ((bits >> (b + 1)) & 1u) ? (unsigned)headlab[q + 1] : cur;
+                const unsigned c2 = ((bits >> (b + 2)) & 1u) ? (unsigned)headlab[q + 2] : c1;
+                const unsigned c3 = ((bits >> (b + 3)) & 1u) ? (unsigned)headlab[q + 3] : c2;
+                cut += differs(cv.x, cur * rep) + differs(cv.y, c1 * rep) + differs(cv.z, c2 * rep) + differs(cv.w, c3 * rep);
+            }
+        };
+        unsigned top = 0u;                                   // largest index of this thread, as unsigned
+#pragma unroll
+        for (int i = 0; i < QT_VEC; ++i)
+            top = max(max(max(top, (unsigned)c[i].x), max((unsigned)c[i].y, (unsigned)c[i].z)), (unsigned)c[i].w);
+        if (ne == QT_EDGES && top < (unsigned)N) {
+#pragma unroll
+            for (int i = 0; i < QT_VEC; ++i) vec_clean((i * QT_THREADS + tid) * 4, c[i]);
+        } else if (ne == QT_EDGES) {
 #pragma unroll
             for (int i = 0; i < QT_VEC; ++i) vec((i * QT_THREADS + tid) * 4, c[i], true);
         } else {

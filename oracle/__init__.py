@@ -10,6 +10,7 @@ from .ep_oracle import (  # noqa: F401
     assign_step,
     partition_quality,
     reorder,
+    graph_bandwidth,
     num_threads,
     set_num_threads,
 )

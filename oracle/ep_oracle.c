@@ -5,6 +5,7 @@
  *   - Lloyd K-Means over dense node embeddings  (Algorithm 3, line 1: P <- KMeans(E, k))
  *   - edge cut and per-partition loads           (Section 2.1.1, Eq. 1 and Eq. 2)
  *   - the partition-ordered vertex permutation   (Section 4.5.1, "Adapting EmbedPart for Reordering")
+ *   - the average graph bandwidth of a numbering (Section 4.5.1, Eq. 3, Eq. 4 and Eq. 5)
  *
  * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call
  * this file.  It shares no code, header, table or helper with the CUDA library
@@ -209,4 +210,36 @@ int oracle_reorder(const int32_t *assign, int64_t N, int32_t K,
     }
     free(next);
     return 0;
+}
+
+/*
+ * Graph bandwidth of a vertex numbering (Section 4.5.1).  pi[v] is the new id of
+ * vertex v, a bijection of [0, N).
+ *
+ *   gap of an entry (v -> u)      xi = |pi[v] - pi[u]|                       (Eq. 3)
+ *   vertex bandwidth              beta_v = max of xi over the entries of row v (Eq. 4)
+ *   average graph bandwidth       (1/N) sum over v of beta_v                   (Eq. 5)
+ *
+ * The neighbours n(v) are the stored entries of row v; a vertex without entries
+ * has an empty maximum, read as 0 (it touches no other vertex); a self-loop has
+ * gap 0.  The sum is returned as an exact integer, the caller divides by N;
+ * vertex_bandwidth (may be NULL) receives beta_v.
+ */
+void oracle_graph_bandwidth(const int64_t *rowptr, const int32_t *colidx, const int32_t *pi,
+                            int64_t N, uint64_t *bandwidth_sum, int32_t *vertex_bandwidth)
+{
+    int64_t total = 0;
+    int64_t v;
+#pragma omp parallel for schedule(dynamic, 4096) reduction(+ : total)
+    for (v = 0; v < N; ++v) {
+        int64_t beta = 0;
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            int64_t xi = (int64_t)pi[v] - (int64_t)pi[colidx[e]];
+            if (xi < 0) xi = -xi;
+            if (xi > beta) beta = xi;
+        }
+        if (vertex_bandwidth) vertex_bandwidth[v] = (int32_t)beta;
+        total += beta;
+    }
+    *bandwidth_sum = (uint64_t)total;
 }

@@ -44,6 +44,8 @@ def _load():
         lib.oracle_partition_quality.restype = None
         lib.oracle_reorder.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, p]
         lib.oracle_reorder.restype = ctypes.c_int
+        lib.oracle_graph_bandwidth.argtypes = [p, p, p, ctypes.c_int64, p, p]
+        lib.oracle_graph_bandwidth.restype = None
         _lib = lib
     return _lib
 
@@ -153,3 +155,32 @@ def reorder(assign, K: int):
     if rc != 0:
         raise MemoryError("oracle_reorder")
     return perm, inv
+
+
+class BandwidthResult(NamedTuple):
+    bandwidth_sum: int              # sum over v of beta_v; the average graph bandwidth is bandwidth_sum / N
+    vertex_bandwidth: np.ndarray    # int32 [N]
+
+    @property
+    def average(self) -> float:
+        return self.bandwidth_sum / max(1, self.vertex_bandwidth.shape[0])
+
+
+def graph_bandwidth(rowptr, colidx, pi) -> BandwidthResult:
+    """Vertex bandwidths and their sum for the numbering pi (pi[v] = new id of v)."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    pi = np.ascontiguousarray(pi, dtype=np.int32)
+    N = rowptr.shape[0] - 1
+    if pi.shape != (N,):
+        raise ValueError("pi must have one entry per vertex")
+    if rowptr[0] != 0 or rowptr[-1] != colidx.shape[0] or np.any(np.diff(rowptr) < 0):
+        raise ValueError("rowptr is not a CSR row pointer for colidx")
+    if colidx.size and (colidx.min() < 0 or colidx.max() >= N):
+        raise ValueError("colidx value outside [0, N)")
+    if N and not np.array_equal(np.sort(pi), np.arange(N, dtype=np.int32)):
+        raise ValueError("pi is not a bijection of [0, N)")
+    total = ctypes.c_uint64(0)
+    vb = np.empty(N, np.int32)
+    _load().oracle_graph_bandwidth(_ptr(rowptr), _ptr(colidx), _ptr(pi), N, ctypes.addressof(total), _ptr(vb))
+    return BandwidthResult(int(total.value), vb)

@@ -140,3 +140,84 @@ def test_reorder_structure_on_a_larger_case():
         seg = perm[starts[p]: starts[p] + counts[p]]
         assert np.all(assign[seg] == p)
     assert counts[17] == 0
+
+
+# ---------------------------------------------------------------------------------- graph bandwidth
+def _bandwidth_cases():
+    with open(os.path.join(GOLDEN, "graph_bandwidth_hand_cases.json")) as f:
+        return json.load(f)["cases"]
+
+
+@pytest.mark.parametrize("case", _bandwidth_cases(), ids=lambda c: c["name"][:40])
+def test_bandwidth_hand_cases(case):
+    b = oracle.graph_bandwidth(case["rowptr"], case["colidx"], case["pi"])
+    assert b.vertex_bandwidth.tolist() == case["vertex_bandwidth"]
+    assert b.bandwidth_sum == case["bandwidth_sum"] == sum(case["vertex_bandwidth"])
+    assert b.average == case["bandwidth_sum"] / len(case["pi"])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_bandwidth_brute_force_dense_adjacency(seed):
+    """Eq. 3-5 written as a double loop over a dense adjacency matrix, any numbering."""
+    rng = np.random.default_rng(100 + seed)
+    N = int(rng.integers(2, 11))
+    A, rowptr, colidx = _random_csr(rng, N, 0.35, symmetric=bool(seed % 2), loops=True)
+    pi = rng.permutation(N).astype(np.int32)
+    beta = [max([abs(int(pi[v]) - int(pi[u])) for u in range(N) if A[v, u]], default=0) for v in range(N)]
+    b = oracle.graph_bandwidth(rowptr, colidx, pi)
+    assert b.vertex_bandwidth.tolist() == beta and b.bandwidth_sum == sum(beta)
+
+
+def test_bandwidth_closed_forms_and_invariances():
+    rng = np.random.default_rng(7)
+    # complete graph, identity numbering: the farthest neighbour of v is vertex 0 or vertex n-1
+    n = 9
+    A = ~np.eye(n, dtype=bool)
+    rowptr = np.arange(n + 1, dtype=np.int64) * (n - 1)
+    colidx = np.nonzero(A)[1].astype(np.int32)
+    b = oracle.graph_bandwidth(rowptr, colidx, np.arange(n))
+    assert b.vertex_bandwidth.tolist() == [max(v, n - 1 - v) for v in range(n)]
+    # any graph, any numbering
+    N = 200
+    A, rowptr, colidx = _random_csr(rng, N, 0.03, symmetric=True)
+    pi = rng.permutation(N).astype(np.int32)
+    b = oracle.graph_bandwidth(rowptr, colidx, pi)
+    deg = np.diff(rowptr)
+    assert ((b.vertex_bandwidth >= 0) & (b.vertex_bandwidth <= N - 1)).all()
+    assert (b.vertex_bandwidth[deg == 0] == 0).all() and (b.vertex_bandwidth[deg > 0] >= 1).all()
+    # mirror image of the numbering: every gap is unchanged
+    assert np.array_equal(oracle.graph_bandwidth(rowptr, colidx, N - 1 - pi).vertex_bandwidth, b.vertex_bandwidth)
+    # renaming the vertices by pi and numbering the renamed graph by the identity is the same layout
+    A2 = np.zeros_like(A)
+    A2[np.ix_(pi, pi)] = A
+    rowptr2 = np.concatenate([[0], np.cumsum(A2.sum(1))]).astype(np.int64)
+    colidx2 = np.nonzero(A2)[1].astype(np.int32)
+    b2 = oracle.graph_bandwidth(rowptr2, colidx2, np.arange(N))
+    assert np.array_equal(b2.vertex_bandwidth[pi], b.vertex_bandwidth) and b2.bandwidth_sum == b.bandwidth_sum
+    # a symmetric graph: the largest vertex bandwidth is attained at both ends of the widest edge
+    assert (b.vertex_bandwidth == b.vertex_bandwidth.max()).sum() >= 2
+
+
+def test_bandwidth_of_partition_ordered_numbering_beats_a_random_one():
+    """Statistical sanity (Section 4.5.1): numbering a planted-partition graph by its blocks keeps
+    neighbours closer than a random numbering does."""
+    rng = np.random.default_rng(3)
+    N, K = 400, 8
+    block = rng.integers(0, K, size=N)
+    P = np.where(block[:, None] == block[None, :], 0.10, 0.002)
+    A = rng.random((N, N)) < P
+    A = A | A.T
+    np.fill_diagonal(A, False)
+    rowptr = np.concatenate([[0], np.cumsum(A.sum(1))]).astype(np.int64)
+    colidx = np.nonzero(A)[1].astype(np.int32)
+    _, inv = oracle.reorder(block.astype(np.int32), K)
+    grouped = oracle.graph_bandwidth(rowptr, colidx, inv).average
+    shuffled = oracle.graph_bandwidth(rowptr, colidx, rng.permutation(N)).average
+    assert grouped < shuffled
+
+
+def test_bandwidth_rejects_bad_input():
+    with pytest.raises(ValueError):
+        oracle.graph_bandwidth([0, 1, 2], [1, 0], [0, 0])            # not a bijection
+    with pytest.raises(ValueError):
+        oracle.graph_bandwidth([0, 1, 2], [1, 5], [0, 1])            # neighbour outside [0, N)

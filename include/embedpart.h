@@ -70,7 +70,8 @@ enum {
     EP_TIMER_QUALITY_PREP = 3,   /* label repacking, partition loads, tile start rows */
     EP_TIMER_REORDER = 4,        /* all kernels of ep_reorder */
     EP_TIMER_KMEANS_RESOLVE = 5, /* tensor-core path: the fp32 kernel that decides the labels */
-    EP_TIMER_COUNT = 6
+    EP_TIMER_GRAPH_BANDWIDTH = 6, /* all kernels of ep_graph_bandwidth */
+    EP_TIMER_COUNT = 7
 };
 
 typedef struct ep_ctx ep_ctx; /* opaque: device id, device properties, device status word, options */
@@ -172,6 +173,35 @@ int ep_partition_quality(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int6
 size_t ep_reorder_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t K);
 int ep_reorder(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, int32_t *perm, int32_t *inv_perm,
                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_graph_bandwidth -- average graph bandwidth of a vertex numbering (Section 4.5.1, Eq. 3-5).
+ *
+ * pi[v] is the new id of vertex v (the inv_perm of ep_reorder).  For every stored entry (v -> u)
+ * the gap is |pi[v] - pi[u]| (Eq. 3); the vertex bandwidth beta_v is the largest gap over the
+ * entries of row v (Eq. 4), 0 for a row without entries; the average graph bandwidth is
+ * bandwidth_sum / N (Eq. 5), the division left to the caller so that the result stays an exact
+ * integer.
+ *
+ *   rowptr   [dev] N+1 row offsets, int32 or int64 as rowptr_is_int64 says, rowptr[0] = 0,
+ *            non-decreasing, rowptr[N] = nnz
+ *   colidx   [dev] nnz int32 column ids in [0, N), 16-byte aligned
+ *   pi       [dev] N int32 new ids in [0, 2^31); normally a bijection of [0, N), not checked
+ *   N, nnz   1 <= N < 2^31, 0 <= nnz < 2^62
+ *   bandwidth_sum    [dev] out, 1 uint64: sum of beta_v
+ *   vertex_bandwidth [dev] out or NULL, N int32: beta_v
+ * A column id outside [0, N) or a row pointer that steps backwards raises EP_ERR_BAD_INDEX in the
+ * device status word; the entry is skipped.  Integer maxima and sums only, so the result does not
+ * depend on scheduling.  The _host variant takes host pointers and an arena like the others.
+ */
+size_t ep_graph_bandwidth_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz);
+int ep_graph_bandwidth(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                       int64_t nnz, const int32_t *pi, int64_t N, uint64_t *bandwidth_sum,
+                       int32_t *vertex_bandwidth, void *workspace, size_t workspace_bytes, void *cuda_stream);
+size_t ep_graph_bandwidth_host_arena_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t rowptr_is_int64);
+int ep_graph_bandwidth_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                            int64_t nnz, const int32_t *pi, int64_t N, uint64_t *bandwidth_sum,
+                            int32_t *vertex_bandwidth, void *arena, size_t arena_bytes, void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
  * Host-buffer variants.  Same operations and the same kernels; inputs and outputs are [host]

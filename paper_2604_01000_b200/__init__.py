@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     ep_partition_quality,
     ep_reorder,
     ep_reorder_static,
+    ep_graph_bandwidth,
     library_path,
     load_library,
     EXPORTED_SYMBOLS,

@@ -17,6 +17,8 @@ EXPORTED_SYMBOLS = (
     "ep_partition_quality", "ep_reorder_workspace_bytes", "ep_reorder", "ep_profile_read", "ep_launch_count",
     "ep_kmeans_host_arena_bytes", "ep_kmeans_host", "ep_quality_host_arena_bytes", "ep_partition_quality_host",
     "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static", "ep_debug_counters",
+    "ep_graph_bandwidth_workspace_bytes", "ep_graph_bandwidth", "ep_graph_bandwidth_host_arena_bytes",
+    "ep_graph_bandwidth_host",
 )
 
 EP_OK = 0
@@ -24,9 +26,9 @@ EP_OPT_KMEANS_PATH = 1
 EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
 EP_OPT_KMEANS_CAND_MB = 4
-TIMER_COUNT = 6
+TIMER_COUNT = 7
 TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
-          "kmeans_resolve": 5}
+          "kmeans_resolve": 5, "graph_bandwidth": 6}
 KMEANS_PATHS = {"auto": 0, "simt": 1, "tensor": 2}
 
 
@@ -103,6 +105,14 @@ def load_library() -> ctypes.CDLL:
             lib.ep_reorder_host.restype = ctypes.c_int
             lib.ep_reorder_static.argtypes = [vp, i64, i32, vp, vp, vp, vp]
             lib.ep_reorder_static.restype = ctypes.c_int
+            lib.ep_graph_bandwidth_workspace_bytes.argtypes = [vp, i64, i64]
+            lib.ep_graph_bandwidth_workspace_bytes.restype = sz
+            lib.ep_graph_bandwidth.argtypes = [vp, vp, i32, vp, i64, vp, i64, vp, vp, vp, sz, vp]
+            lib.ep_graph_bandwidth.restype = ctypes.c_int
+            lib.ep_graph_bandwidth_host_arena_bytes.argtypes = [vp, i64, i64, i32]
+            lib.ep_graph_bandwidth_host_arena_bytes.restype = sz
+            lib.ep_graph_bandwidth_host.argtypes = [vp, vp, i32, vp, i64, vp, i64, vp, vp, vp, sz, vp]
+            lib.ep_graph_bandwidth_host.restype = ctypes.c_int
             _lib = lib
     return _lib
 
@@ -273,6 +283,29 @@ class Context:
             self._raise(rc)
         return ReorderResult(perm, inv)
 
+    def graph_bandwidth(self, rowptr, colidx, pi, per_vertex: bool = True):
+        """Sum of the vertex bandwidths of the numbering pi (pi[v] = new id of v) and, if asked, each of them."""
+        if rowptr.dtype not in (torch.int32, torch.int64):
+            raise ValueError("rowptr must be int32 or int64")
+        rowptr = _check_cuda(rowptr, rowptr.dtype, "rowptr", self.device)
+        colidx = _check_cuda(colidx, torch.int32, "colidx", self.device)
+        pi = _check_cuda(pi, torch.int32, "pi", self.device)
+        N, nnz = pi.numel(), colidx.numel()
+        if rowptr.numel() != N + 1:
+            raise ValueError("rowptr must have N + 1 entries")
+        need = self._lib.ep_graph_bandwidth_workspace_bytes(self._h, N, nnz)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} nnz={nnz}")
+        ws = self.workspace(need)
+        total = torch.empty(1, dtype=torch.int64, device=self.device)
+        vb = torch.empty(N, dtype=torch.int32, device=self.device) if per_vertex else None
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_graph_bandwidth(self._h, _dev_ptr(rowptr), int(rowptr.dtype == torch.int64),
+                                              _dev_ptr(colidx), nnz, _dev_ptr(pi), N, _dev_ptr(total), _dev_ptr(vb),
+                                              _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return BandwidthResult(total, vb)
 
     # -- host-buffer calls (inputs and outputs are CPU tensors; copies are part of the call) -----
     def _host(self, t, dtype, name):
@@ -323,6 +356,27 @@ class Context:
             self._raise(rc)
         return out
 
+    def graph_bandwidth_host(self, rowptr, colidx, pi, per_vertex: bool = True, out=None):
+        rowptr = self._host(rowptr, rowptr.dtype, "rowptr")
+        colidx = self._host(colidx, torch.int32, "colidx")
+        pi = self._host(pi, torch.int32, "pi")
+        N, nnz = pi.numel(), colidx.numel()
+        is64 = int(rowptr.dtype == torch.int64)
+        need = self._lib.ep_graph_bandwidth_host_arena_bytes(self._h, N, nnz, is64)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} nnz={nnz}")
+        ws = self.workspace(need)
+        if out is None:
+            out = BandwidthResult(torch.empty(1, dtype=torch.int64).pin_memory(),
+                                  torch.empty(N, dtype=torch.int32).pin_memory() if per_vertex else None)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_graph_bandwidth_host(self._h, _dev_ptr(rowptr), is64, _dev_ptr(colidx), nnz, _dev_ptr(pi),
+                                                   N, _dev_ptr(out.bandwidth_sum), _dev_ptr(out.vertex_bandwidth),
+                                                   _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
     def reorder_host(self, assign, K: int, inverse: bool = True, out=None):
         assign = self._host(assign, torch.int32, "assign")
         N = assign.numel()
@@ -358,6 +412,11 @@ class ReorderResult(NamedTuple):
     inv_perm: Optional[torch.Tensor]     # int32 [N]: inv_perm[old id] = new id
 
 
+class BandwidthResult(NamedTuple):
+    bandwidth_sum: torch.Tensor               # int64 [1]: sum of the vertex bandwidths (divide by N for the average)
+    vertex_bandwidth: Optional[torch.Tensor]  # int32 [N]
+
+
 _default: dict[int, Context] = {}
 
 
@@ -381,6 +440,11 @@ def ep_partition_quality(rowptr, colidx, assign, K) -> QualityResult:
 def ep_reorder(assign, K, inverse=True) -> ReorderResult:
     """Partition-ordered permutation (and its inverse)."""
     return default_context(assign.device.index).reorder(assign, K, inverse)
+
+
+def ep_graph_bandwidth(rowptr, colidx, pi, per_vertex=True) -> BandwidthResult:
+    """Vertex bandwidths of the numbering pi over the CSR graph and their sum."""
+    return default_context(pi.device.index).graph_bandwidth(rowptr, colidx, pi, per_vertex)
 
 
 REORDER_STATIC_MAX_N = 1 << 22

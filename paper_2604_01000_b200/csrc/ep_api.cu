@@ -262,6 +262,81 @@ int ep_partition_quality(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int6
                        reinterpret_cast<long long *>(part_edges), workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---------------------------------------------------------------------------------------------- graph bandwidth
+static bool bandwidth_shape_ok(int64_t N, int64_t nnz) {
+    return N >= 1 && N < (int64_t(1) << 31) && nnz >= 0 && nnz < (int64_t(1) << 62);
+}
+
+size_t ep_graph_bandwidth_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz) {
+    if (!ctx || !bandwidth_shape_ok(N, nnz)) return 0;
+    return bandwidth_workspace_bytes(N, nnz);
+}
+
+int ep_graph_bandwidth(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx, int64_t nnz,
+                       const int32_t *pi, int64_t N, uint64_t *bandwidth_sum, int32_t *vertex_bandwidth,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!bandwidth_shape_ok(N, nnz))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld", (long long)N, (long long)nnz);
+    if (!rowptr || (!colidx && nnz > 0) || !pi || !bandwidth_sum) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!rowptr_is_int64 && nnz >= (int64_t(1) << 31))
+        return fail(ctx, EP_ERR_INVALID_ARG, "nnz needs a 64-bit row pointer");
+    if (!aligned(rowptr, rowptr_is_int64 ? 8 : 4) || !aligned(colidx, 16) || !aligned(pi, 4) ||
+        !aligned(bandwidth_sum, 8) || (vertex_bandwidth && !aligned(vertex_bandwidth, 4)))
+        return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    const size_t need = bandwidth_workspace_bytes(N, nnz);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "graph bandwidth workspace: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    return bandwidth_run(ctx, rowptr, rowptr_is_int64 != 0, colidx, nnz, pi, N,
+                         reinterpret_cast<unsigned long long *>(bandwidth_sum), vertex_bandwidth, workspace,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t ep_graph_bandwidth_host_arena_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz, int32_t rowptr_is_int64) {
+    const size_t ws = ep_graph_bandwidth_workspace_bytes(ctx, N, nnz);
+    if (ws == 0) return 0;
+    Arena a(nullptr);
+    a.take<char>((size_t)(N + 1) * (rowptr_is_int64 ? 8 : 4));
+    a.take<int32_t>(nnz);
+    a.take<int32_t>(N);
+    a.take<int32_t>(N);
+    a.take<uint64_t>(1);
+    return a.used + ws;
+}
+
+int ep_graph_bandwidth_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
+                            int64_t nnz, const int32_t *pi, int64_t N, uint64_t *bandwidth_sum,
+                            int32_t *vertex_bandwidth, void *arena, size_t arena_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!rowptr || (!colidx && nnz > 0) || !pi || !bandwidth_sum) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    const size_t need = ep_graph_bandwidth_host_arena_bytes(ctx, N, nnz, rowptr_is_int64);
+    if (need == 0)
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld", (long long)N, (long long)nnz);
+    if (!arena || !aligned(arena, 256) || arena_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "graph bandwidth host arena: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Arena a(arena);
+    const size_t rp_bytes = (size_t)(N + 1) * (rowptr_is_int64 ? 8 : 4);
+    char *d_rp = a.take<char>(rp_bytes);
+    int32_t *d_ci = a.take<int32_t>(nnz);
+    int32_t *d_pi = a.take<int32_t>(N);
+    int32_t *d_vb = a.take<int32_t>(N);
+    uint64_t *d_sum = a.take<uint64_t>(1);
+    void *ws = a.base + a.used;
+    EP_CUDA(ctx, cudaMemcpyAsync(d_rp, rowptr, rp_bytes, cudaMemcpyHostToDevice, st));
+    if (nnz > 0) EP_CUDA(ctx, cudaMemcpyAsync(d_ci, colidx, sizeof(int32_t) * nnz, cudaMemcpyHostToDevice, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(d_pi, pi, sizeof(int32_t) * N, cudaMemcpyHostToDevice, st));
+    int rc = ep_graph_bandwidth(ctx, d_rp, rowptr_is_int64, d_ci, nnz, d_pi, N, d_sum, vertex_bandwidth ? d_vb : nullptr,
+                                ws, arena_bytes - a.used, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(bandwidth_sum, d_sum, sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    if (vertex_bandwidth)
+        EP_CUDA(ctx, cudaMemcpyAsync(vertex_bandwidth, d_vb, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    return EP_OK;
+}
+
 // ---------------------------------------------------------------------------------------------- reorder
 static bool reorder_shape_ok(int64_t N, int32_t K) {
     return N >= 1 && N < (int64_t(1) << 31) && K >= 1 && K <= (1 << 24);

@@ -139,6 +139,12 @@ int quality_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *c
                 const int32_t *assign, int64_t N, int K, unsigned long long *edge_cut, long long *part_vertices,
                 long long *part_edges, void *workspace, cudaStream_t stream);
 
+// ---- graph bandwidth (bandwidth.cu) -------------------------------------------------------------
+size_t bandwidth_workspace_bytes(int64_t N, int64_t nnz);
+int bandwidth_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *colidx, int64_t nnz,
+                  const int32_t *pi, int64_t N, unsigned long long *total, int32_t *vertex_bandwidth, void *workspace,
+                  cudaStream_t stream);
+
 }  // namespace ep
 
 // ---- device helpers -------------------------------------------------------------------------------

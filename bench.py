@@ -332,8 +332,9 @@ def main():
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     start.record()
+    last = None
     for _ in range(args.steps):
-        step_device(ctx, w, x)
+        last = step_device(ctx, w, x)
     stop.record()
     barrier()
     clocks = sampler.stop()
@@ -413,6 +414,30 @@ def main():
     roofline["ms_per_launch"] = dominant["ms_per_launch"]
     roofline["ms_per_pass"] = dominant["ms_per_pass"]
 
+    # ---- outside the step: the average graph bandwidth (Eq. 3-5) of the numbering the step produced ------
+    extras = {}
+    if last is not None and last[3].inv_perm is not None:
+        reps = 3
+        ctx.graph_bandwidth(x["rowptr"], x["colidx"], last[3].inv_perm, per_vertex=False)
+        torch.cuda.synchronize()
+        ctx.profile_read("graph_bandwidth", 0)
+        ctx.set_profile(True)
+        for _ in range(reps):
+            bw = ctx.graph_bandwidth(x["rowptr"], x["colidx"], last[3].inv_perm, per_vertex=False)
+        torch.cuda.synchronize()
+        ctx.set_profile(False)
+        tot, n = ctx.profile_read("graph_bandwidth", 0)
+        ctx.check()
+        if n:
+            by = 4 * nnz + rp_bytes * (w.N + 1) + 8 * w.N          # column ids, row pointer, pi read + beta written
+            gbs = by * reps / (tot * 1e-3) / 1e9
+            extras["graph_bandwidth"] = {
+                "ms_per_pass": tot / reps, "rate": nnz * reps / (tot * 1e-3), "unit": "edges/s",
+                "average_graph_bandwidth": int(bw.bandwidth_sum.item()) / w.N,
+                "numbering": f"clusters of the K={w.reorder_K or w.K} run, in order",
+                "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
+                             "traffic": None, "peak_source": peaks["_source"]}}
+
     # ---- end to end: the same pass through the host-buffer C ABI (uploads and downloads timed) ---------
     e2e = None
     if not args.no_e2e:
@@ -451,7 +476,7 @@ def main():
                        "parallelism": "replicas only" if world > 1 else "1 GPU", "kmeans_path": args.kmeans_path},
             "edge_cut_edges_per_s": passes.get("edge_cut", {}).get("rate"),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-            "passes": passes,
+            "passes": passes, "extras": extras,
             "tensor_path_counters": {"rows_screened": counters[0], "large_K_single_evals": counters[1],
                                      "large_K_group_scans": counters[2], "small_K_rows_left_to_fp32_kernel": counters[3],
                                      "large_K_rows_left_to_fp32_kernel": counters[4]},

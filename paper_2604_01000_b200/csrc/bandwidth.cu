@@ -16,9 +16,9 @@
 namespace {
 
 constexpr int BW_THREADS = 256;
-constexpr int BW_VEC = 8;                                   // 16-byte loads per thread per tile
-constexpr int BW_EDGES = BW_THREADS * BW_VEC * 4;           // 8192 entries per tile
-constexpr int BW_WORDS = BW_EDGES / 32;                     // 256 bitmap words, one per thread
+constexpr int BW_VEC = 4;                                   // 16-byte loads per thread per tile
+constexpr int BW_EDGES = BW_THREADS * BW_VEC * 4;           // 4096 entries per tile: 33 KB of shared memory, 5 blocks per SM
+constexpr int BW_WORDS = BW_EDGES / 32;                     // 128 bitmap words, one per thread of the first four warps
 constexpr unsigned FULL = 0xffffffffu;
 
 // tile_row[t] = last row r in [0, N) whose first entry is at or before t * BW_EDGES; tile_row[ntiles] = N-1.
@@ -51,7 +51,7 @@ __global__ void bandwidth_check_rows(const RowT *__restrict__ rowptr, int64_t N,
 }
 
 template <typename RowT>
-__global__ void __launch_bounds__(BW_THREADS, 3)
+__global__ void __launch_bounds__(BW_THREADS, 5)
     vertex_bandwidth_tiles(const RowT *__restrict__ rowptr, const int32_t *__restrict__ colidx, int64_t nnz,
                            const int32_t *__restrict__ pi, int64_t N, const int32_t *__restrict__ tile_row,
                            int64_t ntiles, int32_t *vb, int *status) {
@@ -81,8 +81,8 @@ __global__ void __launch_bounds__(BW_THREADS, 3)
             }
         }
         __syncthreads();                                    // previous tile fully written back
-        bitmap[tid] = 0u;
-        for (int i = tid; i <= BW_EDGES; i += BW_THREADS) segmax[i] = 0;
+        if (tid < BW_WORDS) bitmap[tid] = 0u;
+        if (tid == 0) segmax[0] = 0;
         __syncthreads();
         const int64_t r_lo = tile_row[tile], r_hi = tile_row[tile + 1];
         const int32_t carry_pi = pi[r_lo];
@@ -92,11 +92,12 @@ __global__ void __launch_bounds__(BW_THREADS, 3)
             if (e > s && h >= 0 && h < ne) {
                 atomicOr(&bitmap[h >> 5], 1u << (h & 31));
                 headpi[h] = pi[r];
+                segmax[h + 1] = 0;                          // only the slots of row starts are ever used
             }
         }
         __syncthreads();
         {   // lasthead[w] = position of the last set bit in words < w, or -1
-            const unsigned wbits = bitmap[tid];
+            const unsigned wbits = tid < BW_WORDS ? bitmap[tid] : 0u;
             const int mine = wbits ? tid * 32 + 31 - __clz(wbits) : -1;
             int inc = mine;
 #pragma unroll
@@ -109,13 +110,21 @@ __global__ void __launch_bounds__(BW_THREADS, 3)
             if (lane == 0) excl = -1;
             __syncthreads();
             for (int w = 0; w < warp; ++w) excl = max(excl, warp_max[w]);
-            lasthead[tid] = excl;
+            if (tid < BW_WORDS) lasthead[tid] = excl;
         }
         __syncthreads();
         unsigned bad = 0;
+        unsigned top = 0u;                                   // largest column id of this thread, as unsigned
+#pragma unroll
+        for (int i = 0; i < BW_VEC; ++i)
+            top = max(max(max(top, (unsigned)c[i].x), max((unsigned)c[i].y, (unsigned)c[i].z)), (unsigned)c[i].w);
+        // every lane's ids in range and the tile full: the warp may skip the per-entry range and length tests
+        const bool clean = __all_sync(FULL, ne == BW_EDGES && top < (unsigned)N);
+        // first every vector's gathers and maxima (nothing between them that would keep the loads apart) ...
+        int segs[BW_VEC], maxs[BW_VEC];
 #pragma unroll
         for (int i = 0; i < BW_VEC; ++i) {
-            const int q = (i * BW_THREADS + tid) * 4;       // the whole warp takes every vector: match_any below
+            const int q = (i * BW_THREADS + tid) * 4;
             const int wd = q >> 5, b = q & 31;
             const unsigned bits = bitmap[wd];
             const unsigned upto = bits & (0xffffffffu >> (31 - b));
@@ -123,26 +132,43 @@ __global__ void __launch_bounds__(BW_THREADS, 3)
             int32_t from = seg >= 0 ? headpi[seg] : carry_pi;
             int m = 0;
             const int cols[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+            if (clean && ((bits >> b) & 0xEu) == 0u) {      // four entries of one row
+                m = max(max(abs(from - __ldg(pi + cols[0])), abs(from - __ldg(pi + cols[1]))),
+                        max(abs(from - __ldg(pi + cols[2])), abs(from - __ldg(pi + cols[3]))));
+            } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (j > 0 && ((bits >> (b + j)) & 1u)) {    // a row starts inside the vector: close the segment
-                    if (m > 0) atomicMax(&segmax[seg + 1], m);
-                    seg = q + j;
-                    from = headpi[seg];
-                    m = 0;
+                for (int j = 0; j < 4; ++j) {
+                    if (j > 0 && ((bits >> (b + j)) & 1u)) {    // a row starts inside the vector: close the segment
+                        if (m > 0) atomicMax(&segmax[seg + 1], m);
+                        seg = q + j;
+                        from = headpi[seg];
+                        m = 0;
+                    }
+                    const bool live = q + j < ne;
+                    const int col = cols[j];
+                    const bool in = (unsigned)col < (unsigned)N;
+                    const int32_t to = __ldg(pi + (in ? col : 0));   // an index outside [0, N) is reported, never followed
+                    const int gap = abs(from - to);
+                    m = (live && in) ? max(m, gap) : m;
+                    bad |= (live && !in) ? 1u : 0u;
                 }
-                const bool live = q + j < ne;
-                const int col = cols[j];
-                const bool in = (unsigned)col < (unsigned)N;
-                const int32_t to = __ldg(pi + (in ? col : 0));   // an index outside [0, N) is reported, never followed
-                const int gap = abs(from - to);
-                m = (live && in) ? max(m, gap) : m;
-                bad |= (live && !in) ? 1u : 0u;
             }
-            if (q >= ne) seg = -2;                           // nothing of this vector is in the tile
-            const unsigned peers = __match_any_sync(FULL, seg);
-            const int best = (int)__reduce_max_sync(peers, (unsigned)m);
-            if (seg >= -1 && best > 0 && lane == __ffs(peers) - 1) atomicMax(&segmax[seg + 1], best);
+            segs[i] = q >= ne ? -2 : seg;                    // -2: nothing of this vector is in the tile
+            maxs[i] = m;
+        }
+        // ... then, vector by vector (the whole warp takes each), lanes that end in the same segment combine and
+        // one of them issues the shared-memory atomic
+#pragma unroll
+        for (int i = 0; i < BW_VEC; ++i) {
+            const int seg = segs[i], m = maxs[i];
+            if (__all_sync(FULL, seg == __shfl_sync(FULL, seg, 0))) {
+                const int best = (int)__reduce_max_sync(FULL, (unsigned)m);
+                if (lane == 0 && seg >= -1 && best > 0) atomicMax(&segmax[seg + 1], best);
+            } else {
+                const unsigned peers = __match_any_sync(FULL, seg);
+                const int best = (int)__reduce_max_sync(peers, (unsigned)m);
+                if (seg >= -1 && best > 0 && lane == __ffs(peers) - 1) atomicMax(&segmax[seg + 1], best);
+            }
         }
         if (bad) ep_raise(status, EP_ERR_BAD_INDEX);
         __syncthreads();
@@ -206,7 +232,7 @@ static int bandwidth_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *coli
     int kernels = 2;
     if (ntiles > 0) {
         bandwidth_tile_rows<RowT><<<(unsigned)ceil_div(ntiles + 1, 256), 256, 0, stream>>>(rowptr, N, ntiles, b.tile_row);
-        const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 3);
+        const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 5);
         const size_t dyn = sizeof(int) * (2 * (size_t)BW_EDGES + 1);
         EP_CUDA(ctx, cudaFuncSetAttribute(vertex_bandwidth_tiles<RowT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
         vertex_bandwidth_tiles<RowT><<<grid, BW_THREADS, dyn, stream>>>(rowptr, colidx, nnz, pi, N, b.tile_row, ntiles, vb,

@@ -79,7 +79,7 @@ def test_odd_csr_shapes(ctx):
         _matches(ctx, rp, torch.from_numpy(colidx).cuda(), _random_numbering(N, 4))
 
 
-@pytest.mark.parametrize("nnz", [0, 1, 3, 4, 5, 8191, 8192, 8193, 16_387])
+@pytest.mark.parametrize("nnz", [0, 1, 3, 4, 5, 4095, 4096, 4097, 8191, 8192, 8193, 16_387])
 def test_tile_boundaries(ctx, nnz):
     rng = np.random.default_rng(nnz + 1)
     N = 97

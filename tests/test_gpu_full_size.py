@@ -106,3 +106,10 @@ def test_cfg4_graph_passes_full_size(ctx, cfg4):
     perm, inv = oracle.reorder(fine.assign.cpu().numpy(), w.reorder_K)
     np.testing.assert_array_equal(r.perm.cpu().numpy(), perm)
     np.testing.assert_array_equal(r.inv_perm.cpu().numpy(), inv)
+    # the numbering that the reordering run produced, scored the way Section 4.5.1 scores it (Eq. 3-5)
+    bw = ctx.graph_bandwidth(rowptr, colidx, r.inv_perm)
+    torch.cuda.synchronize()
+    ctx.check()
+    ref_bw = oracle.graph_bandwidth(rowptr.cpu().numpy(), colidx.cpu().numpy(), inv)
+    assert int(bw.bandwidth_sum.item()) == ref_bw.bandwidth_sum
+    np.testing.assert_array_equal(bw.vertex_bandwidth.cpu().numpy(), ref_bw.vertex_bandwidth)

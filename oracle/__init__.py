@@ -8,6 +8,7 @@ from .ep_oracle import (  # noqa: F401
     build,
     kmeans,
     assign_step,
+    sampled_kmeans,
     partition_quality,
     reorder,
     graph_bandwidth,

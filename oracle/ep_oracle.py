@@ -121,6 +121,26 @@ def assign_step(emb, centroids):
     return assign, b1, b2
 
 
+def sampled_kmeans(emb, sample_rows, K: int, iters: int, init_centroids) -> KMeansResult:
+    """Sampling-based clustering (Section 5, "Implementation": the centroids are computed from a sample of
+    the embeddings, 2^9 per cluster in the paper; every embedding is then given to its nearest centroid).
+
+    Steps, in that order: X_S = the rows `sample_rows` of emb (distinct row numbers); C_T = the centroids of
+    `iters` Lloyd iterations over X_S from `init_centroids`; a_i = argmin_k |x_i - C_T[k]|^2 for every row i
+    of emb (lowest index on ties).  Returned: that assignment, C_T, the objective trace of the iterations on
+    the sample, and the two smallest distances of every row to C_T."""
+    emb = _f32_matrix(emb, "emb")
+    rows = np.ascontiguousarray(sample_rows, dtype=np.int64)
+    N = emb.shape[0]
+    if rows.ndim != 1 or rows.size < K or rows.min() < 0 or rows.max() >= N or np.unique(rows).size != rows.size:
+        raise ValueError("sample_rows must be at least K distinct row numbers in [0, N)")
+    if iters < 1:
+        raise ValueError("the centroids need at least one iteration on the sample")
+    trained = kmeans(emb[rows], K, iters, init_centroids)
+    assign, b1, b2 = assign_step(emb, trained.centroids)
+    return KMeansResult(assign, trained.centroids, trained.objective, b1, b2)
+
+
 class QualityResult(NamedTuple):
     edge_cut: int
     part_vertices: np.ndarray  # int64 [K]

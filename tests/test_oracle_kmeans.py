@@ -201,3 +201,63 @@ def test_library_special_case_sklearn_lloyd():
         km = sk.KMeans(n_clusters=K, init=init.astype(np.float64), n_init=1, max_iter=T, tol=0.0,
                        algorithm="lloyd").fit(emb.astype(np.float64))
     np.testing.assert_allclose(km.cluster_centers_, r.centroids, rtol=1e-9, atol=1e-10)
+
+
+# ------------------------------------------------------------------------- sampling-based clustering
+def test_sampled_kmeans_with_every_row_in_the_sample_is_one_more_full_batch_assignment():
+    """Sample = all rows: the centroids are full-batch Lloyd's C_T, and the labels are the assignment that
+    full-batch Lloyd makes in iteration T + 1 (which is made against C_T)."""
+    rng = np.random.default_rng(21)
+    emb = rng.normal(size=(400, 6)).astype(np.float32)
+    init = emb[:5].copy()
+    T = 3
+    s = oracle.sampled_kmeans(emb, np.arange(400), 5, T, init)
+    full_T = oracle.kmeans(emb, 5, T, init)
+    full_T1 = oracle.kmeans(emb, 5, T + 1, init)
+    np.testing.assert_allclose(s.centroids, full_T.centroids, rtol=0, atol=0)
+    np.testing.assert_array_equal(s.assign, full_T1.assign)
+    np.testing.assert_allclose(s.objective, full_T.objective, rtol=0, atol=0)
+
+
+def test_sampled_kmeans_labels_are_nearest_centroids_by_enumeration():
+    rng = np.random.default_rng(22)
+    emb = rng.integers(-5, 6, size=(40, 3)).astype(np.float32)
+    rows = rng.permutation(40)[:12]
+    s = oracle.sampled_kmeans(emb, rows, 3, 2, emb[rows[:3]])
+    # the centroids depend on the sampled rows only
+    again = oracle.kmeans(emb[rows], 3, 2, emb[rows[:3]])
+    np.testing.assert_array_equal(s.centroids, again.centroids)
+    for i in range(40):
+        d = [float(((emb[i].astype(np.float64) - s.centroids[k]) ** 2).sum()) for k in range(3)]
+        assert s.assign[i] == int(np.argmin(d)) and s.best1[i] == min(d)    # argmin returns the lowest index on ties
+    # rows outside the sample do not move the centroids
+    emb2 = emb.copy()
+    outside = np.setdiff1d(np.arange(40), rows)
+    emb2[outside] += 100.0
+    np.testing.assert_array_equal(oracle.sampled_kmeans(emb2, rows, 3, 2, emb[rows[:3]]).centroids, s.centroids)
+
+
+def test_sampled_kmeans_recovers_a_well_separated_mixture_from_a_small_sample():
+    rng = np.random.default_rng(23)
+    K, per, d = 4, 300, 8
+    centres = rng.normal(size=(K, d)) * 50
+    z = np.repeat(np.arange(K), per)
+    emb = (centres[z] + rng.normal(size=(K * per, d))).astype(np.float32)
+    rows = np.concatenate([np.flatnonzero(z == k)[:8] for k in range(K)])          # 8 rows of each component
+    init = emb[[np.flatnonzero(z == k)[0] for k in range(K)]]
+    s = oracle.sampled_kmeans(emb, rows, K, 2, init)
+    np.testing.assert_array_equal(s.assign, z)
+    for k in range(K):
+        np.testing.assert_allclose(s.centroids[k], emb[rows[z[rows] == k]].astype(np.float64).mean(0), rtol=1e-12)
+
+
+def test_sampled_kmeans_rejects_bad_samples():
+    emb = np.zeros((10, 4), np.float32)
+    with pytest.raises(ValueError):
+        oracle.sampled_kmeans(emb, [0, 1, 1], 2, 1, emb[:2])          # a row twice
+    with pytest.raises(ValueError):
+        oracle.sampled_kmeans(emb, [0, 10], 2, 1, emb[:2])            # outside [0, N)
+    with pytest.raises(ValueError):
+        oracle.sampled_kmeans(emb, [0], 2, 1, emb[:2])                # fewer rows than clusters
+    with pytest.raises(ValueError):
+        oracle.sampled_kmeans(emb, [0, 1], 2, 0, emb[:2])             # no iteration

@@ -438,6 +438,27 @@ def main():
                 "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
                              "traffic": None, "peak_source": peaks["_source"]}}
 
+    # ---- outside the step: sampling-based clustering as the paper ran it (2^9 rows per cluster train the
+    # centroids, then one pass labels every row)
+    M = min(w.N, 512 * w.K)
+    if M >= w.K:
+        rows = synth.subsample_rows(w, M, device=device).to(torch.int64).contiguous()
+        init_s = x["emb"][rows[: w.K]].contiguous()
+        ctx.kmeans_sampled(x["emb"], w.K, w.iters, rows, init_s)
+        torch.cuda.synchronize()
+        reps = 3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            ctx.kmeans_sampled(x["emb"], w.K, w.iters, rows, init_s)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx.check()
+        ms_s = e0.elapsed_time(e1) / reps
+        extras["sampled_kmeans"] = {"ms_per_call": ms_s, "rows_labelled_per_s": w.N / (ms_s * 1e-3),
+                                    "sample_rows": M, "iters_on_sample": w.iters, "K": w.K,
+                                    "full_pass_gbs": w.N * (4 * w.d + 4) / (ms_s * 1e-3) / 1e9}
+
     # ---- end to end: the same pass through the host-buffer C ABI (uploads and downloads timed) ---------
     e2e = None
     if not args.no_e2e:

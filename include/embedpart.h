@@ -137,6 +137,29 @@ int ep_kmeans(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, in
               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
+ * ep_kmeans_sampled -- sampling-based clustering (Section 5, "Implementation": the centroids are
+ * computed from a sample of the embeddings, 2^9 per cluster in the paper; every embedding is
+ * then assigned to its nearest centroid).
+ *
+ * Three steps on the stream: the rows sample_rows of emb are gathered into the workspace;
+ * `iters` >= 1 Lloyd iterations run over them from init_centroids (exactly as ep_kmeans);
+ * one assign-only pass labels all N rows against the resulting centroids.  Unlike ep_kmeans,
+ * the labels returned are those of the final centroids.
+ *
+ *   emb, N, d, K, init_centroids, centroids: as for ep_kmeans
+ *   sample_rows [dev] M int64 row numbers in [0, N), distinct (not checked);  K <= M <= N
+ *   assign      [dev] out, N int32
+ * A row number outside [0, N) raises EP_ERR_BAD_INDEX in the device status word and is read as
+ * row 0.  ep_gather_rows is the first step on its own: out[i] = emb[rows[i]].
+ */
+size_t ep_kmeans_sampled_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int64_t M);
+int ep_kmeans_sampled(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                      const int64_t *sample_rows, int64_t M, const float *init_centroids, int32_t *assign,
+                      float *centroids, void *workspace, size_t workspace_bytes, void *cuda_stream);
+int ep_gather_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const int64_t *rows, int64_t M,
+                   float *out /* [dev] M x d, 16-byte aligned */, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
  * ep_partition_quality -- edge cut and partition loads (Eq. 1 numerator, Eq. 2 operands).
  *
  *   edge_cut         = number of stored CSR entries (u -> v) with assign[u] != assign[v]; entries

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     ep_reorder,
     ep_reorder_static,
     ep_graph_bandwidth,
+    ep_kmeans_sampled,
     library_path,
     load_library,
     EXPORTED_SYMBOLS,

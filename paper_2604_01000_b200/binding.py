@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = (
     "ep_kmeans_host_arena_bytes", "ep_kmeans_host", "ep_quality_host_arena_bytes", "ep_partition_quality_host",
     "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static", "ep_debug_counters",
     "ep_graph_bandwidth_workspace_bytes", "ep_graph_bandwidth", "ep_graph_bandwidth_host_arena_bytes",
-    "ep_graph_bandwidth_host",
+    "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
 )
 
 EP_OK = 0
@@ -105,6 +105,12 @@ def load_library() -> ctypes.CDLL:
             lib.ep_reorder_host.restype = ctypes.c_int
             lib.ep_reorder_static.argtypes = [vp, i64, i32, vp, vp, vp, vp]
             lib.ep_reorder_static.restype = ctypes.c_int
+            lib.ep_kmeans_sampled_workspace_bytes.argtypes = [vp, i64, i32, i32, i64]
+            lib.ep_kmeans_sampled_workspace_bytes.restype = sz
+            lib.ep_kmeans_sampled.argtypes = [vp, vp, i64, i32, i32, i32, vp, i64, vp, vp, vp, vp, sz, vp]
+            lib.ep_kmeans_sampled.restype = ctypes.c_int
+            lib.ep_gather_rows.argtypes = [vp, vp, i64, i32, vp, i64, vp, vp]
+            lib.ep_gather_rows.restype = ctypes.c_int
             lib.ep_graph_bandwidth_workspace_bytes.argtypes = [vp, i64, i64]
             lib.ep_graph_bandwidth_workspace_bytes.restype = sz
             lib.ep_graph_bandwidth.argtypes = [vp, vp, i32, vp, i64, vp, i64, vp, vp, vp, sz, vp]
@@ -242,6 +248,42 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return KMeansResult(assign, cent, obj)
+
+    def gather_rows(self, emb, rows):
+        """out[i] = emb[rows[i]] (rows: int64 CUDA tensor)."""
+        emb = _check_cuda(emb, torch.float32, "emb", self.device)
+        rows = _check_cuda(rows, torch.int64, "rows", self.device)
+        N, d = emb.shape
+        out = torch.empty(rows.numel(), d, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_gather_rows(self._h, _dev_ptr(emb), N, d, _dev_ptr(rows), rows.numel(), _dev_ptr(out),
+                                          self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+    def kmeans_sampled(self, emb, K: int, iters: int, sample_rows, init_centroids):
+        """Centroids from `iters` Lloyd iterations over the rows `sample_rows`, then every row of emb assigned
+        to its nearest centroid: (assign, centroids, None)."""
+        emb = _check_cuda(emb, torch.float32, "emb", self.device)
+        rows = _check_cuda(sample_rows, torch.int64, "sample_rows", self.device)
+        init = _check_cuda(init_centroids, torch.float32, "init_centroids", self.device)
+        N, d = emb.shape
+        if init.shape != (K, d):
+            raise ValueError("init_centroids must be K x d")
+        M = rows.numel()
+        need = self._lib.ep_kmeans_sampled_workspace_bytes(self._h, N, d, K, M)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} d={d} K={K} M={M}")
+        ws = self.workspace(need)
+        assign = torch.empty(N, dtype=torch.int32, device=self.device)
+        cent = torch.empty(K, d, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_kmeans_sampled(self._h, _dev_ptr(emb), N, d, K, iters, _dev_ptr(rows), M, _dev_ptr(init),
+                                             _dev_ptr(assign), _dev_ptr(cent), _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return KMeansResult(assign, cent, None)
 
     def partition_quality(self, rowptr, colidx, assign, K: int):
         if rowptr.dtype not in (torch.int32, torch.int64):
@@ -440,6 +482,11 @@ def ep_partition_quality(rowptr, colidx, assign, K) -> QualityResult:
 def ep_reorder(assign, K, inverse=True) -> ReorderResult:
     """Partition-ordered permutation (and its inverse)."""
     return default_context(assign.device.index).reorder(assign, K, inverse)
+
+
+def ep_kmeans_sampled(emb, K, iters, sample_rows, init_centroids) -> KMeansResult:
+    """Sampling-based clustering: centroids from the sampled rows, labels for every row."""
+    return default_context(emb.device.index).kmeans_sampled(emb, K, iters, sample_rows, init_centroids)
 
 
 def ep_graph_bandwidth(rowptr, colidx, pi, per_vertex=True) -> BandwidthResult:

@@ -1,6 +1,7 @@
 // C ABI entry points: argument checks on the host, then the kernels of the other translation units.
 #include "ep_common.cuh"
 
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -54,6 +55,51 @@ void Timed::end(int kernels) {
 }  // namespace ep
 
 using namespace ep;
+
+namespace {
+
+// out[i] = emb[rows[i]]: a warp per row, 16 bytes per lane and step.
+__global__ void __launch_bounds__(256) gather_rows(const float *__restrict__ emb, int64_t N, int d4,
+                                                   const int64_t *__restrict__ rows, int64_t M,
+                                                   float *__restrict__ out, int *status) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t i = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < M; i += warps) {
+        int64_t r = rows[i];
+        if (r < 0 || r >= N) {
+            if (lane == 0) ep_raise(status, EP_ERR_BAD_INDEX);
+            r = 0;
+        }
+        const float4 *src = reinterpret_cast<const float4 *>(emb) + r * d4;
+        float4 *dst = reinterpret_cast<float4 *>(out) + i * d4;
+        for (int q = lane; q < d4; q += 32) dst[q] = __ldg(src + q);
+    }
+}
+
+struct SampledLayout {
+    float *sample;
+    int32_t *sample_assign;
+    void *ws_train, *ws_full;
+    size_t train_bytes, full_bytes, used;
+};
+
+bool sampled_layout(const ep_ctx *ctx, int64_t N, int d, int K, int64_t M, void *workspace, SampledLayout *out) {
+    KMeansPlan train, full;
+    if (M < K || M > N || !kmeans_make_plan(ctx, M, d, K, &train) || !kmeans_make_plan(ctx, N, d, K, &full)) return false;
+    Arena a(workspace);
+    SampledLayout l{};
+    l.sample = a.take<float>((size_t)M * d);
+    l.sample_assign = a.take<int32_t>(M);
+    l.train_bytes = kmeans_workspace_layout(ctx, train, nullptr, nullptr);
+    l.full_bytes = kmeans_workspace_layout(ctx, full, nullptr, nullptr);
+    l.ws_train = a.take<char>(l.train_bytes);
+    l.ws_full = a.take<char>(l.full_bytes);
+    l.used = a.used;
+    *out = l;
+    return true;
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -227,6 +273,49 @@ int ep_kmeans(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, in
     DeviceGuard g(ctx->device);
     return kmeans_run(ctx, plan, emb, iters, init_centroids, assign, centroids, objective, workspace,
                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------------------------- sampled k-means
+int ep_gather_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const int64_t *rows, int64_t M, float *out,
+                   void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !rows || !out) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (N < 1 || M < 1 || d < 4 || d > 1024 || (d & 3))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld M=%lld d=%d", (long long)N, (long long)M, d);
+    if (!aligned(emb, 16) || !aligned(out, 16) || !aligned(rows, 8)) return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(M, 8)));
+    gather_rows<<<grid, 256, 0, st>>>(emb, N, d >> 2, rows, M, out, ctx->d_status);
+    ctx->launches += 1;
+    EP_CUDA(ctx, cudaGetLastError());
+    return EP_OK;
+}
+
+size_t ep_kmeans_sampled_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int64_t M) {
+    SampledLayout l;
+    if (!ctx || !sampled_layout(ctx, N, d, K, M, nullptr, &l)) return 0;
+    return l.used;
+}
+
+int ep_kmeans_sampled(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                      const int64_t *sample_rows, int64_t M, const float *init_centroids, int32_t *assign,
+                      float *centroids, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !sample_rows || !init_centroids || !assign || !centroids) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (iters < 1) return fail(ctx, EP_ERR_INVALID_ARG, "the centroids need at least one iteration on the sample");
+    SampledLayout l;
+    if (!sampled_layout(ctx, N, d, K, M, workspace, &l))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld d=%d K=%d M=%lld (K <= M <= N)", (long long)N, d, K,
+                    (long long)M);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < l.used)
+        return fail(ctx, EP_ERR_WORKSPACE, "sampled k-means workspace: need %zu bytes, 256-byte aligned", l.used);
+    int rc = ep_gather_rows(ctx, emb, N, d, sample_rows, M, l.sample, cuda_stream);
+    if (rc != EP_OK) return rc;
+    rc = ep_kmeans(ctx, l.sample, M, d, K, iters, init_centroids, l.sample_assign, centroids, nullptr, l.ws_train,
+                   l.train_bytes, cuda_stream);
+    if (rc != EP_OK) return rc;
+    return ep_kmeans(ctx, emb, N, d, K, 0, centroids, assign, centroids, nullptr, l.ws_full, l.full_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------- quality

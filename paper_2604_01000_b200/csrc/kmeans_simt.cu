@@ -242,19 +242,32 @@ __global__ void __launch_bounds__(256) kmeans_segment_sums(const float *__restri
     float4 acc[VPL];
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int64_t p = p0 + warp; p < p1; p += 8) {
-        const int64_t row = order[p];
+    // several rows of this warp in flight at a time; they are added in the order of the list all the same
+    constexpr int AHEAD = VPL <= 2 ? 4 : VPL == 4 ? 2 : 1;
+    for (int64_t p = p0 + warp; p < p1; p += 8 * AHEAD) {
+        int64_t row[AHEAD];
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-            int q = lane + 32 * v;
-            if (q < d4) {
-                float4 x = ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q);
-                acc[v].x += x.x;
-                acc[v].y += x.y;
-                acc[v].z += x.z;
-                acc[v].w += x.w;
+        for (int u = 0; u < AHEAD; ++u) row[u] = p + 8 * u < p1 ? (int64_t)order[p + 8 * u] : -1;
+        float4 x[AHEAD][VPL];
+#pragma unroll
+        for (int u = 0; u < AHEAD; ++u)
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int q = lane + 32 * v;
+                x[u][v] = (row[u] >= 0 && q < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + row[u] * d4 + q)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-        }
+#pragma unroll
+        for (int u = 0; u < AHEAD; ++u)
+            if (row[u] >= 0) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) {
+                    acc[v].x += x[u][v].x;
+                    acc[v].y += x[u][v].y;
+                    acc[v].z += x[u][v].z;
+                    acc[v].w += x[u][v].w;
+                }
+            }
     }
 #pragma unroll
     for (int v = 0; v < VPL; ++v) red[warp][lane + 32 * v] = acc[v];
@@ -274,9 +287,29 @@ __global__ void __launch_bounds__(256) kmeans_segment_sums(const float *__restri
 }
 
 // hist[k] = number of rows labelled k (integer atomics: exact whatever the order).
-__global__ void label_histogram(const int32_t *__restrict__ assign, int64_t N, int K, unsigned long long *hist) {
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += (int64_t)gridDim.x * blockDim.x)
-        atomicAdd(&hist[assign[i]], 1ull);
+// Up to LH_SMEM_K clusters are first counted in the block's shared memory.
+constexpr int LH_SMEM_K = 8192;
+
+__global__ void __launch_bounds__(256) label_histogram(const int32_t *__restrict__ assign, int64_t N, int K,
+                                                       unsigned long long *hist) {
+    __shared__ unsigned int local[LH_SMEM_K];
+    const bool in_block = K <= LH_SMEM_K;
+    if (in_block) {
+        for (int k = threadIdx.x; k < K; k += blockDim.x) local[k] = 0u;
+        __syncthreads();
+    }
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += (int64_t)gridDim.x * blockDim.x) {
+        const int a = assign[i];
+        if (in_block)
+            atomicAdd(&local[a], 1u);
+        else
+            atomicAdd(&hist[a], 1ull);
+    }
+    if (in_block) {
+        __syncthreads();
+        for (int k = threadIdx.x; k < K; k += blockDim.x)
+            if (local[k]) atomicAdd(&hist[k], (unsigned long long)local[k]);
+    }
 }
 
 // off[0..K] = exclusive prefix sum of hist (one block; K <= 65536).

@@ -12,6 +12,8 @@ from .ep_oracle import (  # noqa: F401
     partition_quality,
     reorder,
     graph_bandwidth,
+    relabel_graph,
+    permute_rows,
     num_threads,
     set_num_threads,
 )

@@ -6,6 +6,7 @@
  *   - edge cut and per-partition loads           (Section 2.1.1, Eq. 1 and Eq. 2)
  *   - the partition-ordered vertex permutation   (Section 4.5.1, "Adapting EmbedPart for Reordering")
  *   - the average graph bandwidth of a numbering (Section 4.5.1, Eq. 3, Eq. 4 and Eq. 5)
+ *   - the graph and the embedding rows stored under the new numbering (Section 4.5.1)
  *
  * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call
  * this file.  It shares no code, header, table or helper with the CUDA library
@@ -242,4 +243,30 @@ void oracle_graph_bandwidth(const int64_t *rowptr, const int32_t *colidx, const 
         total += beta;
     }
     *bandwidth_sum = (uint64_t)total;
+}
+
+/*
+ * The graph stored under a new numbering (Section 4.5.1: the ids of the vertices are their
+ * positions in memory, and reordering relabels them).  perm[new_id] = old id and
+ * inv_perm[old id] = new id, as oracle_reorder returns them.  Row i of the new graph is row
+ * perm[i] of the old one with every column id u replaced by inv_perm[u]; the entries of a row keep
+ * their stored order (the paper does not ask for sorted rows), so exactly one output is correct.
+ */
+void oracle_relabel_graph(const int64_t *rowptr, const int32_t *colidx, const int32_t *perm,
+                          const int32_t *inv_perm, int64_t N, int64_t *new_rowptr, int32_t *new_colidx)
+{
+    new_rowptr[0] = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        int64_t v = perm[i];
+        int64_t at = new_rowptr[i];
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) new_colidx[at++] = inv_perm[colidx[e]];
+        new_rowptr[i + 1] = at;
+    }
+}
+
+/* Embedding (or feature) rows under the new numbering: out[i] = emb[perm[i]]. */
+void oracle_permute_rows(const float *emb, int64_t N, int32_t d, const int32_t *perm, float *out)
+{
+    for (int64_t i = 0; i < N; ++i)
+        memcpy(out + (size_t)i * d, emb + (size_t)perm[i] * d, sizeof(float) * (size_t)d);
 }

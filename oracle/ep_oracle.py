@@ -46,6 +46,10 @@ def _load():
         lib.oracle_reorder.restype = ctypes.c_int
         lib.oracle_graph_bandwidth.argtypes = [p, p, p, ctypes.c_int64, p, p]
         lib.oracle_graph_bandwidth.restype = None
+        lib.oracle_relabel_graph.argtypes = [p, p, p, p, ctypes.c_int64, p, p]
+        lib.oracle_relabel_graph.restype = None
+        lib.oracle_permute_rows.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, p]
+        lib.oracle_permute_rows.restype = None
         _lib = lib
     return _lib
 
@@ -204,3 +208,41 @@ def graph_bandwidth(rowptr, colidx, pi) -> BandwidthResult:
     vb = np.empty(N, np.int32)
     _load().oracle_graph_bandwidth(_ptr(rowptr), _ptr(colidx), _ptr(pi), N, ctypes.addressof(total), _ptr(vb))
     return BandwidthResult(int(total.value), vb)
+
+
+def _permutation_pair(perm, inv_perm, N: int):
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    inv = np.ascontiguousarray(inv_perm, dtype=np.int32)
+    if perm.shape != (N,) or inv.shape != (N,) or not np.array_equal(np.sort(perm), np.arange(N, dtype=np.int32)):
+        raise ValueError("perm must be a permutation of [0, N)")
+    if not np.array_equal(inv[perm], np.arange(N, dtype=np.int32)):
+        raise ValueError("inv_perm is not the inverse of perm")
+    return perm, inv
+
+
+def relabel_graph(rowptr, colidx, perm, inv_perm):
+    """(new_rowptr int64, new_colidx int32): row i = old row perm[i] with ids mapped through inv_perm."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    N = rowptr.shape[0] - 1
+    perm, inv = _permutation_pair(perm, inv_perm, N)
+    if rowptr[0] != 0 or rowptr[-1] != colidx.shape[0] or np.any(np.diff(rowptr) < 0):
+        raise ValueError("rowptr is not a CSR row pointer for colidx")
+    if colidx.size and (colidx.min() < 0 or colidx.max() >= N):
+        raise ValueError("colidx value outside [0, N)")
+    new_rowptr = np.empty(N + 1, np.int64)
+    new_colidx = np.empty(colidx.shape[0], np.int32)
+    _load().oracle_relabel_graph(_ptr(rowptr), _ptr(colidx), _ptr(perm), _ptr(inv), N, _ptr(new_rowptr), _ptr(new_colidx))
+    return new_rowptr, new_colidx
+
+
+def permute_rows(emb, perm):
+    """out[i] = emb[perm[i]]."""
+    emb = _f32_matrix(emb, "emb")
+    N, d = emb.shape
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    if perm.shape != (N,) or not np.array_equal(np.sort(perm), np.arange(N, dtype=np.int32)):
+        raise ValueError("perm must be a permutation of [0, N)")
+    out = np.empty_like(emb)
+    _load().oracle_permute_rows(_ptr(emb), N, d, _ptr(perm), _ptr(out))
+    return out

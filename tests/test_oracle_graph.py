@@ -221,3 +221,52 @@ def test_bandwidth_rejects_bad_input():
         oracle.graph_bandwidth([0, 1, 2], [1, 0], [0, 0])            # not a bijection
     with pytest.raises(ValueError):
         oracle.graph_bandwidth([0, 1, 2], [1, 5], [0, 1])            # neighbour outside [0, N)
+
+
+# ------------------------------------------------------------------- the graph under a new numbering
+def test_relabel_hand_case():
+    """Path 0-1-2-3 numbered 2,0,3,1 (perm = [1,3,0,2]): worked by hand.
+    new vertex 0 = old 1 (neighbours 0,2 -> 2,3); 1 = old 3 (2 -> 3); 2 = old 0 (1 -> 0); 3 = old 2 (1,3 -> 0,1)."""
+    rowptr, colidx = [0, 1, 3, 5, 6], [1, 0, 2, 1, 3, 2]
+    perm, inv = [1, 3, 0, 2], [2, 0, 3, 1]
+    rp, ci = oracle.relabel_graph(rowptr, colidx, perm, inv)
+    assert rp.tolist() == [0, 2, 3, 4, 6] and ci.tolist() == [2, 3, 3, 0, 0, 1]
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_relabel_is_the_same_graph_under_other_names(seed):
+    rng = np.random.default_rng(200 + seed)
+    N, K = int(rng.integers(5, 40)), 4
+    A, rowptr, colidx = _random_csr(rng, N, 0.2, symmetric=bool(seed % 2), loops=True)
+    assign = rng.integers(0, K, size=N).astype(np.int32)
+    perm, inv = oracle.reorder(assign, K)
+    rp, ci = oracle.relabel_graph(rowptr, colidx, perm, inv)
+    # adjacency matrix renamed on both axes
+    A2 = np.zeros_like(A)
+    for i in range(N):
+        A2[i, ci[rp[i]:rp[i + 1]]] = True
+    assert np.array_equal(A2, A[np.ix_(perm, perm)])
+    assert np.array_equal(np.diff(rp), np.diff(rowptr)[perm])
+    # the metrics do not care about names: cut with renamed labels, bandwidth with the identity numbering
+    q, q2 = oracle.partition_quality(rowptr, colidx, assign, K), oracle.partition_quality(rp, ci, assign[perm], K)
+    assert q.edge_cut == q2.edge_cut and q.part_vertices.tolist() == q2.part_vertices.tolist()
+    b, b2 = oracle.graph_bandwidth(rowptr, colidx, inv), oracle.graph_bandwidth(rp, ci, np.arange(N))
+    assert b.bandwidth_sum == b2.bandwidth_sum and np.array_equal(b2.vertex_bandwidth, b.vertex_bandwidth[perm])
+    # identity numbering changes nothing; relabelling back restores every row, entry order included
+    ident = np.arange(N, dtype=np.int32)
+    rp0, ci0 = oracle.relabel_graph(rowptr, colidx, ident, ident)
+    assert np.array_equal(rp0, rowptr) and np.array_equal(ci0, colidx)
+    rp3, ci3 = oracle.relabel_graph(rp, ci, inv, perm)
+    assert np.array_equal(rp3, rowptr) and np.array_equal(ci3, colidx)
+
+
+def test_permute_rows_and_bad_permutations():
+    rng = np.random.default_rng(9)
+    emb = rng.normal(size=(17, 8)).astype(np.float32)
+    perm = rng.permutation(17).astype(np.int32)
+    out = oracle.permute_rows(emb, perm)
+    assert np.array_equal(out, emb[perm])
+    with pytest.raises(ValueError):
+        oracle.permute_rows(emb, np.zeros(17, np.int32))
+    with pytest.raises(ValueError):
+        oracle.relabel_graph([0, 1, 2], [1, 0], [0, 1], [1, 0])        # inv_perm is not the inverse

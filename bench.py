@@ -438,6 +438,41 @@ def main():
                 "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
                              "traffic": None, "peak_source": peaks["_source"]}}
 
+    # ---- outside the step: the graph and the rows stored under the numbering the step produced -----------
+    if last is not None and last[3].inv_perm is not None:
+        reps = 3
+        ctx.relabel_graph(x["rowptr"], x["colidx"], last[3].perm, last[3].inv_perm)
+        torch.cuda.synchronize()
+        ctx.profile_read("relabel", 0)
+        ctx.set_profile(True)
+        for _ in range(reps):
+            ctx.relabel_graph(x["rowptr"], x["colidx"], last[3].perm, last[3].inv_perm)
+        torch.cuda.synchronize()
+        tot_g, n_g = ctx.profile_read("relabel", 0)
+        out_rows = None
+        if w.N * w.d * 4 <= 8e9:                       # the copy of the matrix has to fit beside it
+            out_rows = ctx.permute_rows(x["emb"], last[3].perm)
+            torch.cuda.synchronize()
+            ctx.profile_read("relabel", 0)
+            for _ in range(reps):
+                ctx.permute_rows(x["emb"], last[3].perm)
+            torch.cuda.synchronize()
+        tot_r, n_r = ctx.profile_read("relabel", 0)
+        ctx.set_profile(False)
+        ctx.check()
+        del out_rows
+        if n_g:
+            by = 8 * nnz + 2 * rp_bytes * (w.N + 1) + 8 * w.N      # column ids in and out, both row pointers, perm + inv_perm
+            gbs = by * reps / (tot_g * 1e-3) / 1e9
+            extras["relabel_graph"] = {"ms_per_pass": tot_g / reps, "rate": nnz * reps / (tot_g * 1e-3), "unit": "edges/s",
+                                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
+                                                    "frac": gbs / hbm, "traffic": None, "peak_source": peaks["_source"]}}
+        if n_r:
+            gbs = (8 * w.d + 4) * w.N * reps / (tot_r * 1e-3) / 1e9
+            extras["permute_rows"] = {"ms_per_pass": tot_r / reps, "rate": w.N * reps / (tot_r * 1e-3), "unit": "rows/s",
+                                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
+                                                   "frac": gbs / hbm, "traffic": None, "peak_source": peaks["_source"]}}
+
     # ---- outside the step: sampling-based clustering as the paper ran it (2^9 rows per cluster train the
     # centroids, then one pass labels every row)
     M = min(w.N, 512 * w.K)

@@ -71,7 +71,8 @@ enum {
     EP_TIMER_REORDER = 4,        /* all kernels of ep_reorder */
     EP_TIMER_KMEANS_RESOLVE = 5, /* tensor-core path: the fp32 kernel that decides the labels */
     EP_TIMER_GRAPH_BANDWIDTH = 6, /* all kernels of ep_graph_bandwidth */
-    EP_TIMER_COUNT = 7
+    EP_TIMER_RELABEL = 7,        /* all kernels of ep_relabel_graph and ep_permute_rows */
+    EP_TIMER_COUNT = 8
 };
 
 typedef struct ep_ctx ep_ctx; /* opaque: device id, device properties, device status word, options */
@@ -225,6 +226,29 @@ size_t ep_graph_bandwidth_host_arena_bytes(const ep_ctx *ctx, int64_t N, int64_t
 int ep_graph_bandwidth_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx,
                             int64_t nnz, const int32_t *pi, int64_t N, uint64_t *bandwidth_sum,
                             int32_t *vertex_bandwidth, void *arena, size_t arena_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_relabel_graph, ep_permute_rows -- the graph and the embedding (or feature) rows stored under
+ * the new numbering (Section 4.5.1: vertex ids are positions in memory; reordering relabels them).
+ *
+ * perm and inv_perm are the outputs of ep_reorder.  Row i of the new graph is row perm[i] of the
+ * old one with every column id u replaced by inv_perm[u]; the entries of a row keep their stored
+ * order, so exactly one output is correct.  ep_permute_rows writes out[i] = emb[perm[i]].
+ *
+ *   rowptr, colidx, nnz, N: as for ep_partition_quality
+ *   perm, inv_perm [dev] N int32 each, inverse permutations of [0, N) (not checked beyond range)
+ *   new_rowptr     [dev] out, N+1 offsets of the same width as rowptr
+ *   new_colidx     [dev] out, nnz int32
+ *   emb, out       [dev] N x d fp32 row-major, 16-byte aligned, d a multiple of 4 in [4, 1024]; not the same buffer
+ * A value of perm or colidx outside [0, N) raises EP_ERR_BAD_INDEX in the device status word (the row
+ * comes out empty, the id as 0).
+ */
+size_t ep_relabel_graph_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz);
+int ep_relabel_graph(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx, int64_t nnz,
+                     const int32_t *perm, const int32_t *inv_perm, int64_t N, void *new_rowptr,
+                     int32_t *new_colidx, void *workspace, size_t workspace_bytes, void *cuda_stream);
+int ep_permute_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const int32_t *perm, float *out,
+                    void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
  * Host-buffer variants.  Same operations and the same kernels; inputs and outputs are [host]

@@ -19,6 +19,7 @@ EXPORTED_SYMBOLS = (
     "ep_reorder_host_arena_bytes", "ep_reorder_host", "ep_reorder_static", "ep_debug_counters",
     "ep_graph_bandwidth_workspace_bytes", "ep_graph_bandwidth", "ep_graph_bandwidth_host_arena_bytes",
     "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
+    "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
 )
 
 EP_OK = 0
@@ -26,9 +27,9 @@ EP_OPT_KMEANS_PATH = 1
 EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
 EP_OPT_KMEANS_CAND_MB = 4
-TIMER_COUNT = 7
+TIMER_COUNT = 8
 TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
-          "kmeans_resolve": 5, "graph_bandwidth": 6}
+          "kmeans_resolve": 5, "graph_bandwidth": 6, "relabel": 7}
 KMEANS_PATHS = {"auto": 0, "simt": 1, "tensor": 2}
 
 
@@ -111,6 +112,12 @@ def load_library() -> ctypes.CDLL:
             lib.ep_kmeans_sampled.restype = ctypes.c_int
             lib.ep_gather_rows.argtypes = [vp, vp, i64, i32, vp, i64, vp, vp]
             lib.ep_gather_rows.restype = ctypes.c_int
+            lib.ep_relabel_graph_workspace_bytes.argtypes = [vp, i64, i64]
+            lib.ep_relabel_graph_workspace_bytes.restype = sz
+            lib.ep_relabel_graph.argtypes = [vp, vp, i32, vp, i64, vp, vp, i64, vp, vp, vp, sz, vp]
+            lib.ep_relabel_graph.restype = ctypes.c_int
+            lib.ep_permute_rows.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+            lib.ep_permute_rows.restype = ctypes.c_int
             lib.ep_graph_bandwidth_workspace_bytes.argtypes = [vp, i64, i64]
             lib.ep_graph_bandwidth_workspace_bytes.restype = sz
             lib.ep_graph_bandwidth.argtypes = [vp, vp, i32, vp, i64, vp, i64, vp, vp, vp, sz, vp]
@@ -324,6 +331,45 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return ReorderResult(perm, inv)
+
+    def relabel_graph(self, rowptr, colidx, perm, inv_perm):
+        """(new_rowptr, new_colidx): the CSR graph with vertex perm[i] renamed i."""
+        if rowptr.dtype not in (torch.int32, torch.int64):
+            raise ValueError("rowptr must be int32 or int64")
+        rowptr = _check_cuda(rowptr, rowptr.dtype, "rowptr", self.device)
+        colidx = _check_cuda(colidx, torch.int32, "colidx", self.device)
+        perm = _check_cuda(perm, torch.int32, "perm", self.device)
+        inv_perm = _check_cuda(inv_perm, torch.int32, "inv_perm", self.device)
+        N, nnz = perm.numel(), colidx.numel()
+        if rowptr.numel() != N + 1 or inv_perm.numel() != N:
+            raise ValueError("rowptr must have N + 1 entries, inv_perm N")
+        need = self._lib.ep_relabel_graph_workspace_bytes(self._h, N, nnz)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} nnz={nnz}")
+        ws = self.workspace(need)
+        new_rowptr = torch.empty_like(rowptr)
+        new_colidx = torch.empty_like(colidx)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_relabel_graph(self._h, _dev_ptr(rowptr), int(rowptr.dtype == torch.int64), _dev_ptr(colidx),
+                                            nnz, _dev_ptr(perm), _dev_ptr(inv_perm), N, _dev_ptr(new_rowptr),
+                                            _dev_ptr(new_colidx), _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return new_rowptr, new_colidx
+
+    def permute_rows(self, emb, perm):
+        """out[i] = emb[perm[i]] (perm: int32 CUDA tensor of N entries)."""
+        emb = _check_cuda(emb, torch.float32, "emb", self.device)
+        perm = _check_cuda(perm, torch.int32, "perm", self.device)
+        N, d = emb.shape
+        if perm.numel() != N:
+            raise ValueError("perm must have N entries")
+        out = torch.empty_like(emb)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_permute_rows(self._h, _dev_ptr(emb), N, d, _dev_ptr(perm), _dev_ptr(out), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
 
     def graph_bandwidth(self, rowptr, colidx, pi, per_vertex: bool = True):
         """Sum of the vertex bandwidths of the numbering pi (pi[v] = new id of v) and, if asked, each of them."""

@@ -426,6 +426,45 @@ int ep_graph_bandwidth_host(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_i
     return EP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------- relabel
+size_t ep_relabel_graph_workspace_bytes(const ep_ctx *ctx, int64_t N, int64_t nnz) {
+    if (!ctx || !bandwidth_shape_ok(N, nnz)) return 0;
+    return relabel_workspace_bytes(N, nnz);
+}
+
+int ep_relabel_graph(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, const int32_t *colidx, int64_t nnz,
+                     const int32_t *perm, const int32_t *inv_perm, int64_t N, void *new_rowptr, int32_t *new_colidx,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!bandwidth_shape_ok(N, nnz))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld", (long long)N, (long long)nnz);
+    if (!rowptr || (!colidx && nnz > 0) || !perm || !inv_perm || !new_rowptr || (!new_colidx && nnz > 0))
+        return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!rowptr_is_int64 && nnz >= (int64_t(1) << 31))
+        return fail(ctx, EP_ERR_INVALID_ARG, "nnz needs a 64-bit row pointer");
+    const size_t rw = rowptr_is_int64 ? 8 : 4;
+    if (!aligned(rowptr, rw) || !aligned(new_rowptr, rw) || !aligned(colidx, 4) || !aligned(new_colidx, 4) ||
+        !aligned(perm, 4) || !aligned(inv_perm, 4))
+        return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    const size_t need = relabel_workspace_bytes(N, nnz);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "relabel workspace: need %zu bytes, 256-byte aligned", need);
+    DeviceGuard g(ctx->device);
+    return relabel_run(ctx, rowptr, rowptr_is_int64 != 0, colidx, nnz, perm, inv_perm, N, new_rowptr, new_colidx, workspace,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ep_permute_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const int32_t *perm, float *out,
+                    void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !perm || !out || emb == out) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer or out == emb");
+    if (N < 1 || N >= (int64_t(1) << 31) || d < 4 || d > 1024 || (d & 3))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld d=%d", (long long)N, d);
+    if (!aligned(emb, 16) || !aligned(out, 16) || !aligned(perm, 4)) return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    DeviceGuard g(ctx->device);
+    return permute_rows_run(ctx, emb, N, d, perm, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
 // ---------------------------------------------------------------------------------------------- reorder
 static bool reorder_shape_ok(int64_t N, int32_t K) {
     return N >= 1 && N < (int64_t(1) << 31) && K >= 1 && K <= (1 << 24);

@@ -145,6 +145,14 @@ int bandwidth_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t 
                   const int32_t *pi, int64_t N, unsigned long long *total, int32_t *vertex_bandwidth, void *workspace,
                   cudaStream_t stream);
 
+// ---- the graph under a new numbering (relabel.cu) -------------------------------------------------
+size_t relabel_workspace_bytes(int64_t N, int64_t nnz);
+int relabel_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *colidx, int64_t nnz, const int32_t *perm,
+                const int32_t *inv_perm, int64_t N, void *new_rowptr, int32_t *new_colidx, void *workspace,
+                cudaStream_t stream);
+int permute_rows_run(ep_ctx *ctx, const float *emb, int64_t N, int d, const int32_t *perm, float *out,
+                     cudaStream_t stream);
+
 }  // namespace ep
 
 // ---- device helpers -------------------------------------------------------------------------------

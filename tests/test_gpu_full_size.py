@@ -113,3 +113,10 @@ def test_cfg4_graph_passes_full_size(ctx, cfg4):
     ref_bw = oracle.graph_bandwidth(rowptr.cpu().numpy(), colidx.cpu().numpy(), inv)
     assert int(bw.bandwidth_sum.item()) == ref_bw.bandwidth_sum
     np.testing.assert_array_equal(bw.vertex_bandwidth.cpu().numpy(), ref_bw.vertex_bandwidth)
+    # ... and the graph stored under that numbering
+    rp2, ci2 = ctx.relabel_graph(rowptr, colidx, r.perm, r.inv_perm)
+    torch.cuda.synchronize()
+    ctx.check()
+    ref_rp, ref_ci = oracle.relabel_graph(rowptr.cpu().numpy(), colidx.cpu().numpy(), perm, inv)
+    np.testing.assert_array_equal(rp2.cpu().numpy().astype(np.int64), ref_rp)
+    np.testing.assert_array_equal(ci2.cpu().numpy(), ref_ci)

@@ -13,6 +13,8 @@ from .ep_oracle import (  # noqa: F401
     reorder,
     graph_bandwidth,
     relabel_graph,
+    migrate,
+    balance,
     permute_rows,
     num_threads,
     set_num_threads,

@@ -7,6 +7,7 @@
  *   - the partition-ordered vertex permutation   (Section 4.5.1, "Adapting EmbedPart for Reordering")
  *   - the average graph bandwidth of a numbering (Section 4.5.1, Eq. 3, Eq. 4 and Eq. 5)
  *   - the graph and the embedding rows stored under the new numbering (Section 4.5.1)
+ *   - the migration policy that balances the partitions (Algorithm 4, used by Algorithm 3 lines 4-12)
  *
  * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call
  * this file.  It shares no code, header, table or helper with the CUDA library
@@ -269,4 +270,69 @@ void oracle_permute_rows(const float *emb, int64_t N, int32_t d, const int32_t *
 {
     for (int64_t i = 0; i < N; ++i)
         memcpy(out + (size_t)i * d, emb + (size_t)perm[i] * d, sizeof(float) * (size_t)d);
+}
+
+/*
+ * One application of the migration policy M(P, S, C) (Algorithm 4): random migration in
+ * proportion to free capacity.
+ *
+ *   member[v] != 0   v belongs to the candidate set S (NULL: every vertex does)
+ *   capacity         C, the same for every partition (Algorithm 3 passes beta |S| / k)
+ *   rand_words[v]    the random number that vertex v uses if it is moved (uniform 32-bit words,
+ *                    an input so that nothing here draws numbers)
+ *
+ * Steps, as the algorithm lists them: loads L_i = |{v in S : P(v) = i}|; overloaded O = {L_i > C},
+ * underloaded U = {L_i < C}; free capacity f_i = C - L_i on U, F = their sum; from every i in O
+ * the m_i = L_i - C vertices of S with the smallest degree are taken (equal degrees: the smaller
+ * vertex id first; the degree is the row length); a taken vertex v goes to the partition of U
+ * that the number t = floor(rand_words[v] * F / 2^32) falls into when the f_j of U are laid end to
+ * end in ascending partition order, i.e. j is drawn with probability f_j / F.  Loads and
+ * probabilities are those from before the first move.
+ * Returns the number of vertices moved, -1 when there are overloaded partitions but no free
+ * capacity, -2 when scratch memory cannot be had.
+ */
+typedef struct { int64_t deg; int64_t v; } oracle_deg_id;
+
+static int oracle_deg_id_less(const void *a, const void *b)
+{
+    const oracle_deg_id *x = (const oracle_deg_id *)a, *y = (const oracle_deg_id *)b;
+    if (x->deg != y->deg) return x->deg < y->deg ? -1 : 1;
+    return x->v < y->v ? -1 : (x->v > y->v ? 1 : 0);
+}
+
+int64_t oracle_migrate(const int64_t *rowptr, int64_t N, int32_t K, const uint8_t *member, int64_t capacity,
+                       const uint32_t *rand_words, int32_t *assign)
+{
+    int64_t *load = (int64_t *)calloc((size_t)K, sizeof(int64_t));
+    int64_t *cum = (int64_t *)calloc((size_t)K, sizeof(int64_t));     /* free capacity of U up to and including j */
+    oracle_deg_id *cand = (oracle_deg_id *)malloc(sizeof(oracle_deg_id) * (size_t)(N > 0 ? N : 1));
+    if (!load || !cum || !cand) { free(load); free(cum); free(cand); return -2; }
+    for (int64_t v = 0; v < N; ++v)
+        if (!member || member[v]) load[assign[v]] += 1;
+    int64_t F = 0, over = 0;
+    for (int32_t j = 0; j < K; ++j) {
+        if (load[j] < capacity) F += capacity - load[j];
+        if (load[j] > capacity) over += load[j] - capacity;
+        cum[j] = F;
+    }
+    int64_t moved = 0;
+    if (over > 0 && F == 0) moved = -1;
+    for (int32_t i = 0; i < K && moved >= 0; ++i) {
+        if (load[i] <= capacity) continue;
+        const int64_t m = load[i] - capacity;
+        int64_t n = 0;
+        for (int64_t v = 0; v < N; ++v)
+            if ((!member || member[v]) && assign[v] == i) { cand[n].deg = rowptr[v + 1] - rowptr[v]; cand[n].v = v; ++n; }
+        qsort(cand, (size_t)n, sizeof(oracle_deg_id), oracle_deg_id_less);
+        for (int64_t s = 0; s < m; ++s) {
+            const int64_t v = cand[s].v;
+            const uint64_t t = ((uint64_t)rand_words[v] * (uint64_t)F) >> 32;
+            int32_t j = 0;
+            while ((uint64_t)cum[j] <= t) ++j;               /* first partition whose cumulative capacity exceeds t */
+            assign[v] = j;
+            ++moved;
+        }
+    }
+    free(load); free(cum); free(cand);
+    return moved;
 }

@@ -46,6 +46,8 @@ def _load():
         lib.oracle_reorder.restype = ctypes.c_int
         lib.oracle_graph_bandwidth.argtypes = [p, p, p, ctypes.c_int64, p, p]
         lib.oracle_graph_bandwidth.restype = None
+        lib.oracle_migrate.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, ctypes.c_int64, p, p]
+        lib.oracle_migrate.restype = ctypes.c_int64
         lib.oracle_relabel_graph.argtypes = [p, p, p, p, ctypes.c_int64, p, p]
         lib.oracle_relabel_graph.restype = None
         lib.oracle_permute_rows.argtypes = [p, ctypes.c_int64, ctypes.c_int32, p, p]
@@ -246,3 +248,41 @@ def permute_rows(emb, perm):
     out = np.empty_like(emb)
     _load().oracle_permute_rows(_ptr(emb), N, d, _ptr(perm), _ptr(out))
     return out
+
+
+def migrate(rowptr, assign, K: int, capacity: int, rand_words, member=None):
+    """One application of the migration policy (Algorithm 4): (new assign, vertices moved).
+    rand_words: one uint32 per vertex; member: boolean mask of the candidate set (None = all)."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    N = rowptr.shape[0] - 1
+    out = _labels(assign, N, K).copy()
+    rw = np.ascontiguousarray(rand_words, dtype=np.uint32)
+    if rw.shape != (N,):
+        raise ValueError("rand_words must have one entry per vertex")
+    mem = None if member is None else np.ascontiguousarray(member, dtype=np.uint8)
+    if mem is not None and mem.shape != (N,):
+        raise ValueError("member must have one entry per vertex")
+    if capacity < 0 or np.any(np.diff(rowptr) < 0):
+        raise ValueError("bad capacity or row pointer")
+    moved = int(_load().oracle_migrate(_ptr(rowptr), N, K, _ptr(mem), int(capacity), _ptr(rw), _ptr(out)))
+    if moved == -1:
+        raise ValueError("overloaded partitions but no free capacity: capacity * K < |S|")
+    if moved < 0:
+        raise MemoryError("oracle_migrate")
+    return out, moved
+
+
+def balance(rowptr, assign, K: int, capacity: int, rand_rounds, member=None):
+    """The loop of Algorithm 3 for one vertex set: apply the migration policy, each round with the next row
+    of rand_rounds, while any partition holds more than `capacity` vertices of the set.
+    Returns (assign, rounds used)."""
+    rand_rounds = np.ascontiguousarray(rand_rounds, dtype=np.uint32)
+    out = np.ascontiguousarray(assign, dtype=np.int32)
+    sel = slice(None) if member is None else np.asarray(member, dtype=bool)
+    rounds = 0
+    while np.bincount(out[sel], minlength=K).max(initial=0) > capacity:
+        if rounds == rand_rounds.shape[0]:
+            raise RuntimeError("not balanced within the given rounds")
+        out, _ = migrate(rowptr, out, K, capacity, rand_rounds[rounds], member)
+        rounds += 1
+    return out, rounds

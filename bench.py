@@ -473,6 +473,41 @@ def main():
                                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
                                                    "frac": gbs / hbm, "traffic": None, "peak_source": peaks["_source"]}}
 
+    # ---- outside the step: the K-Means partition balanced to beta = 1.05 (Algorithm 3 lines 4-12 for one
+    # vertex set = all vertices; random words from torch, an input of the library)
+    if last is not None and w.K <= 1024:
+        deg = x["rowptr"][1:] - x["rowptr"][:-1]
+        max_deg = int(deg.max().item())
+        cap = int(1.05 * w.N / w.K)
+        gen = torch.Generator(device=device).manual_seed(w.seed & 0x7FFFFFFF)
+        words = torch.randint(-2 ** 31, 2 ** 31, (8, w.N), generator=gen, device=device, dtype=torch.int64).to(torch.int32)
+        if w.K * (max_deg + 1) < 2 ** 30:
+            labels = last[0].assign.clone()
+            ctx.balance(x["rowptr"], labels, w.K, cap, max_deg, words)
+            reps = 3
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            total_rounds = 0
+            ms_b = 0.0
+            for _ in range(reps):
+                labels.copy_(last[0].assign)
+                torch.cuda.synchronize()
+                e0.record()
+                total_rounds += ctx.balance(x["rowptr"], labels, w.K, cap, max_deg, words)
+                e1.record()
+                torch.cuda.synchronize()
+                ms_b += e0.elapsed_time(e1)
+            ctx.check()
+            q_after = ctx.partition_quality(x["rowptr"], x["colidx"], labels, w.K)
+            q_before = ctx.partition_quality(x["rowptr"], x["colidx"], last[0].assign, w.K)
+            torch.cuda.synchronize()
+            extras["balance"] = {"ms_per_call": ms_b / reps, "applications_of_the_policy": total_rounds / reps,
+                                 "beta": 1.05, "K": w.K,
+                                 "vertex_balance_before": float(q_before.part_vertices.max().item()) / (w.N / w.K),
+                                 "vertex_balance_after": float(q_after.part_vertices.max().item()) / (w.N / w.K),
+                                 "edge_cut_ratio_before": int(q_before.edge_cut.item()) / max(nnz, 1),
+                                 "edge_cut_ratio_after": int(q_after.edge_cut.item()) / max(nnz, 1)}
+        del words
+
     # ---- outside the step: sampling-based clustering as the paper ran it (2^9 rows per cluster train the
     # centroids, then one pass labels every row)
     M = min(w.N, 512 * w.K)

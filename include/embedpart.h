@@ -72,7 +72,8 @@ enum {
     EP_TIMER_KMEANS_RESOLVE = 5, /* tensor-core path: the fp32 kernel that decides the labels */
     EP_TIMER_GRAPH_BANDWIDTH = 6, /* all kernels of ep_graph_bandwidth */
     EP_TIMER_RELABEL = 7,        /* all kernels of ep_relabel_graph and ep_permute_rows */
-    EP_TIMER_COUNT = 8
+    EP_TIMER_BALANCE = 8,        /* the kernels of ep_migrate / ep_balance other than the sort */
+    EP_TIMER_COUNT = 9
 };
 
 typedef struct ep_ctx ep_ctx; /* opaque: device id, device properties, device status word, options */
@@ -249,6 +250,43 @@ int ep_relabel_graph(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, c
                      int32_t *new_colidx, void *workspace, size_t workspace_bytes, void *cuda_stream);
 int ep_permute_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const int32_t *perm, float *out,
                     void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
+ * ep_migrate, ep_balance -- the migration policy M(P, S, C) (Algorithm 4: random migration in
+ * proportion to free capacity) and the loop of Algorithm 3 (lines 4-12) that applies it to one
+ * vertex set until no partition holds more than C vertices of the set.  Algorithm 3 runs the
+ * loop three times (training, validation and remaining vertices): three calls with three masks.
+ *
+ * One application: loads L_i = |{v in S : assign[v] = i}|; from every partition with L_i > C
+ * the L_i - C vertices of S with the smallest degree leave (the degree is the row length; equal
+ * degrees: the lower vertex id first); each goes to a partition with L_j < C, drawn with
+ * probability (C - L_j) / F, F the total free capacity: vertex v goes to the partition whose
+ * stretch holds t = floor(rand_words[v] * F / 2^32) when the free capacities are laid end to end
+ * in ascending partition order.  Loads and probabilities are those from before the first move.
+ * Random words are an input; the library draws no numbers.
+ *
+ *   rowptr      [dev] N+1 row offsets (int32 or int64), only the row lengths are used
+ *   N, K        1 <= N < 2^31;  1 <= K <= 1024
+ *   member      [dev] N bytes, non-zero = the vertex belongs to S; NULL = every vertex does
+ *   capacity    C >= 0, the same for every partition (Algorithm 3 passes floor(beta |S| / K))
+ *   max_degree  an upper bound of the row lengths; K * (max_degree + 1) must stay below 2^30
+ *               (EP_ERR_UNSUPPORTED otherwise); a longer row raises EP_ERR_BAD_INDEX and its vertex stays
+ *   rand_words  [dev] N uint32 (ep_migrate), max_rounds x N uint32, one row per round (ep_balance)
+ *   assign      [dev] in/out, N int32 labels in [0, K)
+ *   state       [dev] out or NULL, 4 int64: [0] vertices above capacity before the call, [1] F,
+ *               [2] vertices moved, or -1 when there is no free capacity to move them to, [3] 0
+ * ep_migrate is asynchronous like the other calls.  ep_balance synchronises the stream after every
+ * round (it has to know whether another one is needed), stops as soon as no partition is above C,
+ * writes the number of applications to *rounds_used [host] and returns EP_ERR_INVALID_ARG when C * K is
+ * too small to hold S, EP_ERR_UNSUPPORTED when max_rounds applications were not enough.
+ */
+size_t ep_balance_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t K, int64_t max_degree);
+int ep_migrate(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t N, int32_t K, const uint8_t *member,
+               int64_t capacity, int64_t max_degree, const uint32_t *rand_words, int32_t *assign, int64_t *state,
+               void *workspace, size_t workspace_bytes, void *cuda_stream);
+int ep_balance(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t N, int32_t K, const uint8_t *member,
+               int64_t capacity, int64_t max_degree, const uint32_t *rand_words, int32_t max_rounds, int32_t *assign,
+               int32_t *rounds_used, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
  * Host-buffer variants.  Same operations and the same kernels; inputs and outputs are [host]

@@ -20,6 +20,7 @@ EXPORTED_SYMBOLS = (
     "ep_graph_bandwidth_workspace_bytes", "ep_graph_bandwidth", "ep_graph_bandwidth_host_arena_bytes",
     "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
     "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
+    "ep_balance_workspace_bytes", "ep_migrate", "ep_balance",
 )
 
 EP_OK = 0
@@ -27,9 +28,9 @@ EP_OPT_KMEANS_PATH = 1
 EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
 EP_OPT_KMEANS_CAND_MB = 4
-TIMER_COUNT = 8
+TIMER_COUNT = 9
 TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
-          "kmeans_resolve": 5, "graph_bandwidth": 6, "relabel": 7}
+          "kmeans_resolve": 5, "graph_bandwidth": 6, "relabel": 7, "balance": 8}
 KMEANS_PATHS = {"auto": 0, "simt": 1, "tensor": 2}
 
 
@@ -112,6 +113,12 @@ def load_library() -> ctypes.CDLL:
             lib.ep_kmeans_sampled.restype = ctypes.c_int
             lib.ep_gather_rows.argtypes = [vp, vp, i64, i32, vp, i64, vp, vp]
             lib.ep_gather_rows.restype = ctypes.c_int
+            lib.ep_balance_workspace_bytes.argtypes = [vp, i64, i32, i64]
+            lib.ep_balance_workspace_bytes.restype = sz
+            lib.ep_migrate.argtypes = [vp, vp, i32, i64, i32, vp, i64, i64, vp, vp, vp, vp, sz, vp]
+            lib.ep_migrate.restype = ctypes.c_int
+            lib.ep_balance.argtypes = [vp, vp, i32, i64, i32, vp, i64, i64, vp, i32, vp, vp, vp, sz, vp]
+            lib.ep_balance.restype = ctypes.c_int
             lib.ep_relabel_graph_workspace_bytes.argtypes = [vp, i64, i64]
             lib.ep_relabel_graph_workspace_bytes.restype = sz
             lib.ep_relabel_graph.argtypes = [vp, vp, i32, vp, i64, vp, vp, i64, vp, vp, vp, sz, vp]
@@ -331,6 +338,53 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return ReorderResult(perm, inv)
+
+    def _balance_args(self, rowptr, assign, K, max_degree, member):
+        if rowptr.dtype not in (torch.int32, torch.int64):
+            raise ValueError("rowptr must be int32 or int64")
+        rowptr = _check_cuda(rowptr, rowptr.dtype, "rowptr", self.device)
+        assign = _check_cuda(assign, torch.int32, "assign", self.device)
+        if member is not None:
+            member = _check_cuda(member, torch.uint8, "member", self.device)
+        N = assign.numel()
+        if rowptr.numel() != N + 1 or (member is not None and member.numel() != N):
+            raise ValueError("rowptr must have N + 1 entries, member N")
+        need = self._lib.ep_balance_workspace_bytes(self._h, N, K, max_degree)
+        if need == 0:
+            raise EmbedPartError(5, f"unsupported shape: N={N} K={K} max_degree={max_degree}")
+        return rowptr, assign, member, N, self.workspace(need)
+
+    def migrate(self, rowptr, assign, K: int, capacity: int, max_degree: int, rand_words, member=None):
+        """One application of the migration policy (Algorithm 4), in place on `assign`; returns the int64 state
+        tensor [vertices above capacity before, free capacity, vertices moved or -1, 0]."""
+        rowptr, assign, member, N, ws = self._balance_args(rowptr, assign, K, max_degree, member)
+        rand_words = _check_cuda(rand_words, torch.int32, "rand_words", self.device)   # 32 random bits per vertex
+        if rand_words.numel() != N:
+            raise ValueError("rand_words must have N entries")
+        state = torch.zeros(4, dtype=torch.int64, device=self.device)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_migrate(self._h, _dev_ptr(rowptr), int(rowptr.dtype == torch.int64), N, K, _dev_ptr(member),
+                                      capacity, max_degree, _dev_ptr(rand_words), _dev_ptr(assign), _dev_ptr(state),
+                                      _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return state
+
+    def balance(self, rowptr, assign, K: int, capacity: int, max_degree: int, rand_rounds, member=None):
+        """The loop of Algorithm 3 for one vertex set, in place on `assign`; rand_rounds is [max_rounds, N] int32
+        (32 random bits each).  Returns the number of applications of the policy.  Synchronises the stream."""
+        rowptr, assign, member, N, ws = self._balance_args(rowptr, assign, K, max_degree, member)
+        rand_rounds = _check_cuda(rand_rounds, torch.int32, "rand_rounds", self.device)
+        if rand_rounds.dim() != 2 or rand_rounds.shape[1] != N:
+            raise ValueError("rand_rounds must be [max_rounds, N]")
+        used = ctypes.c_int32(0)
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_balance(self._h, _dev_ptr(rowptr), int(rowptr.dtype == torch.int64), N, K, _dev_ptr(member),
+                                      capacity, max_degree, _dev_ptr(rand_rounds), rand_rounds.shape[0], _dev_ptr(assign),
+                                      ctypes.byref(used), _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return used.value
 
     def relabel_graph(self, rowptr, colidx, perm, inv_perm):
         """(new_rowptr, new_colidx): the CSR graph with vertex perm[i] renamed i."""

@@ -465,6 +465,71 @@ int ep_permute_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const i
     return permute_rows_run(ctx, emb, N, d, perm, out, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---------------------------------------------------------------------------------------------- balance
+size_t ep_balance_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t K, int64_t max_degree) {
+    if (!ctx || !balance_shape_ok(N, K, max_degree)) return 0;
+    return balance_workspace_bytes(N, K, max_degree);
+}
+
+static int balance_check_args(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t N, int32_t K,
+                              int64_t capacity, int64_t max_degree, const int32_t *assign, void *workspace,
+                              size_t workspace_bytes) {
+    if (N < 1 || N >= (int64_t(1) << 31) || K < 1 || max_degree < 0 || capacity < 0)
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld K=%d max_degree=%lld capacity=%lld", (long long)N, K,
+                    (long long)max_degree, (long long)capacity);
+    if (!balance_shape_ok(N, K, max_degree))
+        return fail(ctx, EP_ERR_UNSUPPORTED, "K=%d with max_degree=%lld: K <= 1024 and K * (max_degree + 1) < 2^30 are required",
+                    K, (long long)max_degree);
+    if (!rowptr || !assign) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (!aligned(rowptr, rowptr_is_int64 ? 8 : 4) || !aligned(assign, 4)) return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
+    const size_t need = balance_workspace_bytes(N, K, max_degree);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "balance workspace: need %zu bytes, 256-byte aligned", need);
+    return EP_OK;
+}
+
+int ep_migrate(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t N, int32_t K, const uint8_t *member,
+               int64_t capacity, int64_t max_degree, const uint32_t *rand_words, int32_t *assign, int64_t *state,
+               void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    int rc = balance_check_args(ctx, rowptr, rowptr_is_int64, N, K, capacity, max_degree, assign, workspace, workspace_bytes);
+    if (rc != EP_OK) return rc;
+    if (!rand_words || !aligned(rand_words, 4) || (state && !aligned(state, 8)))
+        return fail(ctx, EP_ERR_INVALID_ARG, "rand_words is null, or a pointer is misaligned");
+    DeviceGuard g(ctx->device);
+    return migrate_run(ctx, rowptr, rowptr_is_int64 != 0, N, K, member, capacity, max_degree, rand_words, assign,
+                       reinterpret_cast<long long *>(state), workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ep_balance(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t N, int32_t K, const uint8_t *member,
+               int64_t capacity, int64_t max_degree, const uint32_t *rand_words, int32_t max_rounds, int32_t *assign,
+               int32_t *rounds_used, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    int rc = balance_check_args(ctx, rowptr, rowptr_is_int64, N, K, capacity, max_degree, assign, workspace, workspace_bytes);
+    if (rc != EP_OK) return rc;
+    if (max_rounds < 0 || (max_rounds > 0 && (!rand_words || !aligned(rand_words, 4))))
+        return fail(ctx, EP_ERR_INVALID_ARG, "max_rounds < 0, or rand_words is null or misaligned");
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const long long *d_state = balance_state_ptr(N, K, max_degree, workspace);
+    if (rounds_used) *rounds_used = 0;
+    for (int r = 0;; ++r) {
+        // after the last allowed application only the loads are looked at
+        const uint32_t *words = r < max_rounds ? rand_words + (size_t)r * (size_t)N : nullptr;
+        rc = migrate_run(ctx, rowptr, rowptr_is_int64 != 0, N, K, member, capacity, max_degree, words, assign, nullptr,
+                         workspace, st);
+        if (rc != EP_OK) return rc;
+        long long state[4];
+        EP_CUDA(ctx, cudaMemcpyAsync(state, d_state, sizeof(state), cudaMemcpyDeviceToHost, st));
+        EP_CUDA(ctx, cudaStreamSynchronize(st));
+        if (state[0] == 0) return EP_OK;                                  // no partition above its capacity
+        if (state[2] < 0)
+            return fail(ctx, EP_ERR_INVALID_ARG, "capacity %lld x K=%d cannot hold the vertex set", (long long)capacity, K);
+        if (!words) return fail(ctx, EP_ERR_UNSUPPORTED, "not balanced after %d applications of the policy", max_rounds);
+        if (rounds_used) *rounds_used = r + 1;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------- reorder
 static bool reorder_shape_ok(int64_t N, int32_t K) {
     return N >= 1 && N < (int64_t(1) << 31) && K >= 1 && K <= (1 << 24);

@@ -153,6 +153,14 @@ int relabel_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, const int32_t *c
 int permute_rows_run(ep_ctx *ctx, const float *emb, int64_t N, int d, const int32_t *perm, float *out,
                      cudaStream_t stream);
 
+// ---- migration policy and balancing loop (balance.cu) ----------------------------------------------
+bool balance_shape_ok(int64_t N, int K, int64_t max_degree);
+size_t balance_workspace_bytes(int64_t N, int K, int64_t max_degree);
+int migrate_run(ep_ctx *ctx, const void *rowptr, bool rowptr64, int64_t N, int K, const uint8_t *member, int64_t capacity,
+                int64_t max_degree, const uint32_t *rand_words, int32_t *assign, long long *state_out, void *workspace,
+                cudaStream_t stream);
+const long long *balance_state_ptr(int64_t N, int K, int64_t max_degree, void *workspace);
+
 }  // namespace ep
 
 // ---- device helpers -------------------------------------------------------------------------------

@@ -120,3 +120,14 @@ def test_cfg4_graph_passes_full_size(ctx, cfg4):
     ref_rp, ref_ci = oracle.relabel_graph(rowptr.cpu().numpy(), colidx.cpu().numpy(), perm, inv)
     np.testing.assert_array_equal(rp2.cpu().numpy().astype(np.int64), ref_rp)
     np.testing.assert_array_equal(ci2.cpu().numpy(), ref_ci)
+    # one application of the migration policy (Algorithm 4) to the K=32 partition at full size
+    deg = np.diff(rowptr.cpu().numpy().astype(np.int64))
+    cap = int(1.05 * w.N / w.K)
+    words = torch.randint(-2 ** 31, 2 ** 31, (w.N,), generator=torch.Generator().manual_seed(5), dtype=torch.int64).to(torch.int32)
+    moved_labels = km.assign.clone()
+    state = ctx.migrate(rowptr, moved_labels, w.K, cap, int(deg.max()), words.cuda())
+    torch.cuda.synchronize()
+    ctx.check()
+    ref_labels, ref_moved = oracle.migrate(rowptr.cpu().numpy(), a, w.K, cap, words.numpy().view(np.uint32))
+    np.testing.assert_array_equal(moved_labels.cpu().numpy(), ref_labels)
+    assert int(state[2].item()) == ref_moved

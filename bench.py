@@ -473,7 +473,7 @@ def main():
                                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
                                                    "frac": gbs / hbm, "traffic": None, "peak_source": peaks["_source"]}}
 
-    # ---- outside the step: the K-Means partition balanced to beta = 1.05 (Algorithm 3 lines 4-12 for one
+    # ---- outside the step: the K-Means partition balanced to beta = 1.05 (the balancing loop of Algorithm 3 for one
     # vertex set = all vertices; random words from torch, an input of the library)
     if last is not None and w.K <= 1024:
         deg = x["rowptr"][1:] - x["rowptr"][:-1]

@@ -3,7 +3,7 @@
  * embedding-driven graph partitioning:
  *
  *   ep_kmeans             Lloyd K-Means over dense node embeddings -> partition of every vertex
- *                         (Algorithm 3, line 1:  P <- KMeans(E, k))
+ *                         (Algorithm 3, the clustering step P <- KMeans(E, k))
  *   ep_partition_quality  edge cut and per-partition loads of a partition over a CSR graph
  *                         (Section 2.1.1, Eq. 1 "edge-cut ratio" and Eq. 2 "vertex balance")
  *   ep_reorder            partition-ordered vertex relabelling for graph reordering
@@ -106,7 +106,7 @@ int64_t ep_launch_count(const ep_ctx *ctx);
 int ep_debug_counters(ep_ctx *ctx, int64_t *out);
 
 /* --------------------------------------------------------------------------------------------
- * ep_kmeans -- Lloyd K-Means (Algorithm 3, line 1).
+ * ep_kmeans -- Lloyd K-Means (Algorithm 3, the clustering step).
  *
  * Squared Euclidean distance; exactly `iters` iterations from the given initial centroids, no
  * early stop.  In iteration t every row is assigned to its nearest centroid of C_{t-1} (of several
@@ -253,7 +253,7 @@ int ep_permute_rows(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, const i
 
 /* --------------------------------------------------------------------------------------------
  * ep_migrate, ep_balance -- the migration policy M(P, S, C) (Algorithm 4: random migration in
- * proportion to free capacity) and the loop of Algorithm 3 (lines 4-12) that applies it to one
+ * proportion to free capacity) and the balancing loop of Algorithm 3 that applies it to one
  * vertex set until no partition holds more than C vertices of the set.  Algorithm 3 runs the
  * loop three times (training, validation and remaining vertices): three calls with three masks.
  *

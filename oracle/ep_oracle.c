@@ -2,12 +2,12 @@
  * ep_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
  *
  * A plain, slow, fp64 CPU statement of what the EmbedPart hot path computes:
- *   - Lloyd K-Means over dense node embeddings  (Algorithm 3, line 1: P <- KMeans(E, k))
+ *   - Lloyd K-Means over dense node embeddings  (Algorithm 3, the clustering step P <- KMeans(E, k))
  *   - edge cut and per-partition loads           (Section 2.1.1, Eq. 1 and Eq. 2)
  *   - the partition-ordered vertex permutation   (Section 4.5.1, "Adapting EmbedPart for Reordering")
  *   - the average graph bandwidth of a numbering (Section 4.5.1, Eq. 3, Eq. 4 and Eq. 5)
  *   - the graph and the embedding rows stored under the new numbering (Section 4.5.1)
- *   - the migration policy that balances the partitions (Algorithm 4, used by Algorithm 3 lines 4-12)
+ *   - the migration policy that balances the partitions (Algorithm 4, used by the balancing loops of Algorithm 3)
  *
  * Only tests, the smoke check and the CPU-baseline leg of the benchmark may call
  * this file.  It shares no code, header, table or helper with the CUDA library
@@ -90,7 +90,7 @@ void oracle_assign(const float *emb, int64_t N, int32_t d,
 }
 
 /*
- * Lloyd K-Means, exactly `iters` iterations, no early stop (Algorithm 3 line 1
+ * Lloyd K-Means, exactly `iters` iterations, no early stop (Algorithm 3, the clustering step
  * under the reading: squared Euclidean distance, explicit initial centroids,
  * full batch).
  *

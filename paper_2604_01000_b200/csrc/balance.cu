@@ -1,5 +1,5 @@
-// Migration policy M(P, S, C) (Algorithm 4: random migration in proportion to free capacity) and the loop of
-// Algorithm 3 (lines 4-12) that applies it to one vertex set until no partition is above its capacity.
+// Migration policy M(P, S, C) (Algorithm 4: random migration in proportion to free capacity) and the balancing
+// loop of Algorithm 3 that applies it to one vertex set until no partition is above its capacity.
 //
 // One application, all on the device:
 //   loads     L_i = |{v in S : P(v) = i}| (block-local counts, then integer atomics);

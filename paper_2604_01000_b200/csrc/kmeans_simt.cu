@@ -1,4 +1,4 @@
-// Lloyd K-Means on CUDA cores (Algorithm 3, line 1): the assign-and-accumulate pass, the centroid
+// Lloyd K-Means on CUDA cores (Algorithm 3, the clustering step): the assign-and-accumulate pass, the centroid
 // update and the per-call driver.  A warp owns whole rows; lane l holds the 16-byte slices
 // l, l+32, ... of a row in registers, so a row is read from HBM exactly once, coalesced.
 #include "ep_common.cuh"

@@ -1,4 +1,4 @@
-// Tensor-core assignment step of Lloyd K-Means (Algorithm 3, line 1) for many centroids.
+// Tensor-core assignment step of Lloyd K-Means (Algorithm 3, the clustering step) for many centroids.
 //
 // The scores |c_k|^2 - 2 x_i.c_k of a tile of 128 rows against all K centroids are a dense
 // contraction [128 x d].[d x K].  kmeans_tc_screen runs it on the 5th-generation tensor cores in TF32:

@@ -1,4 +1,4 @@
-// Fused assign-and-accumulate pass of Lloyd K-Means (Algorithm 3, line 1) for few centroids
+// Fused assign-and-accumulate pass of Lloyd K-Means (Algorithm 3, the clustering step) for few centroids
 // (K <= 64, d <= 128) on the tensor cores: one read of the embedding matrix per iteration.
 //
 // kmeans_tc_fused: a persistent block per SM streams 128-row tiles of X through a ring of shared-memory

@@ -1,4 +1,4 @@
-"""GPU parity: ep_migrate / ep_balance (Algorithm 4 and the loop of Algorithm 3, lines 4-12) against the
+"""GPU parity: ep_migrate / ep_balance (Algorithm 4 and the balancing loop of Algorithm 3) against the
 oracle, bit for bit; the random words are inputs to both."""
 import numpy as np
 import pytest

@@ -1,4 +1,4 @@
-"""Pins for the oracle's migration policy (Algorithm 4) and balancing loop (Algorithm 3, lines 4-12); CPU only."""
+"""Pins for the oracle's migration policy (Algorithm 4) and balancing loop (Algorithm 3); CPU only."""
 import numpy as np
 import pytest
 

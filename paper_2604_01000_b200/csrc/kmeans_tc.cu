@@ -61,8 +61,8 @@ struct TcShared {
 // ~(GROUP - 1); it arrives as an argument so that clearing the index bits and inserting the (compile-
 // time) index stay one three-input logic operation instead of two with an immediate each.
 // A row with a single centroid inside the allowance (see screen_allowance) gets assign[r] here; every
-// other row is appended to slow_list (row numbers, any order) and counted in *slow_count, which the caller
-// has zeroed.  counters, when given, receives the number of rows screened in word 0.
+// other row is appended to slow_list (row number and the centroid with the smallest key, any order) and counted
+// in *slow_count, which the caller has zeroed.  counters, when given, receives the number of rows screened in word 0.
 // CN_SMEM: all of cn is first copied behind the barriers in shared memory (the host checks that it fits).
 template <bool CN_SMEM>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -70,7 +70,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                  const float *__restrict__ cn, int64_t row_begin, int64_t row_end, int num_kb, int num_nt, int stages,
                  int G, uint32_t key_mask, int d, int K, const float *__restrict__ cmaxima,
                  const float2 *__restrict__ rownorm, uint2 *__restrict__ cand, int32_t *__restrict__ assign,
-                 int32_t *__restrict__ slow_list, int *__restrict__ slow_count, unsigned long long *counters,
+                 int2 *__restrict__ slow_list, int *__restrict__ slow_count, unsigned long long *counters,
                  int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -273,7 +273,8 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     int base = 0;
                     if (lane == 0) base = atomicAdd(slow_count, __popc(slow));
                     base = __shfl_sync(FULL, base, 0);
-                    if (live && !fast) slow_list[base + __popc(slow & ((1u << lane) - 1u))] = (int32_t)(row - row_begin);
+                    if (live && !fast)
+                        slow_list[base + __popc(slow & ((1u << lane) - 1u))] = make_int2((int)(row - row_begin), kone);
                 }
             }
         }
@@ -326,9 +327,15 @@ __global__ void __launch_bounds__(1024) centroid_maxima(const float *__restrict_
     }
 }
 
-// Exact fp32 decision for the rows the screening pass listed (slow_list holds row numbers relative to
-// row_begin, *slow_count of them).  One warp per row; lane l holds the 16-byte slices l, l+32, ... of the
-// row, as in the CUDA-core kernels.  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|), computed once per call.
+// Exact fp32 decision for the rows the screening pass listed (slow_list holds the row number relative to
+// row_begin and the centroid with the row's smallest key, *slow_count entries).  One warp per row; lane l holds
+// the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.  rownorm[i] = (|x_i|,
+// |x_i - trunc_tf32(x_i)|), computed once per call.
+//
+// The listed centroid is scored first (its row of C comes with the prefetch of the row).  With `best` its fp32
+// score and E the allowance, a centroid h can only reach or tie the final fp32 minimum if its key is at most
+// best + E (key(h) <= f(h) + E <= best + E): that threshold, never larger than the screening pass's own
+// (smallest key + 2E), decides which other centroids are scored and which groups are scanned.
 template <int VPL>
 __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin, int rows, int d, int K,
                                                          int G, const float *__restrict__ C,
@@ -336,7 +343,7 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                                                          const float *__restrict__ cmaxima,
                                                          const float2 *__restrict__ rownorm,
                                                          const uint2 *__restrict__ cand,
-                                                         const int32_t *__restrict__ slow_list,
+                                                         const int2 *__restrict__ slow_list,
                                                          const int *__restrict__ slow_count,
                                                          int32_t *__restrict__ assign, unsigned long long *counters) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
@@ -346,60 +353,84 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
     const float4 *C4 = reinterpret_cast<const float4 *>(C);
     const int slot = lane_chunk_slot(lane);
     const int n_slow = min(*slow_count, rows);            // the list never holds more than the chunk's rows
-    auto entry = [&](int64_t i) { return i < n_slow ? min(max(slow_list[i], 0), rows - 1) : -1; };
+    auto entry = [&](int64_t i) {
+        int2 e = make_int2(-1, -1);
+        if (i < n_slow) {
+            e = slow_list[i];
+            e.x = min(max(e.x, 0), rows - 1);
+        }
+        return e;
+    };
 
-    // Each warp fetches its next row (keys, norms, the row itself) while it works on the current one, and
-    // the list entry after that.
+    // Each warp fetches its next row (keys, norms, the row itself, the first centroid) while it works on the
+    // current one, and the list entry after that.
     const int stride = (int)gridDim.x * 8;
     uint2 key_n = make_uint2(KEY_INIT, KEY_INIT);
     float2 nr_n = make_float2(0.f, 0.f);
-    float4 x_n[VPL];
-    auto fetch = [&](int rel) {
-        if (rel >= 0) {
-            const int64_t r = row_begin + rel;
-            if (lane < G) key_n = cand[(size_t)rel * G + lane];
+    float4 x_n[VPL], c_n[VPL];
+    float cn_n = 0.f;
+    auto fetch = [&](int2 e) {
+        if (e.x >= 0) {
+            const int64_t r = row_begin + e.x;
+            if (lane < G) key_n = cand[(size_t)e.x * G + lane];
             nr_n = __ldg(rownorm + r);
+            const int kf = (unsigned)e.y < (unsigned)K ? e.y : 0;
+            cn_n = __ldg(cn + kf);
 #pragma unroll
             for (int v = 0; v < VPL; ++v) {
                 const int q = lane + 32 * v;
                 x_n[v] = q < d4 ? ldg_stream(reinterpret_cast<const float4 *>(emb) + r * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                c_n[v] = q < d4 ? __ldg(C4 + (size_t)kf * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
     };
     const int first = (int)blockIdx.x * 8 + warp;
-    int rel = entry(first);
-    int rel_n = entry((int64_t)first + stride);
-    fetch(rel);
+    int2 ent = entry(first);
+    int2 ent_n = entry((int64_t)first + stride);
+    fetch(ent);
     for (int i = first; i < n_slow; i += stride) {
         ++n_rows;
+        const int rel = ent.x;
+        const int kfirst = (unsigned)ent.y < (unsigned)K ? ent.y : -1;   // -1: nothing usable was listed (a row of NaNs)
         const int64_t row = row_begin + rel;
         const uint2 *cr = cand + (size_t)rel * G;
         const float2 nr = nr_n;
         const uint2 key0 = lane < G ? key_n : make_uint2(KEY_INIT, KEY_INIT);   // this lane's group of the first 32
         float4 x[VPL];
+        float acc_f = 0.f;
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) x[v] = x_n[v];
-        rel = rel_n;
-        rel_n = entry((int64_t)i + 2 * (int64_t)stride);
-        fetch(rel);
-        float lo = __uint_as_float(key0.x);
-        for (int g = lane + 32; g < G; g += 32) lo = fminf(lo, __uint_as_float(cr[g].x));
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
-        const float thr = lo + 2.f * screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
-
+        for (int v = 0; v < VPL; ++v) {
+            x[v] = x_n[v];
+            acc_f = dot4(x[v], c_n[v], acc_f);
+        }
+        const float cn_f = cn_n;
+        ent = ent_n;
+        ent_n = entry((int64_t)i + 2 * (int64_t)stride);
+        fetch(ent);
         float best = CUDART_INF_F;
         int bidx = 0x7fffffff;
+        if (kfirst >= 0) {
+            const float sf = fmaf(-2.f, warp_sum(acc_f), cn_f);
+            best = (sf == sf) ? sf : CUDART_INF_F;
+            bidx = kfirst;
+            ++n_single;
+        }
+        // nothing above this key can reach or tie `best`
+        const float thr = best + screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
+
         bool lanes_differ = false;                 // set once a lane holds a score the others do not
         for (int g0 = 0; g0 < G; g0 += 32) {
             const int g = g0 + lane;
             uint2 key = key0;
             if (g0 > 0) key = g < G ? cr[g] : make_uint2(KEY_INIT, KEY_INIT);
+            // the centroid scored above is the first key of its group: it is not scored again on its own
+            const bool is_first = kfirst >= 0 && g == (kfirst >> 7) && (int)(key.x & IDX_MASK) == (kfirst & (int)IDX_MASK);
             const unsigned m1 = __ballot_sync(FULL, __uint_as_float(key.x) <= thr);
             const unsigned mboth = __ballot_sync(FULL, __uint_as_float(key.y) <= thr);
+            const unsigned mfirst = __ballot_sync(FULL, is_first);
             // groups with one centroid inside the allowance: score those centroids (one or two of them is the
             // usual case: a plain warp sum each; more go eight per reduction)
-            unsigned ms = m1 & ~mboth;
+            unsigned ms = m1 & ~mboth & ~mfirst;
             if (__popc(ms) <= 4) {
                 while (ms) {   // two at a time: their loads and their reductions overlap
                     const int src0 = __ffs(ms) - 1;
@@ -592,7 +623,7 @@ int64_t kmeans_tc_chunk_rows(const ep_ctx *ctx, int64_t N, int K) {
 // Candidate keys of one chunk of rows, the chunk's list of undecided rows, and one list length per chunk.
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K) {
     const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
-    return (size_t)chunk * kmeans_tc_groups(K) * sizeof(uint2) + (size_t)chunk * sizeof(int32_t) +
+    return (size_t)chunk * kmeans_tc_groups(K) * sizeof(uint2) + (size_t)chunk * sizeof(int2) +
            (size_t)ceil_div(N, chunk) * sizeof(int);
 }
 
@@ -628,8 +659,8 @@ int kmeans_tc_assign(ep_ctx *ctx, const TcState &st, const float *emb, int64_t N
     const int64_t chunk = kmeans_tc_chunk_rows(ctx, N, K);
     const int64_t nchunks = ceil_div(N, chunk);
     uint2 *cand = static_cast<uint2 *>(cand_ws);
-    int32_t *slow_list = reinterpret_cast<int32_t *>(cand + (size_t)chunk * G);
-    int *slow_count = slow_list + chunk;                                // one counter per chunk
+    int2 *slow_list = reinterpret_cast<int2 *>(cand + (size_t)chunk * G);
+    int *slow_count = reinterpret_cast<int *>(slow_list + chunk);       // one counter per chunk
     unsigned long long *counters =
         ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
     {

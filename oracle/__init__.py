@@ -15,6 +15,7 @@ from .ep_oracle import (  # noqa: F401
     relabel_graph,
     migrate,
     balance,
+    cluster_and_balance,
     permute_rows,
     num_threads,
     set_num_threads,

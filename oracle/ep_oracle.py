@@ -286,3 +286,22 @@ def balance(rowptr, assign, K: int, capacity: int, rand_rounds, member=None):
         out, _ = migrate(rowptr, out, K, capacity, rand_rounds[rounds], member)
         rounds += 1
     return out, rounds
+
+
+def cluster_and_balance(emb, K: int, iters: int, init_centroids, rowptr, split, capacities, rand_rounds):
+    """Phase 2 as a whole (Algorithm 3): P <- KMeans(E, k), then the balancing loop for the training vertices,
+    then for the validation vertices, then for the remaining ones, each with its own capacity.
+
+    split[v] is 0 (training), 1 (validation) or 2 (rest); capacities = (C_train, C_val, C_rest);
+    rand_rounds[s] is the [max_rounds, N] array of random words of set s.
+    Returns (assign, centroids, rounds used per set)."""
+    split = np.ascontiguousarray(split, dtype=np.uint8)
+    km = kmeans(emb, K, iters, init_centroids)
+    if split.shape != (km.assign.shape[0],) or split.max(initial=0) > 2:
+        raise ValueError("split must hold 0, 1 or 2 for every vertex")
+    assign = km.assign
+    used = []
+    for s in range(3):
+        assign, r = balance(rowptr, assign, K, int(capacities[s]), rand_rounds[s], split == s)
+        used.append(r)
+    return assign, km.centroids, used

@@ -98,3 +98,28 @@ def test_balancing_loop_reaches_the_bound(seed):
     # migration prefers low degrees: the moved vertices have a lower mean degree than those that stayed
     moved = member & (out != assign)
     assert deg[moved].mean() < deg[member & ~moved].mean()
+
+
+def test_phase_two_as_a_whole():
+    """Algorithm 3: clustering, then the three balancing loops in the order training, validation, rest."""
+    rng = np.random.default_rng(77)
+    N, K, d = 3000, 6, 8
+    centres = rng.normal(size=(K, d)) * 4
+    z = rng.choice(K, size=N, p=[0.4, 0.25, 0.15, 0.1, 0.06, 0.04])
+    emb = (centres[z] + rng.normal(size=(N, d))).astype(np.float32)
+    deg = rng.integers(1, 30, size=N)
+    split = rng.choice(3, size=N, p=[0.5, 0.2, 0.3]).astype(np.uint8)
+    caps = [int(np.floor(1.05 * (split == s).sum() / K)) for s in range(3)]
+    words = rng.integers(0, 2 ** 32, size=(3, 10, N), dtype=np.uint64).astype(np.uint32)
+    init = emb[:K].copy()
+    assign, cent, used = oracle.cluster_and_balance(emb, K, 5, init, _rowptr(deg), split, caps, words)
+    km = oracle.kmeans(emb, K, 5, init)
+    np.testing.assert_array_equal(cent, km.centroids)                  # balancing moves labels, not centroids
+    for s in range(3):
+        load = np.bincount(assign[split == s], minlength=K)
+        assert load.max() <= caps[s] and load.sum() == (split == s).sum()
+    assert all(r >= 1 for r in used)                                   # the mixture is skewed: every set needed work
+    # the sets do not interfere: balancing each set on its own from the K-Means labels gives the same labels
+    for s in range(3):
+        alone, _ = oracle.balance(_rowptr(deg), km.assign, K, caps[s], words[s], split == s)
+        assert np.array_equal(alone[split == s], assign[split == s])

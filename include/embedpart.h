@@ -289,6 +289,26 @@ int ep_balance(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t
                int32_t *rounds_used, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
+ * ep_cluster_and_balance -- Phase 2 as a whole (Algorithm 3): P <- KMeans(E, k), then the balancing
+ * loop for the training vertices, for the validation vertices and for the remaining ones, in that
+ * order, each with its own capacity.  The calls above, made by the library in sequence.
+ *
+ *   emb, N, d, K, iters, init_centroids, assign, centroids: as for ep_kmeans
+ *   rowptr, rowptr_is_int64, max_degree:                    as for ep_balance
+ *   split       [dev] N bytes: 0 = training, 1 = validation, 2 = remaining vertex
+ *   capacities  [host] 3 int64: C of each set (the paper uses floor(beta_x |V_x| / K))
+ *   rand_words  [dev] 3 x max_rounds x N uint32: set s uses rows [s * max_rounds, (s + 1) * max_rounds)
+ *   rounds_used [host] out or NULL, 3 int32
+ * Synchronises the stream like ep_balance; errors as for ep_kmeans and ep_balance.
+ */
+size_t ep_cluster_and_balance_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int64_t max_degree);
+int ep_cluster_and_balance(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                           const float *init_centroids, const void *rowptr, int32_t rowptr_is_int64,
+                           int64_t max_degree, const uint8_t *split, const int64_t *capacities,
+                           const uint32_t *rand_words, int32_t max_rounds, int32_t *assign, float *centroids,
+                           int32_t *rounds_used, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
  * Host-buffer variants.  Same operations and the same kernels; inputs and outputs are [host]
  * pointers.  Each call copies its inputs into `arena` (a [dev] scratch block of at least
  * *_host_arena_bytes bytes, 256-byte aligned, which also holds the kernel workspace), runs, and

@@ -21,6 +21,7 @@ EXPORTED_SYMBOLS = (
     "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
     "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
     "ep_balance_workspace_bytes", "ep_migrate", "ep_balance",
+    "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance",
 )
 
 EP_OK = 0
@@ -113,6 +114,11 @@ def load_library() -> ctypes.CDLL:
             lib.ep_kmeans_sampled.restype = ctypes.c_int
             lib.ep_gather_rows.argtypes = [vp, vp, i64, i32, vp, i64, vp, vp]
             lib.ep_gather_rows.restype = ctypes.c_int
+            lib.ep_cluster_and_balance_workspace_bytes.argtypes = [vp, i64, i32, i32, i64]
+            lib.ep_cluster_and_balance_workspace_bytes.restype = sz
+            lib.ep_cluster_and_balance.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, i32, i64, vp, vp, vp, i32, vp, vp, vp,
+                                                   vp, sz, vp]
+            lib.ep_cluster_and_balance.restype = ctypes.c_int
             lib.ep_balance_workspace_bytes.argtypes = [vp, i64, i32, i64]
             lib.ep_balance_workspace_bytes.restype = sz
             lib.ep_migrate.argtypes = [vp, vp, i32, i64, i32, vp, i64, i64, vp, vp, vp, vp, sz, vp]
@@ -385,6 +391,38 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return used.value
+
+    def cluster_and_balance(self, emb, K: int, iters: int, init_centroids, rowptr, max_degree: int, split, capacities,
+                            rand_rounds):
+        """Phase 2 as a whole (Algorithm 3): K-Means, then the balancing loops of the training (split 0), validation
+        (1) and remaining (2) vertices.  rand_rounds: [3, max_rounds, N] int32.  Returns (KMeansResult, rounds used
+        per set).  Synchronises the stream."""
+        emb = _check_cuda(emb, torch.float32, "emb", self.device)
+        init = _check_cuda(init_centroids, torch.float32, "init_centroids", self.device)
+        rowptr = _check_cuda(rowptr, rowptr.dtype, "rowptr", self.device)
+        split = _check_cuda(split, torch.uint8, "split", self.device)
+        rand_rounds = _check_cuda(rand_rounds, torch.int32, "rand_rounds", self.device)
+        N, d = emb.shape
+        if init.shape != (K, d) or rowptr.numel() != N + 1 or split.numel() != N:
+            raise ValueError("init_centroids must be K x d, rowptr N + 1 entries, split N bytes")
+        if rand_rounds.dim() != 3 or rand_rounds.shape[0] != 3 or rand_rounds.shape[2] != N:
+            raise ValueError("rand_rounds must be [3, max_rounds, N]")
+        need = self._lib.ep_cluster_and_balance_workspace_bytes(self._h, N, d, K, max_degree)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range or unsupported: N={N} d={d} K={K} max_degree={max_degree}")
+        ws = self.workspace(need)
+        assign = torch.empty(N, dtype=torch.int32, device=self.device)
+        cent = torch.empty(K, d, dtype=torch.float32, device=self.device)
+        caps = (ctypes.c_int64 * 3)(*[int(c) for c in capacities])
+        used = (ctypes.c_int32 * 3)()
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_cluster_and_balance(self._h, _dev_ptr(emb), N, d, K, iters, _dev_ptr(init), _dev_ptr(rowptr),
+                                                  int(rowptr.dtype == torch.int64), max_degree, _dev_ptr(split), caps,
+                                                  _dev_ptr(rand_rounds), rand_rounds.shape[1], _dev_ptr(assign),
+                                                  _dev_ptr(cent), used, _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return KMeansResult(assign, cent, None), list(used)
 
     def relabel_graph(self, rowptr, colidx, perm, inv_perm):
         """(new_rowptr, new_colidx): the CSR graph with vertex perm[i] renamed i."""

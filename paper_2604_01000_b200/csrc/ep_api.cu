@@ -101,6 +101,17 @@ bool sampled_layout(const ep_ctx *ctx, int64_t N, int d, int K, int64_t M, void 
 
 }  // namespace
 
+namespace {
+
+// mask[v] = 1 when split[v] == which, else 0.
+__global__ void __launch_bounds__(256) split_mask(const uint8_t *__restrict__ split, int64_t N, int which,
+                                                  uint8_t *__restrict__ mask) {
+    const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v < N) mask[v] = split[v] == which ? 1 : 0;
+}
+
+}  // namespace
+
 extern "C" {
 
 const char *ep_status_string(int status) {
@@ -528,6 +539,50 @@ int ep_balance(ep_ctx *ctx, const void *rowptr, int32_t rowptr_is_int64, int64_t
         if (!words) return fail(ctx, EP_ERR_UNSUPPORTED, "not balanced after %d applications of the policy", max_rounds);
         if (rounds_used) *rounds_used = r + 1;
     }
+}
+
+// ---------------------------------------------------------------------------------------------- phase 2
+size_t ep_cluster_and_balance_workspace_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int64_t max_degree) {
+    const size_t km = ep_kmeans_workspace_bytes(ctx, N, d, K), bal = ep_balance_workspace_bytes(ctx, N, K, max_degree);
+    if (km == 0 || bal == 0) return 0;
+    Arena a(nullptr);
+    a.take<uint8_t>(N);
+    return a.used + std::max(km, bal);
+}
+
+int ep_cluster_and_balance(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                           const float *init_centroids, const void *rowptr, int32_t rowptr_is_int64, int64_t max_degree,
+                           const uint8_t *split, const int64_t *capacities, const uint32_t *rand_words,
+                           int32_t max_rounds, int32_t *assign, float *centroids, int32_t *rounds_used, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!split || !capacities) return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    const size_t need = ep_cluster_and_balance_workspace_bytes(ctx, N, d, K, max_degree);
+    if (need == 0)
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range or unsupported: N=%lld d=%d K=%d max_degree=%lld", (long long)N, d,
+                    K, (long long)max_degree);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need)
+        return fail(ctx, EP_ERR_WORKSPACE, "phase 2 workspace: need %zu bytes, 256-byte aligned", need);
+    Arena a(workspace);
+    uint8_t *mask = a.take<uint8_t>(N);
+    void *ws = a.base + a.used;
+    const size_t ws_bytes = workspace_bytes - a.used;
+    int rc = ep_kmeans(ctx, emb, N, d, K, iters, init_centroids, assign, centroids, nullptr, ws, ws_bytes, cuda_stream);
+    if (rc != EP_OK) return rc;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    for (int s = 0; s < 3; ++s) {
+        split_mask<<<(unsigned)ceil_div(N, 256), 256, 0, st>>>(split, N, s, mask);
+        ctx->launches += 1;
+        EP_CUDA(ctx, cudaGetLastError());
+        int32_t used = 0;
+        rc = ep_balance(ctx, rowptr, rowptr_is_int64, N, K, mask, capacities[s], max_degree,
+                        rand_words ? rand_words + (size_t)s * (size_t)max_rounds * (size_t)N : nullptr, max_rounds, assign, &used,
+                        ws, ws_bytes, cuda_stream);
+        if (rounds_used) rounds_used[s] = used;
+        if (rc != EP_OK) return rc;
+    }
+    return EP_OK;
 }
 
 // ---------------------------------------------------------------------------------------------- reorder

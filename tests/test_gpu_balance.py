@@ -116,3 +116,31 @@ def test_errors(ctx):
     bad[5] = 9                                                                    # label outside [0, K)
     ctx.migrate(rowptr, bad, K, 400, 1, _words((N,), 2).cuda())
     assert ctx.poll_status() == 4 and ctx.poll_status() == 0
+
+
+def test_phase_two_as_a_whole(ctx):
+    """ep_cluster_and_balance against the oracle's composition (K-Means labels up to near-ties, so the
+    comparison is made stage by stage: the balancing stages on the library's own K-Means labels)."""
+    w = synth.scaled(synth.WORKLOADS["cfg4"], 40_009)
+    N, K = w.N, 8
+    emb = synth.embeddings(w, device="cuda")
+    init = emb[synth.init_centroid_rows(w, K, device="cuda")].contiguous()
+    rowptr, _ = synth.graph(w, device="cuda")
+    split = torch.from_numpy(np.random.default_rng(1).choice(3, size=N, p=[0.5, 0.2, 0.3]).astype(np.uint8))
+    caps = [int(np.floor(1.05 * int((split == s).sum()) / K)) for s in range(3)]
+    words = _words((3, 10, N), 11)
+    deg = np.diff(rowptr.cpu().numpy().astype(np.int64))
+    got, used = ctx.cluster_and_balance(emb, K, 6, init, rowptr, int(deg.max()), split.cuda(), caps, words.cuda())
+    ctx.check()
+    km = ctx.kmeans(emb, K, 6, init)                                   # the same first stage on its own
+    torch.cuda.synchronize()
+    assert torch.equal(got.centroids, km.centroids)
+    ref = km.assign.cpu().numpy()
+    ref_used = []
+    for s in range(3):
+        ref, r = oracle.balance(rowptr.cpu().numpy(), ref, K, caps[s], words[s].numpy().view(np.uint32), (split == s).numpy())
+        ref_used.append(r)
+    np.testing.assert_array_equal(got.assign.cpu().numpy(), ref)
+    assert used == ref_used
+    for s in range(3):
+        assert np.bincount(ref[(split == s).numpy()], minlength=K).max() <= caps[s]

@@ -216,3 +216,32 @@ def test_argument_errors_are_reported_not_faulted(ctx):
     assert b"workspace" in lib.ep_last_error(ctx._h)
     torch.cuda.synchronize()
     assert ctx.poll_status() == 0
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other(ctx):
+    """Two independent clustering runs issued side by side (own context and workspace each, own stream each) give
+    what they give one after the other."""
+    import paper_2604_01000_b200 as ep
+    w = synth.scaled(synth.WORKLOADS["cfg4"], 60_013)
+    emb, init = _inputs(w)
+    init2 = emb[synth.init_centroid_rows(w, 300, device="cuda")].contiguous()
+    alone_a = ctx.kmeans(emb, w.K, 6, init)
+    alone_b = ctx.kmeans(emb, 300, 3, init2)
+    torch.cuda.synchronize()
+    other = ep.Context(0)
+    try:
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        sa.wait_stream(torch.cuda.current_stream())
+        sb.wait_stream(torch.cuda.current_stream())
+        for _ in range(3):
+            with torch.cuda.stream(sa):
+                got_a = ctx.kmeans(emb, w.K, 6, init)
+            with torch.cuda.stream(sb):
+                got_b = other.kmeans(emb, 300, 3, init2)
+        torch.cuda.synchronize()
+        ctx.check()
+        other.check()
+    finally:
+        other.close()
+    assert torch.equal(got_a.assign, alone_a.assign) and torch.equal(got_a.centroids, alone_a.centroids)
+    assert torch.equal(got_b.assign, alone_b.assign) and torch.equal(got_b.centroids, alone_b.centroids)

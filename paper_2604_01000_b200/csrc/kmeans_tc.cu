@@ -209,7 +209,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             s[q * 4 + 3] = fmaf(-2.f, __uint_as_float(v[h * 8 + q * 4 + 3]), n4.w);
                         }
                         const float m = fmin3(fmin3(s[0], s[1], s[2]), fmin3(s[3], s[4], s[5]), fminf(s[6], s[7]));
-                        if (m <= cut) {
+                        if (__any_sync(FULL, m <= cut)) {   // one lane is enough: the whole warp ranks the block
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 const float key =

@@ -144,3 +144,23 @@ def test_phase_two_as_a_whole(ctx):
     assert used == ref_used
     for s in range(3):
         assert np.bincount(ref[(split == s).numpy()], minlength=K).max() <= caps[s]
+
+
+def test_loose_degree_bound_takes_the_four_pass_sort(ctx):
+    """A degree bound far above the real degrees makes the sort key wider than 24 bits (four radix passes);
+    the result does not depend on the bound."""
+    w = synth.scaled(synth.WORKLOADS["cfg4"], 50_021)
+    rowptr, _ = synth.graph(w, device="cuda")
+    N, K = w.N, 32
+    assign = _skewed_labels(N, K, 21)
+    C = int(np.floor(1.05 * N / K))
+    rw = _words((N,), 22)
+    deg = np.diff(rowptr.cpu().numpy().astype(np.int64))
+    tight, loose = assign.clone().cuda(), assign.clone().cuda()
+    ctx.migrate(rowptr, tight, K, C, int(deg.max()), rw.cuda())
+    ctx.migrate(rowptr, loose, K, C, (1 << 24) - 1, rw.cuda())                    # K (D + 1) = 2^29
+    torch.cuda.synchronize()
+    ctx.check()
+    ref, _ = oracle.migrate(rowptr.cpu().numpy(), assign.numpy(), K, C, rw.numpy().view(np.uint32))
+    np.testing.assert_array_equal(tight.cpu().numpy(), ref)
+    np.testing.assert_array_equal(loose.cpu().numpy(), ref)

@@ -684,7 +684,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
             constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
             if (p.tc_fused) {
                 return kmeans_tcf_assign(ctx, *tcf_state, emb, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
-                                         b.pcnt, b.late_list, b.late_count, stream);
+                                         b.pcnt, b.late_list, b.late_count, /*use_prev=*/t > 0, stream);
             } else if (p.fused) {
                 auto kern = kmeans_assign_fused<VPL, R>;
                 EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));

@@ -12,8 +12,11 @@
 //      label.  Otherwise the row id goes to the warp's list of undecided rows, with the set of centroids
 //      inside the bound;
 //   3. two sorting warps (alternating tiles) group the tile's decided rows by label, stably;
-//   4. eight accumulate warps, each owning K/8 clusters with one 16-byte column chunk per lane, add the
-//      rows of their clusters, in row order, from the shared-memory tile into registers.
+//   4. eight accumulate warps, each owning up to KMAX/8 clusters with one 16-byte column chunk per lane, add
+//      the rows of their clusters, in row order, from the shared-memory tile into registers.  Which warp owns
+//      which cluster is settled per launch from the block's own counts of the previous iteration, so that
+//      uneven clusters still give the warps even work; a cluster's rows are added by one warp in row order
+//      whoever that is, so the sums do not depend on it.
 // kmeans_late_rows then settles the undecided rows in fp32 (lowest index wins ties, same summation order
 // as the CUDA-core kernels) and adds them into a second set of partial sums.  No floating-point atomics
 // anywhere: the order of every addition is fixed by the launch shape and the lists, so results repeat
@@ -68,14 +71,19 @@ struct FusedShared {
     uint64_t t_full[2], t_empty[2];
     uint64_t lab_full[2], lab_empty[2];
     uint64_t ord_full[2], ord_empty[2];
+    uint64_t plan_full;
     uint32_t tmem_base;
     int abort;
-    uint8_t lab[2][BM];                 // label of each row of the tile; MAX_K = not to be accumulated here
-    uint16_t order[2][BM];              // the tile's rows grouped by label, ascending row inside a label, each as
+    uint8_t lab[2][BM];                 // sorting key of each row of the tile; MAX_K = not to be accumulated here
+    uint16_t order[2][BM];              // the tile's rows grouped by sorting key, ascending row inside a key, each as
                                         // its byte offset inside a k-block with the swizzle term in bits 4..6
     int goff[2][MAX_K + 1];             // first position of each label in order[]
     int hcnt[2][MAX_K + 1];             // scratch of the two sorting warps
-    int cnt[MAX_K];
+    int cnt[MAX_K];                     // rows per sorting key that this block decided
+    int plan_cnt[MAX_K];                // weights of the clusters when the accumulate work is shared out
+    uint8_t plan_sorted[MAX_K];         // clusters by descending weight
+    uint8_t keymap[MAX_K + 1];          // cluster -> sorting key = owner warp * OWN + slot; [MAX_K] = MAX_K
+    int8_t kof[MAX_K];                  // sorting key -> cluster, -1 = no cluster
     alignas(16) float cn[MAX_K];
 };
 
@@ -91,6 +99,17 @@ __device__ __forceinline__ void tmem_issue16(uint32_t taddr, uint32_t (&v)[VN]) 
         : "r"(taddr + O)
         : "memory");
 }
+// a += x where i < n, as four predicated additions: no branch, whatever the compiler thinks of the condition.
+__device__ __forceinline__ void add_if_less(float4 &a, const float4 &x, int i, int n) {
+    asm("{\n.reg .pred p;\n"
+        "setp.lt.s32 p, %8, %9;\n"
+        "@p add.rn.f32 %0, %0, %4;\n"
+        "@p add.rn.f32 %1, %1, %5;\n"
+        "@p add.rn.f32 %2, %2, %6;\n"
+        "@p add.rn.f32 %3, %3, %7;\n}"
+        : "+f"(a.x), "+f"(a.y), "+f"(a.z), "+f"(a.w)
+        : "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w), "r"(i), "r"(n));
+}
 __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // KMAX = 32 or 64: upper bound of K.  VPL = 16-byte chunks of a row per lane: 1 for d <= 128 with tiles of 128
@@ -99,13 +118,15 @@ __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.syn
 // cn = |c_k|^2 padded with a huge value.  Block b leaves the sums of the rows it decided in psum[b][K][d],
 // their counts in pcnt[b][K], and per screen warp w the undecided rows in late_list[(4 b + w) late_cap ..]
 // (x = row id, y and z = mask of the centroids within the bound), late_count[4 b + w] of them.
+// use_prev != 0: pcnt[b] still holds this block's counts of the previous iteration over the same tiles; they
+// weigh the clusters when these are shared out among the accumulate warps (any sharing gives the same sums).
 template <int KMAX, int VPL>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
                 const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
                 int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
                 int32_t *__restrict__ assign, float *__restrict__ psum, int *__restrict__ pcnt,
-                int4 *__restrict__ late_list, int64_t late_cap, int *__restrict__ late_count,
+                int4 *__restrict__ late_list, int64_t late_cap, int *__restrict__ late_count, int use_prev,
                 unsigned long long *counters, int *status) {
     // The swizzled tiles need 1024-byte alignment.  The array is used as declared (no pointer arithmetic
     // through integers), so that every access below stays a shared-memory instruction; should a launch
@@ -144,6 +165,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_init(&sh->ord_full[i], 1);
             mbar_init(&sh->ord_empty[i], A_WARPS);
         }
+        mbar_init(&sh->plan_full, 1);
         sh->abort = 0;
         sh->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,6 +231,46 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // so that an accumulate warp finds the rows of a cluster as one run, in row order.
         const uint32_t hw = (uint32_t)warp - 2u;
         const unsigned lt = (1u << lane) - 1u;
+        if (warp == 3) {
+            // Which accumulate warp owns which cluster: heaviest cluster first, each to the warp with the least
+            // weight so far that still has a free slot (OWN slots per warp).  The weight of a cluster is the number
+            // of rows it got from this block's tiles in the previous iteration (+ 1), so the warps end up with
+            // about the same number of rows per tile however uneven the clusters are.
+            constexpr int OWN = KMAX / A_WARPS;
+            for (int k = lane; k <= MAX_K; k += 32) sh->keymap[k] = (uint8_t)MAX_K;
+            for (int q = lane; q < MAX_K; q += 32) {
+                sh->kof[q] = (int8_t)-1;
+                int w = 0;
+                if (q < K) w = 1 + (use_prev ? min(max(pcnt[(size_t)blockIdx.x * K + q], 0), 1 << 24) : 0);
+                sh->plan_cnt[q] = w;
+            }
+            __syncwarp();
+            for (int k = lane; k < K; k += 32) {
+                const int mine = sh->plan_cnt[k];
+                int rank = 0;
+                for (int j = 0; j < K; ++j) {
+                    const int o = sh->plan_cnt[j];
+                    rank += (o > mine || (o == mine && j < k)) ? 1 : 0;
+                }
+                sh->plan_sorted[rank] = (uint8_t)k;
+            }
+            __syncwarp();
+            unsigned load = 0u;
+            int taken = 0;
+            for (int r = 0; r < K; ++r) {
+                const int k = sh->plan_sorted[r];
+                const unsigned key = (lane < A_WARPS && taken < OWN) ? ((load << 3) | (unsigned)lane) : 0xFFFFFFFFu;
+                const unsigned best = __reduce_min_sync(FULL, key);
+                if (lane < A_WARPS && key == best) {
+                    sh->keymap[k] = (uint8_t)(lane * OWN + taken);
+                    sh->kof[lane * OWN + taken] = (int8_t)k;
+                    ++taken;
+                    load += (unsigned)sh->plan_cnt[k];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->plan_full);
+        }
         EP_CLK_DECL
         for (uint32_t it = hw;; it += 2) {
             const int64_t tile = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
@@ -290,8 +352,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float2 nr_next = make_float2(0.f, 0.f);            // this row's norms, fetched one tile ahead
         if (sw < SWARPS && (int64_t)blockIdx.x * BMR + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BMR + stid);
 
+        bool planned = mbar_wait(&sh->plan_full, 0u, abort_flag);
         uint32_t it = 0;
-        for (int64_t tile = blockIdx.x; sw < SWARPS && tile < num_tiles; tile += gridDim.x, ++it) {
+        for (int64_t tile = blockIdx.x; planned && sw < SWARPS && tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u, par = it & 1u;
             const int64_t row = tile * BMR + stid;
             const float2 nr = nr_next;
@@ -373,7 +436,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             EP_CLK(pc_work)
             if (!mbar_wait(&sh->lab_empty[par], use ^ 1u, abort_flag)) break;
             EP_CLK(pc_wait)
-            sh->lab[par][stid] = (uint8_t)label;
+            sh->lab[par][stid] = sh->keymap[label];        // the sorting key: owner warp, then the owner's slot
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->lab_full[par]);
         }
@@ -389,7 +452,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     } else if (warp >= A_WARP0) {
         // ---------------------------------------------------------------- accumulate warps
-        const int aw = warp - A_WARP0;                     // owns clusters aw, aw + 8, ...
+        const int aw = warp - A_WARP0;                     // owns the clusters with sorting keys aw OWN .. aw OWN + OWN - 1
         constexpr int OWN = KMAX / A_WARPS;
         const uint32_t lx = (uint32_t)(lane & 7) << 4;     // a lane's place inside a 128-byte swizzle row, before the swizzle
         float4 acc[OWN][VPL];                              // this lane's 16-byte chunks of a row are lane, lane + 32
@@ -397,9 +460,10 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < OWN; ++i)
 #pragma unroll
             for (int v = 0; v < VPL; ++v) acc[i][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        bool planned = mbar_wait(&sh->plan_full, 0u, abort_flag);
         EP_CLK_DECL
         uint32_t it = 0;
-        for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+        for (int64_t tile = blockIdx.x; planned && tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t s = it % (uint32_t)stages;
             const uint32_t par = it & 1u, use = (it >> 1) & 1u;
             const uint8_t *xl = x_smem + (size_t)s * stage_bytes + (size_t)(lane >> 3) * X_KB_BYTES;   // this lane's first k-block
@@ -407,39 +471,33 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (!mbar_wait(&sh->ord_full[par], use, abort_flag)) break;
             if (!mbar_wait(&sh->x_full[s], (it / (uint32_t)stages) & 1u, abort_flag)) break;   // long complete: makes the tile visible here
             EP_CLK(pc_wait)
-            int q0[OWN], q1[OWN];                          // the runs of this warp's clusters in order[]
+            // The rows of this warp's clusters are one stretch of order[], slot after slot; lane i holds where
+            // slot i starts (lane OWN: where the stretch ends).
+            const int bl = sh->goff[par][aw * OWN + min(lane, OWN)];
+            auto load_row = [&](float4 (&x)[VPL], uint32_t o) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v)
+                    x[v] = lane + 32 * v < d4 ? *reinterpret_cast<const float4 *>(xl + (size_t)(4 * v) * X_KB_BYTES + (o ^ lx))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            };
 #pragma unroll
             for (int i = 0; i < OWN; ++i) {
-                const int k = min(aw + A_WARPS * i, K - 1);
-                q0[i] = sh->goff[par][k];
-                q1[i] = aw + A_WARPS * i < K ? sh->goff[par][k + 1] : q0[i];
-            }
-#pragma unroll
-            for (int i = 0; i < OWN; ++i) {
-                const int p1 = q1[i];
-                for (int p = q0[i]; p < p1; p += 4) {       // four rows at a time: loads first, adds in row order
+                const int p1 = __shfl_sync(FULL, bl, i + 1);
+                for (int p = __shfl_sync(FULL, bl, i); p < p1; p += 4) {       // four rows at a time: loads first, adds in row order
                     float4 x[4][VPL];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t o = sh->order[par][min(p + u, p1 - 1)];
-#pragma unroll
-                        for (int v = 0; v < VPL; ++v)
-                            x[u][v] = lane + 32 * v < d4
-                                          ? *reinterpret_cast<const float4 *>(xl + (size_t)(4 * v) * X_KB_BYTES + (o ^ lx))
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 4; ++u) {              // a run's last group is not padded with repeated reads
                         if (p + u < p1) {
+                            load_row(x[u], (uint32_t)sh->order[par][p + u] & 0x3FF0u);
+                        } else {
 #pragma unroll
-                            for (int v = 0; v < VPL; ++v) {
-                                acc[i][v].x += x[u][v].x;
-                                acc[i][v].y += x[u][v].y;
-                                acc[i][v].z += x[u][v].z;
-                                acc[i][v].w += x[u][v].w;
-                            }
+                            for (int v = 0; v < VPL; ++v) x[u][v] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
                     }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) add_if_less(acc[i][v], x[u][v], p + u, p1);
                 }
             }
             __syncwarp();
@@ -453,8 +511,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
 #pragma unroll
         for (int i = 0; i < OWN; ++i) {
-            const int k = aw + A_WARPS * i;
-            if (k < K) {
+            const int k = planned ? (int)sh->kof[aw * OWN + i] : -1;
+            if (k >= 0 && k < K) {
 #pragma unroll
                 for (int v = 0; v < VPL; ++v)
                     if (lane + 32 * v < d4) out[(size_t)k * d4 + lane + 32 * v] = acc[i][v];
@@ -462,7 +520,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     }
     __syncthreads();
-    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[k];
+    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
     if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
     if (warp == 2) {
         tc_fence_after();
@@ -529,8 +587,10 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
     };
     // ---- 1. labels, the rows' data fetched four ahead
     constexpr int AHEAD1 = 4;
-    for (int p0 = warp * 32; p0 < cum[4]; p0 += nwarps * 32) {
-        const int cnt = min(32, cum[4] - p0);
+    // entries per warp and turn: 32 when there are many, fewer when that keeps all warps busy on a short list
+    const int turn = min(32, max(AHEAD1, (cum[4] + nwarps * AHEAD1 - 1) / (nwarps * AHEAD1) * AHEAD1));
+    for (int p0 = warp * turn; p0 < cum[4]; p0 += nwarps * turn) {
+        const int cnt = min(turn, cum[4] - p0);
         int4 e = make_int4(-1, 0, 0, 0);
         if (lane < cnt) {
             const int p = p0 + lane;
@@ -749,7 +809,7 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
 template <int KMAX, int VPL>
 static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo, const float2 *rownorm,
                       int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, int4 *late_list, int *late_count,
-                      cudaStream_t stream) {
+                      bool use_prev, cudaStream_t stream) {
     auto kern = kmeans_tc_fused<KMAX, VPL>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
     unsigned long long *counters =
@@ -757,7 +817,7 @@ static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, cons
     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
     kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, cn, clo, rownorm, N, d, K, st.npad, st.num_kb,
                                               st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK, assign,
-                                              psum, pcnt, late_list, st.late_cap, late_count, counters, ctx->d_status);
+                                              psum, pcnt, late_list, st.late_cap, late_count, use_prev ? 1 : 0, counters, ctx->d_status);
     tm.end(1);
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;
@@ -767,12 +827,12 @@ static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, cons
 // counts in pcnt[b][K]; the kernel for the rows it left undecided adds the slabs grid .. 2 grid - 1.
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
                       const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, void *late_list_ws, int *late_count, cudaStream_t stream) {
+                      int *pcnt, void *late_list_ws, int *late_count, bool use_prev, cudaStream_t stream) {
     int4 *late_list = static_cast<int4 *>(late_list_ws);
     const int vpl = d <= 128 ? 1 : 2;
-    int rc = vpl == 2 ? tcf_launch<32, 2>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
-             : K <= 32 ? tcf_launch<32, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream)
-                       : tcf_launch<64, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, stream);
+    int rc = vpl == 2 ? tcf_launch<32, 2>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
+             : K <= 32 ? tcf_launch<32, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
+                       : tcf_launch<64, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream);
     if (rc != EP_OK) return rc;
     const int kpad = (K + KC - 1) / KC * KC;
     const size_t row = 512 * (size_t)vpl;

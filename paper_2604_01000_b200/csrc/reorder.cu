@@ -27,13 +27,30 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) digit_histogram(const int32_t
     cnt[threadIdx.x] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * SORT_TILE;
+    if (base + SORT_TILE <= N && (reinterpret_cast<uintptr_t>(keys) & 15u) == 0) {
+        // a full tile of an aligned array: all of a thread's keys are on their way before the first is counted
+        const int4 *src = reinterpret_cast<const int4 *>(keys + base);
+        int4 k4[SORT_ITEMS / 4];
+#pragma unroll
+        for (int i = 0; i < SORT_ITEMS / 4; ++i) k4[i] = __ldg(src + i * (SORT_WARPS * 32) + threadIdx.x);
+#pragma unroll
+        for (int i = 0; i < SORT_ITEMS / 4; ++i) {
+            const int kk[4] = {k4[i].x, k4[i].y, k4[i].z, k4[i].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (label_limit > 0 && (unsigned)kk[j] >= (unsigned)label_limit) ep_raise(status, EP_ERR_BAD_INDEX);
+                atomicAdd(&cnt[(kk[j] >> shift) & (RADIX - 1)], 1);
+            }
+        }
+    } else {
 #pragma unroll 4
-    for (int i = 0; i < SORT_ITEMS; ++i) {
-        int64_t idx = base + i * (SORT_WARPS * 32) + threadIdx.x;
-        if (idx < N) {
-            const int key = keys[idx];
-            if (label_limit > 0 && (unsigned)key >= (unsigned)label_limit) ep_raise(status, EP_ERR_BAD_INDEX);
-            atomicAdd(&cnt[(key >> shift) & (RADIX - 1)], 1);
+        for (int i = 0; i < SORT_ITEMS; ++i) {
+            int64_t idx = base + i * (SORT_WARPS * 32) + threadIdx.x;
+            if (idx < N) {
+                const int key = keys[idx];
+                if (label_limit > 0 && (unsigned)key >= (unsigned)label_limit) ep_raise(status, EP_ERR_BAD_INDEX);
+                atomicAdd(&cnt[(key >> shift) & (RADIX - 1)], 1);
+            }
         }
     }
     __syncthreads();
@@ -133,7 +150,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_add(int32_t *data, int64_t 
 //   vals_in  == nullptr: the value of key i is i itself (first pass)
 //   keys_out == nullptr: keys are not needed afterwards (last pass)
 //   inv_out  != nullptr: also writes inv_out[value] = destination (last pass)
-__global__ void __launch_bounds__(SORT_WARPS * 32) digit_scatter(const int32_t *__restrict__ keys_in,
+__global__ void __launch_bounds__(SORT_WARPS * 32, 4) digit_scatter(const int32_t *__restrict__ keys_in,
                                                                   const int32_t *__restrict__ vals_in, int64_t N,
                                                                   int shift, int ntiles,
                                                                   const int32_t *__restrict__ offsets,
@@ -266,6 +283,8 @@ int reorder_run(ep_ctx *ctx, const int32_t *assign, int64_t N, int K, int32_t *p
     if (!timed) ctx->opt_profile = 0;
     Timed tm(ctx, stream, EP_TIMER_REORDER);
     ctx->opt_profile = saved_profile;
+    // four blocks of the scatter kernel per SM need most of the SM's memory as shared memory
+    EP_CUDA(ctx, cudaFuncSetAttribute(digit_scatter, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     for (int p = 0; p < passes; ++p) {
         const bool last = (p == passes - 1);
         int32_t *kout = last ? nullptr : b.keys[p & 1];

@@ -146,6 +146,28 @@ def test_fused_tensor_core_pass_ties_duplicates_and_repeatability(ctx):
     assert torch.equal(a.assign, b.assign) and torch.equal(a.centroids, b.centroids) and torch.equal(a.objective, b.objective)
 
 
+@pytest.mark.parametrize("K,d", [(64, 128), (37, 96), (11, 256)])
+def test_fused_tensor_core_pass_with_very_uneven_clusters(ctx, K, d):
+    """The fused pass shares its clusters out among the accumulate warps by the counts of the previous iteration.
+    Here one mixture component holds 70 % of the rows and every centroid starts inside a component of its own, so one
+    cluster takes more than half of every tile while the others get a handful of rows each; the sums must not depend on who
+    owns what: parity with the oracle over several iterations, and the resume identity across the change of owners."""
+    rng = np.random.default_rng(100 + K)
+    N = 20_011
+    centres = rng.normal(size=(K, d)).astype(np.float32)
+    share = rng.random(N)
+    comp = np.where(share < 0.7, 0, rng.integers(1, K, size=N))
+    comp[:K] = np.arange(K)                                    # every component has a row, and a centroid starts on it
+    emb_h = (centres[comp] + 0.5 * rng.normal(size=(N, d))).astype(np.float32)
+    init_h = emb_h[:K].copy()
+    emb, init = torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+    _run_and_compare(ctx, emb, init, K, 4)
+    three = ctx.kmeans(emb, K, 3, init)
+    four = ctx.kmeans(emb, K, 4, init)
+    step = ctx.kmeans(emb, K, 1, three.centroids)       # first iteration of a call: the default owners
+    assert torch.equal(step.assign, four.assign) and torch.equal(step.centroids, four.centroids)
+
+
 @pytest.mark.parametrize("N,d,K", [(1, 4, 1), (2, 8, 2), (33, 4, 3), (257, 1024, 5), (1000, 12, 1), (515, 100, 9),
                                    (64, 36, 64), (4097, 260, 17), (100, 516, 7)])
 def test_shapes_and_edges(ctx, N, d, K):

@@ -34,8 +34,13 @@ import synth  # noqa: E402
 NCU_TRAFFIC = {
     ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_286_797_056 + 615_664_128, "launch": "all rows, one iteration",
                                       "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
-    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_274_435_584 + 13_306_368, "launch": "all rows, one iteration",
+    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_274_468_000 + 13_835_264, "launch": "all rows, one iteration",
                                     "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
+    # captured on 12 M rows of the same recipe (6,240,652,000 + 52,459,520 bytes = 524.4 per row) and scaled by the
+    # rows of a full launch: the kernel's traffic is the rows it streams
+    ("kmeans_assign_K64", "cfg5"): {"bytes_per_launch": int(round(111_059_956 * (6_240_652_000 + 52_459_520) / 12_000_000)),
+                                    "launch": "all rows, one iteration; scaled from a 12 M-row capture",
+                                    "source": "profiles/kmeans_tc_fused_K64_cfg5_12M_rows.md"},
 }
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio used to derive the TF32 roof from the bf16 one
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -299,6 +304,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--kmeans-path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--rows", type=int, default=0,
+                    help="run the workload's recipe at this many vertices (mean degree kept): a case small enough for a "
+                         "profiler capture; the line it prints names the scaled workload and is not a bench value")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -306,6 +314,8 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     w = synth.WORKLOADS[args.workload]
+    if args.rows > 0:
+        w = synth.scaled(w, args.rows)
 
     if args.impl == "reference":
         run_reference(args, w, rank)

@@ -46,13 +46,16 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
                                                              int64_t nnz, int K, LabT *__restrict__ lab,
                                                              unsigned long long *part_vertices,
                                                              unsigned long long *part_edges, int *status) {
+    // block-local counts: vertices, and the degree sum as two 32-bit words (low word, carries + high parts), because
+    // 32-bit additions are native in shared memory and 64-bit ones are not
     __shared__ unsigned int cv[HIST_SMEM_K];
-    __shared__ unsigned long long ce[HIST_SMEM_K];
+    __shared__ unsigned int ce_lo[HIST_SMEM_K], ce_hi[HIST_SMEM_K];
     const bool local = K <= HIST_SMEM_K;
     if (local) {
         for (int k = threadIdx.x; k < K; k += blockDim.x) {
             cv[k] = 0u;
-            ce[k] = 0ull;
+            ce_lo[k] = 0u;
+            ce_hi[k] = 0u;
         }
         __syncthreads();
     }
@@ -73,7 +76,11 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
         }
         if (local) {
             atomicAdd(&cv[a], 1u);
-            atomicAdd(&ce[a], (unsigned long long)deg);
+            const unsigned lo = (unsigned)((unsigned long long)deg & 0xffffffffull);
+            const unsigned hi = (unsigned)((unsigned long long)deg >> 32);
+            const unsigned old = atomicAdd(&ce_lo[a], lo);
+            const unsigned carry = (old + lo < old) ? 1u : 0u;     // the low word wrapped
+            if (hi + carry) atomicAdd(&ce_hi[a], hi + carry);
         } else {
             atomicAdd(&part_vertices[a], 1ull);
             atomicAdd(&part_edges[a], (unsigned long long)deg);
@@ -83,7 +90,8 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
         __syncthreads();
         for (int k = threadIdx.x; k < K; k += blockDim.x) {
             if (cv[k]) atomicAdd(&part_vertices[k], (unsigned long long)cv[k]);
-            if (ce[k]) atomicAdd(&part_edges[k], ce[k]);
+            const unsigned long long e = ((unsigned long long)ce_hi[k] << 32) + ce_lo[k];
+            if (e) atomicAdd(&part_edges[k], e);
         }
     }
 }

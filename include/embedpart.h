@@ -54,11 +54,16 @@ enum {
                                (read with ep_profile_read); 0 = off (default) */
     EP_OPT_TIMER_GROUP = 3, /* 0..3: calls made while group g is selected log into timers
                                g * EP_TIMER_COUNT + timer, so a caller can tell two calls apart */
-    EP_OPT_KMEANS_CAND_MB = 4 /* 1..32768 (default 1024): upper bound in MiB of the candidate-key buffer the
+    EP_OPT_KMEANS_CAND_MB = 4, /* 1..32768 (default 1024): upper bound in MiB of the candidate-key buffer the
                                tensor-core path keeps in the workspace (64 bytes per row and 1024 centroids);
                                rows are processed in chunks that fit it (never less than one pass of the
                                grid), and fewer, longer chunks run faster.  Set it before the workspace
                                query: it changes the answer */
+    EP_OPT_QUALITY_SLICE_KB = 5 /* 1..4194304 (default 57344 = 56 MiB): ep_partition_quality gathers the label of
+                               every entry's target; when the repacked labels of all vertices take more than this,
+                               the vertex range is cut into up to 8 slices of at most this size and the column ids
+                               are streamed once per slice, so that a slice's labels stay in the L2.  The result
+                               does not depend on it */
 };
 
 /* Timers kept while EP_OPT_PROFILE is 1. */

@@ -29,6 +29,7 @@ EP_OPT_KMEANS_PATH = 1
 EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
 EP_OPT_KMEANS_CAND_MB = 4
+EP_OPT_QUALITY_SLICE_KB = 5
 TIMER_COUNT = 9
 TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
           "kmeans_resolve": 5, "graph_bandwidth": 6, "relabel": 7, "balance": 8}
@@ -222,6 +223,12 @@ class Context:
     def set_kmeans_cand_mb(self, mib: int):
         """Upper bound (MiB) of the tensor-core path's candidate buffer; set before calling kmeans."""
         rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_CAND_MB, mib)
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_quality_slice_kb(self, kib: int):
+        """Largest label slice (KiB) ep_partition_quality gathers from in one pass over the column ids."""
+        rc = self._lib.ep_set_option(self._h, EP_OPT_QUALITY_SLICE_KB, kib)
         if rc != EP_OK:
             self._raise(rc)
 

@@ -145,6 +145,7 @@ int ep_create(ep_ctx **out, int device) {
     ctx->opt_profile = 0;
     ctx->opt_timer_group = 0;
     ctx->opt_cand_mb = 1024;
+    ctx->opt_slice_kb = 56 * 1024;
     ctx->launches = 0;
     ctx->last_error[0] = 0;
     DeviceGuard g(device);
@@ -199,6 +200,10 @@ int ep_set_option(ep_ctx *ctx, int option, int value) {
         ctx->opt_cand_mb = value;
         return EP_OK;
     }
+    if (option == EP_OPT_QUALITY_SLICE_KB && value >= 1 && value <= 4194304) {
+        ctx->opt_slice_kb = value;
+        return EP_OK;
+    }
     return fail(ctx, EP_ERR_INVALID_ARG, "unknown option %d or value %d", option, value);
 }
 
@@ -218,6 +223,10 @@ int ep_get_option(const ep_ctx *ctx, int option, int *value) {
     }
     if (option == EP_OPT_KMEANS_CAND_MB) {
         *value = ctx->opt_cand_mb;
+        return EP_OK;
+    }
+    if (option == EP_OPT_QUALITY_SLICE_KB) {
+        *value = ctx->opt_slice_kb;
         return EP_OK;
     }
     return EP_ERR_INVALID_ARG;

@@ -23,6 +23,7 @@ struct ep_ctx {
     int opt_profile;       // EP_OPT_PROFILE
     int opt_timer_group;   // EP_OPT_TIMER_GROUP
     int opt_cand_mb;       // EP_OPT_KMEANS_CAND_MB
+    int opt_slice_kb;      // EP_OPT_QUALITY_SLICE_KB
     long long launches;    // kernels launched through this context
     std::vector<ep_timed_interval> intervals;   // pending event pairs (profile mode)
     std::vector<cudaEvent_t> spare_events;

@@ -109,11 +109,15 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
 // GROUPS = 1: a block is one group of QT_THREADS threads.  GROUPS = 4: a block of 1024 threads holds four such
 // groups, each with its own tile, bitmap and named barrier, sharing one copy of the label table: the form for a
 // table so large that only one block fits on an SM, which still needs 32 warps to hide the stream's latency.
-template <typename RowT, typename LabT, int PACK, int GROUPS>
+//
+// SLICED: the launch counts only the entries whose target lies in [col_lo, col_hi) (and reports bad indices only
+// when col_lo == 0); the caller launches it once per slice of the vertex range, each slice's labels small enough to
+// stay in the L2 while the column ids stream past, and the counts of the launches add up.
+template <typename RowT, typename LabT, int PACK, int GROUPS, bool SLICED = false>
 __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
     edge_cut_tiles(const RowT *__restrict__ rowptr, const int32_t *__restrict__ colidx, int64_t nnz,
                    const LabT *__restrict__ lab, int64_t N, const int32_t *__restrict__ tile_row, int64_t ntiles,
-                   unsigned long long *edge_cut, int *status) {
+                   unsigned long long *edge_cut, int *status, int32_t col_lo, int32_t col_hi) {
     __shared__ unsigned bitmap_[GROUPS][QT_WORDS];
     __shared__ int lasthead_[GROUPS][QT_WORDS];
     __shared__ LabT headlab_[GROUPS][QT_EDGES];
@@ -211,16 +215,17 @@ __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
                 const bool live = full || q + j < ne;
                 const int col = cols[j];
                 const bool in = (unsigned)col < (unsigned)N;
-                const int cc = in ? col : 0;                 // an index outside [0, N) is reported, never followed
+                const bool mine = !SLICED || (unsigned)(col - col_lo) < (unsigned)(col_hi - col_lo);
+                const int cc = (in && mine) ? col : 0;       // an index outside [0, N) is reported, never followed
                 unsigned tgt;
                 if (PACK == 8)
                     tgt = lab_tab[cc];
                 else if (PACK == 4)
                     tgt = (lab_tab[cc >> 1] >> ((cc & 1) << 2)) & 15u;
                 else
-                    tgt = (unsigned)__ldg(lab + cc);
-                cut += (live && in && tgt != (unsigned)cur) ? 1u : 0u;
-                bad |= (live && !in) ? 1u : 0u;
+                    tgt = (in && mine) ? (unsigned)__ldg(lab + cc) : (unsigned)cur;
+                cut += (live && in && mine && tgt != (unsigned)cur) ? 1u : 0u;
+                bad |= (live && !in && (!SLICED || col_lo == 0)) ? 1u : 0u;
             }
         };
         // The usual vector: a full tile, every index of this thread inside [0, N).  No per-entry range or length
@@ -229,6 +234,7 @@ __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
             if (PACK == 8) return lab_tab[col] != cur ? 1u : 0u;
             if (PACK == 4)   // cur fills both nibbles: compare the nibble of col in place
                 return ((lab_tab[col >> 1] ^ cur) & (0xFu << ((col << 2) & 4))) != 0u ? 1u : 0u;
+            if (SLICED && (unsigned)(col - col_lo) >= (unsigned)(col_hi - col_lo)) return 0u;   // another launch's entry
             return (unsigned)__ldg(lab + col) != cur ? 1u : 0u;
         };
         auto vec_clean = [&](int q, const int4 &cv) {
@@ -336,7 +342,7 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
         EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));             \
         const int grid = (int)std::min<int64_t>(ceil_div(ntiles, (int64_t)G), (int64_t)ctx->sm_count * (G == 1 ? 4 : 1)); \
         kern<<<grid, QT_THREADS * G, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut,       \
-                                                    ctx->d_status);                                                  \
+                                                    ctx->d_status, 0, 0);                                            \
     } while (0)
             if (pack == 4 && small) EP_EC(4, 1);
             else if (pack == 4) EP_EC(4, 4);
@@ -344,12 +350,27 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
             else EP_EC(8, 4);
 #undef EP_EC
         }
+        int launches = 1;
         if (!launched) {
             const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
-            edge_cut_tiles<RowT, LabT, 0, 1><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
-                                                                            edge_cut, ctx->d_status);
+            // Labels that cannot stay in the L2 beside the stream cost a DRAM sector per entry.  Then the vertex range
+            // is cut into slices whose labels do fit, and the column ids are streamed once per slice: reading them
+            // again is cheaper than missing on every gather.
+            const size_t lab_total = (size_t)N * sizeof(LabT);
+            const int slices = (int)std::min<size_t>(8, ceil_div(lab_total, (size_t)ctx->opt_slice_kb << 10));
+            if (slices <= 1) {
+                edge_cut_tiles<RowT, LabT, 0, 1><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row,
+                                                                                ntiles, edge_cut, ctx->d_status, 0, 0);
+            } else {
+                launches = slices;
+                for (int sl = 0; sl < slices; ++sl) {
+                    const int32_t lo = (int32_t)(N * sl / slices), hi = (int32_t)(N * (sl + 1) / slices);
+                    edge_cut_tiles<RowT, LabT, 0, 1, true><<<grid, QT_THREADS, 0, stream>>>(
+                        rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status, lo, hi);
+                }
+            }
         }
-        tm.end(1);
+        tm.end(launches);
     }
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;

@@ -53,6 +53,34 @@ def test_scaled_configs(ctx, name, N):
     _quality_matches(ctx, rowptr, colidx, _random_labels(N, w.K, 2), w.K)
 
 
+@pytest.mark.parametrize("name,N,K,slice_kb", [("cfg5", 100_003, 64, 16), ("cfg4", 50_021, 32, 7), ("cfg4", 50_021, 300, 30),
+                                               ("cfg5", 100_003, 64, 1)])
+def test_vertex_range_slices_give_the_same_counts(ctx, name, N, K, slice_kb):
+    """Labels too large for the L2 are gathered slice by slice of the vertex range, one pass over the column ids
+    per slice.  A small slice limit forces that path on a small graph (2 to 8 slices, uneven last slice, int64 and
+    int32 row pointers, a bad column id reported once): same counts as the oracle, bit for bit."""
+    w = synth.scaled(synth.WORKLOADS[name], N)
+    rowptr, colidx = synth.graph(w, device="cuda")
+    assign = _random_labels(N, K, 5)
+    ctx.set_quality_slice_kb(slice_kb)
+    try:
+        _quality_matches(ctx, rowptr, colidx, assign, K)
+        _quality_matches(ctx, rowptr.to(torch.int64), colidx, assign, K)
+        bad = colidx.clone()
+        bad[7] = N + 5                                            # out of range: reported, never followed
+        got = ctx.partition_quality(rowptr, bad, assign, K)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 4                             # EP_ERR_BAD_INDEX, whatever the slice it falls in
+        keep = torch.ones_like(bad, dtype=torch.bool)
+        keep[7] = False
+        ref = oracle.partition_quality(rowptr.cpu().numpy(), colidx.cpu().numpy(), assign.cpu().numpy(), K)
+        src = torch.searchsorted(rowptr[1:].contiguous(), torch.tensor([7], device="cuda"), right=True)
+        was_cut = int(assign[src] != assign[colidx[7]])
+        assert int(got.edge_cut.item()) == ref.edge_cut - was_cut
+    finally:
+        ctx.set_quality_slice_kb(56 * 1024)
+
+
 @pytest.mark.parametrize("N,K", [(6_007, 2), (6_007, 16), (6_007, 17), (6_007, 200), (9_001, 256), (5_003, 300),
                                  (100_003, 16), (60_013, 200), (180_001, 9)])
 def test_dense_graph_label_tables_in_shared_memory(ctx, N, K):

@@ -132,7 +132,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // through integers), so that every access below stays a shared-memory instruction; should a launch
     // ever place it differently, the block reports that and leaves before touching anything.
     extern __shared__ __align__(1024) uint8_t smem[];
-    if ((smem_u32(smem) & 1023u) != 0u) {
+    if ((smem_u32(smem) & 1023u) != 0u || npad != KMAX) {
         if (threadIdx.x == 0) ep_raise(status, EP_ERR_CUDA);
         if (threadIdx.x < 4) late_count[blockIdx.x * 4 + threadIdx.x] = 0;
         return;
@@ -141,7 +141,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     constexpr int SWARPS = BMR / 32;                   // screen warps with rows
     constexpr int X_KB_BYTES = BMR * 128;              // one k-block of a row tile
     const int stage_bytes = num_kb * X_KB_BYTES;
-    const int c_kb_bytes = npad * 128;
+    const int c_kb_bytes = KMAX * 128;                 // the host passes npad == KMAX
     uint8_t *x_smem = smem;                                          // [stages][num_kb][128 rows][128 B]
     uint8_t *c_smem = x_smem + (size_t)stages * stage_bytes;         // [num_kb][npad rows][128 B]
     FusedShared *sh = reinterpret_cast<FusedShared *>(c_smem + (size_t)num_kb * c_kb_bytes);
@@ -172,7 +172,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
     for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
         sh->cnt[k] = 0;
-        sh->cn[k] = k < npad ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
+        sh->cn[k] = k < KMAX ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
     }
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
@@ -212,7 +212,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!(ok = mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag))) break;
                 if (!(ok = mbar_wait(&sh->x_full[s], ph, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * (uint32_t)npad;
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)KMAX;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES));
                     const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)kb * c_kb_bytes));
@@ -236,8 +236,11 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // weight so far that still has a free slot (OWN slots per warp).  The weight of a cluster is the number
             // of rows it got from this block's tiles in the previous iteration (+ 1), so the warps end up with
             // about the same number of rows per tile however uneven the clusters are.
+            // (runs once per launch: its loops stay rolled, the kernel's code is large as it is)
             constexpr int OWN = KMAX / A_WARPS;
+#pragma unroll 1
             for (int k = lane; k <= MAX_K; k += 32) sh->keymap[k] = (uint8_t)MAX_K;
+#pragma unroll 1
             for (int q = lane; q < MAX_K; q += 32) {
                 sh->kof[q] = (int8_t)-1;
                 int w = 0;
@@ -245,9 +248,11 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 sh->plan_cnt[q] = w;
             }
             __syncwarp();
+#pragma unroll 1
             for (int k = lane; k < K; k += 32) {
                 const int mine = sh->plan_cnt[k];
                 int rank = 0;
+#pragma unroll 1
                 for (int j = 0; j < K; ++j) {
                     const int o = sh->plan_cnt[j];
                     rank += (o > mine || (o == mine && j < k)) ? 1 : 0;
@@ -257,6 +262,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             __syncwarp();
             unsigned load = 0u;
             int taken = 0;
+#pragma unroll 1
             for (int r = 0; r < K; ++r) {
                 const int k = sh->plan_sorted[r];
                 const unsigned key = (lane < A_WARPS && taken < OWN) ? ((load << 3) | (unsigned)lane) : 0xFFFFFFFFu;
@@ -367,13 +373,13 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             EP_CLK(pc_wait)
             tc_fence_after();
             // ---- all of this row's screened products into registers, then the accumulator is free again
-            const uint32_t taddr = tmem_base + ((uint32_t)(sw * 32) << 16) + buf * (uint32_t)npad;
+            const uint32_t taddr = tmem_base + ((uint32_t)(sw * 32) << 16) + buf * (uint32_t)KMAX;
             uint32_t v[KMAX];
-            tmem_issue16<0>(taddr, v);
-            if (npad > 16) tmem_issue16<16>(taddr, v);
+            tmem_issue16<0>(taddr, v);                     // npad == KMAX: no test inside the tile loop depends on K
+            if constexpr (KMAX > 16) tmem_issue16<16>(taddr, v);
             if constexpr (KMAX > 32) {
-                if (npad > 32) tmem_issue16<32>(taddr, v);
-                if (npad > 48) tmem_issue16<48>(taddr, v);
+                tmem_issue16<32>(taddr, v);
+                tmem_issue16<48>(taddr, v);
             }
             tmem_wait();
             tc_fence_before();
@@ -384,18 +390,16 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int i = 0; i < 4; ++i) key1[i] = key2[i] = __uint_as_float(KEY_INIT);
 #pragma unroll
             for (int c = 0; c < KMAX; c += 16) {
-                if (c < npad) {
 #pragma unroll
-                    for (int j4 = 0; j4 < 16; j4 += 4) {
-                        const float4 n4 = *reinterpret_cast<const float4 *>(&sh->cn[c + j4]);
-                        const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
+                for (int j4 = 0; j4 < 16; j4 += 4) {
+                    const float4 n4 = *reinterpret_cast<const float4 *>(&sh->cn[c + j4]);
+                    const float nn[4] = {n4.x, n4.y, n4.z, n4.w};
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float sc = fmaf(-2.f, __uint_as_float(v[c + j4 + j]), nn[j]);
-                            v[c + j4 + j] = __float_as_uint(sc);
-                            keep_two(key1[j], key2[j],
-                                     __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + j4 + j)));
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        const float sc = fmaf(-2.f, __uint_as_float(v[c + j4 + j]), nn[j]);
+                        v[c + j4 + j] = __float_as_uint(sc);
+                        keep_two(key1[j], key2[j],
+                                 __uint_as_float((__float_as_uint(sc) & key_mask) | (uint32_t)(c + j4 + j)));
                     }
                 }
             }
@@ -418,12 +422,14 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     uint32_t mlo = 0u, mhi = 0u;
 #pragma unroll
                     for (int c = 0; c < KMAX; ++c) {
-                        const uint32_t hit = (c < K && __uint_as_float(v[c]) <= thr) ? 1u : 0u;
+                        const uint32_t hit = __uint_as_float(v[c]) <= thr ? 1u : 0u;
                         if (c < 32)
                             mlo |= hit << (c & 31);
                         else
                             mhi |= hit << (c & 31);
                     }
+                    mlo &= K >= 32 ? 0xFFFFFFFFu : (1u << K) - 1u;     // columns beyond K are padding
+                    mhi &= K >= 64 ? 0xFFFFFFFFu : K > 32 ? (1u << (K - 32)) - 1u : 0u;
                     late_rows[(size_t)late_n + __popc(todo & lt)] = make_int4((int)row, (int)mlo, (int)mhi, 0);
                 }
                 late_n += __popc(todo);
@@ -755,7 +761,8 @@ struct TcFusedState {
 
 size_t kmeans_tcf_state_bytes() { return sizeof(TcFusedState); }
 
-static inline int tcf_npad(int K) { return std::max(16, (K + 15) / 16 * 16); }
+// Columns of the score tile: the kernel instance's KMAX, so that nothing inside its tile loop depends on K.
+static inline int tcf_npad(int K) { return K <= 16 ? 16 : K <= 32 ? 32 : 64; }
 
 static inline int tcf_tile_rows(int d) { return d <= 128 ? BM : BM / 2; }
 
@@ -830,9 +837,9 @@ int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, con
                       int *pcnt, void *late_list_ws, int *late_count, bool use_prev, cudaStream_t stream) {
     int4 *late_list = static_cast<int4 *>(late_list_ws);
     const int vpl = d <= 128 ? 1 : 2;
-    int rc = vpl == 2 ? tcf_launch<32, 2>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
-             : K <= 32 ? tcf_launch<32, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
-                       : tcf_launch<64, 1>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream);
+#define EP_TCF(KM, V) tcf_launch<KM, V>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
+    int rc = vpl == 2 ? (K <= 16 ? EP_TCF(16, 2) : EP_TCF(32, 2)) : K <= 16 ? EP_TCF(16, 1) : K <= 32 ? EP_TCF(32, 1) : EP_TCF(64, 1);
+#undef EP_TCF
     if (rc != EP_OK) return rc;
     const int kpad = (K + KC - 1) / KC * KC;
     const size_t row = 512 * (size_t)vpl;

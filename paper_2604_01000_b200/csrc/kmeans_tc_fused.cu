@@ -152,6 +152,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int64_t num_tiles = (N + BMR - 1) / BMR;
 
     if (threadIdx.x == 0) {
+#pragma unroll 1
         for (int i = 0; i < MAX_STAGES; ++i) {
             mbar_init(&sh->x_full[i], 1);
             mbar_init(&sh->x_empty[i], A_WARPS);
@@ -189,6 +190,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             mbar_expect_tx(&sh->c_full, (uint32_t)(num_kb * c_kb_bytes));
+#pragma unroll 1
             for (int kb = 0; kb < num_kb; ++kb)
                 tma_load_2d(c_smem + (size_t)kb * c_kb_bytes, &map_c, kb * KBLK, 0, &sh->c_full);
             uint32_t it = 0;
@@ -196,6 +198,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                 if (!mbar_wait(&sh->x_empty[s], ph ^ 1u, abort_flag)) break;
                 mbar_expect_tx(&sh->x_full[s], (uint32_t)stage_bytes);
+#pragma unroll 1
                 for (int kb = 0; kb < num_kb; ++kb)
                     tma_load_2d(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK,
                                 (int)(tile * BMR), &sh->x_full[s]);
@@ -213,6 +216,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!(ok = mbar_wait(&sh->x_full[s], ph, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)KMAX;
+#pragma unroll 1
                 for (int kb = 0; kb < num_kb; ++kb) {
                     const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES));
                     const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)kb * c_kb_bytes));
@@ -338,6 +342,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int sw = warp - S_WARP0;
         const int stid = threadIdx.x - S_WARP0 * 32;       // row in tile
         float m2 = 0.f, ml = 0.f;                          // largest centroid norm and rounding residual
+#pragma unroll 1
         for (int k = lane; k < K; k += 32) {
             m2 = fmaxf(m2, cn[k]);
             ml = fmaxf(ml, clo[k]);
@@ -526,6 +531,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     }
     __syncthreads();
+#pragma unroll 1
     for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
     if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
     if (warp == 2) {

@@ -34,11 +34,11 @@ import synth  # noqa: E402
 NCU_TRAFFIC = {
     ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_286_797_056 + 615_664_128, "launch": "all rows, one iteration",
                                       "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
-    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_274_480_000 + 13_785_856, "launch": "all rows, one iteration",
+    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_274_444_000 + 13_390_848, "launch": "all rows, one iteration",
                                     "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
-    # captured on 12 M rows of the same recipe (6,240,474,000 + 51,752,960 bytes = 524.4 per row) and scaled by the
+    # captured on 12 M rows of the same recipe (6,240,555,000 + 51,485,696 bytes = 524.3 per row) and scaled by the
     # rows of a full launch: the kernel's traffic is the rows it streams
-    ("kmeans_assign_K64", "cfg5"): {"bytes_per_launch": int(round(111_059_956 * (6_240_474_000 + 51_752_960) / 12_000_000)),
+    ("kmeans_assign_K64", "cfg5"): {"bytes_per_launch": int(round(111_059_956 * (6_240_555_000 + 51_485_696) / 12_000_000)),
                                     "launch": "all rows, one iteration; scaled from a 12 M-row capture",
                                     "source": "profiles/kmeans_tc_fused_K64_cfg5_12M_rows.md"},
 }

@@ -32,17 +32,37 @@ def _rank(rank, world, port, out):
     out.put((rank, ms, rate))
 
 
-def test_two_ranks_agree_on_the_slowest_time_and_the_whole_job_rate():
+def _two_ranks():
+    """Runs _rank as two gloo processes; None when the rendezvous itself failed (the port was taken between
+    finding it and binding it, a rank did not come up), so that the caller can try again on another port."""
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
     port = _free_port()
     procs = [ctx.Process(target=_rank, args=(r, 2, port, out)) for r in range(2)]
     for p in procs:
         p.start()
-    got = sorted(out.get(timeout=120) for _ in procs)
+    got = []
+    try:
+        got = sorted(out.get(timeout=120) for _ in procs)
+    except Exception:
+        pass
     for p in procs:
         p.join(timeout=60)
-        assert p.exitcode == 0
+        if p.is_alive():
+            p.kill()
+            p.join()
+    if len(got) != 2 or any(p.exitcode != 0 for p in procs):
+        return None
+    return got
+
+
+def test_two_ranks_agree_on_the_slowest_time_and_the_whole_job_rate():
+    got = None
+    for _ in range(3):
+        got = _two_ranks()
+        if got is not None:
+            break
+    assert got is not None, "two gloo ranks did not come up on 127.0.0.1 in three tries"
     assert [g[1] for g in got] == [20.0, 20.0]                       # the slower rank's 20 ms on both
     assert [g[2] for g in got] == [2 * 1000 * 4 / 0.020] * 2          # both replicas' units over that time
 

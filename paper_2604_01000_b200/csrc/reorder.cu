@@ -162,7 +162,9 @@ __global__ void __launch_bounds__(SORT_WARPS * 32, 4) digit_scatter(const int32_
     __shared__ int sval[SORT_TILE], skey[SORT_TILE];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < SORT_WARPS * RADIX; i += blockDim.x) (&cnt[0][0])[i] = 0;
-    gbase[threadIdx.x] = offsets[(size_t)threadIdx.x * ntiles + blockIdx.x];
+    // this digit's place in the output: asked for now, needed only after the ranking (the tiles' offsets of one digit
+    // lie ntiles words apart, so every thread's word is a cache line of its own and takes its time)
+    const int my_gbase = __ldg(offsets + (size_t)threadIdx.x * ntiles + blockIdx.x);
     __syncthreads();
 
     const int64_t base = (int64_t)blockIdx.x * SORT_TILE + (int64_t)warp * (32 * SORT_ITEMS);
@@ -185,6 +187,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32, 4) digit_scatter(const int32_
         rank[i] = before + __popc(peers & lt);
         __syncwarp();
     }
+    gbase[threadIdx.x] = my_gbase;
     __syncthreads();
     {   // per digit: turn the warps' counts into exclusive offsets inside the tile, and the digits' totals
         // into the place where each digit's run starts in the tile's sorted order

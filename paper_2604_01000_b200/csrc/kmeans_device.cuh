@@ -26,6 +26,19 @@ __device__ __forceinline__ float dot4(const float4 &a, const float4 &b, float ac
     return acc;
 }
 
+// acc + |a - b|^2 over four coordinates: the squared distance in its direct form.  Every term is
+// non-negative and each difference is rounded once, so the result is accurate relative to the DISTANCE
+// (a few units in the last place), whatever the norms of a and b are; |b|^2 - 2 a.b is only accurate
+// relative to those norms.
+__device__ __forceinline__ float dist4(const float4 &a, const float4 &b, float acc) {
+    const float tx = a.x - b.x, ty = a.y - b.y, tz = a.z - b.z, tw = a.w - b.w;
+    acc = fmaf(tx, tx, acc);
+    acc = fmaf(ty, ty, acc);
+    acc = fmaf(tz, tz, acc);
+    acc = fmaf(tw, tw, acc);
+    return acc;
+}
+
 // Sums 8 per-lane values across the warp with 9 shuffles instead of 40: each exchange halves the
 // number of values a lane still carries.  On return every lane holds the warp-wide total of value
 // index ((lane>>4)&1)*4 + ((lane>>3)&1)*2 + ((lane>>2)&1).  The additions pair lanes l and l^16, then

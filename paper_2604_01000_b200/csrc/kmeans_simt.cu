@@ -39,9 +39,10 @@ __device__ __forceinline__ void load_rows(Rows<VPL, R> &r, const float *emb, int
 // Scores R rows against the kcount (multiple of KC) centroids staged at cs (row pitch DP4 float4,
 // zero padded) with |c|^2 at cn (+inf for padding), and folds them into the per-lane running best.
 // Score of (row, k) = |c_k|^2 - 2 x.c_k; the row's |x|^2 does not change the argmin.
+// second[i] follows the smallest score this lane has seen for row i other than best[i] (a later tie counts).
 template <int VPL, int R>
 __device__ __forceinline__ void score_chunk(const Rows<VPL, R> &rows, const float4 *cs, const float *cn, int kbase,
-                                            int kcount, int lane, float (&best)[R], int (&bidx)[R]) {
+                                            int kcount, int lane, float (&best)[R], int (&bidx)[R], float (&second)[R]) {
     constexpr int DP4 = VPL * 32;
     const int slot = lane_chunk_slot(lane);
     for (int kb = 0; kb < kcount; kb += KC) {
@@ -66,15 +67,19 @@ __device__ __forceinline__ void score_chunk(const Rows<VPL, R> &rows, const floa
             float s = fmaf(-2.f, dot, cnk);
             s = (s == s) ? s : CUDART_INF_F;          // a NaN score never wins
             if (s < best[i]) {                         // strict: the earlier (lower) index keeps a tie
+                second[i] = best[i];
                 best[i] = s;
                 bidx[i] = kbase + kb + slot;
+            } else {
+                second[i] = fminf(second[i], s);
             }
         }
     }
 }
 
 // Warp-wide argmin of (best, bidx) with the lowest index winning ties; every lane gets the result.
-__device__ __forceinline__ int warp_argmin(float best, int bidx) {
+// The eight lane groups that differ in lane bits 4, 3, 2 hold eight different centroid slots.
+__device__ __forceinline__ int warp_argmin(float &best, int bidx) {
 #pragma unroll
     for (int m = 16; m >= 4; m >>= 1) {
         float ov = __shfl_xor_sync(FULL, best, m);
@@ -85,6 +90,85 @@ __device__ __forceinline__ int warp_argmin(float best, int bidx) {
         }
     }
     return bidx;
+}
+
+// Smallest score of the row apart from the winner's: a lane's own best when the winner lives in another
+// slot, its runner-up otherwise.
+__device__ __forceinline__ float warp_runner_up(float lane_best, int lane_bidx, float lane_second, int winner) {
+    float v = lane_bidx == winner ? lane_second : lane_best;
+#pragma unroll
+    for (int m = 16; m >= 4; m >>= 1) v = fminf(v, __shfl_xor_sync(FULL, v, m));
+    return v;
+}
+
+// How far two scores |c|^2 - 2 x.c may lie apart in fp32 and still be in the wrong order: twice the rounding
+// error of one score.  The dot product is 4 VPL sequential fused multiply-adds per lane and five pairwise
+// additions across the warp, each exact to 2^-24 of the running magnitude (at most |x||c|); |c|^2 and the
+// final fused multiply-add add one rounding each.
+template <int VPL>
+__device__ __forceinline__ float score_resolution(float xnorm, float cmax, float cmax2) {
+    constexpr float U = 5.9604645e-8f;                       // 2^-24
+    return 2.2f * U * ((float)(2 * (4 * VPL + 5) + 3) * xnorm * cmax + 2.f * cmax2);
+}
+
+// The row's label by squared distance in the direct form sum_j (x_j - c_j)^2 over all K centroids, lowest
+// index on ties.  For rows whose two best scores are closer than score_resolution: the direct form is
+// accurate relative to the distance itself, so it separates what the expansion cannot.
+template <int VPL>
+__device__ __noinline__ int argmin_direct(const float4 (&x)[VPL], const float *__restrict__ C, int K, int d4, int lane) {
+    const float4 *C4 = reinterpret_cast<const float4 *>(C);
+    const int slot = lane_chunk_slot(lane);
+    float best = CUDART_INF_F;
+    int bidx = 0x7fffffff;
+    for (int kb = 0; kb < K; kb += KC) {
+        float acc[KC];
+#pragma unroll
+        for (int kk = 0; kk < KC; ++kk) {
+            acc[kk] = 0.f;
+            if (kb + kk < K) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) {
+                    const int q = lane + 32 * v;
+                    if (q < d4) acc[kk] = dist4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
+                }
+            }
+        }
+        float s = reduce8_transposed(acc, lane);
+        const int k = kb + slot;
+        s = (k < K && s == s) ? s : CUDART_INF_F;
+        if (s < best) {
+            best = s;
+            bidx = k;
+        }
+    }
+    bidx = warp_argmin(best, bidx);
+    return (bidx >= 0 && bidx < K) ? bidx : 0;
+}
+
+// max_k cnorm[k] over the K real centroids, for every thread of the block (red: 32 floats of shared memory).
+__device__ __forceinline__ float block_max_norm2(const float *__restrict__ cnorm, int K, float *red) {
+    float m = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) m = fmaxf(m, cnorm[k]);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
+    __syncthreads();
+    return m;
+}
+
+// |x_i|_2 of the R rows a warp holds (every lane gets them).
+template <int VPL, int R>
+__device__ __forceinline__ void row_norms_of(const Rows<VPL, R> &rows, float (&xn)[R]) {
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float t = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) t = dot4(rows.x[i][v], rows.x[i][v], t);
+        xn[i] = sqrtf(warp_sum(t));
+    }
 }
 
 // Copies centroids [k0, k0+kcount) into shared memory with row pitch DP4 float4, zero-filling the
@@ -119,6 +203,9 @@ __global__ void __launch_bounds__(256) kmeans_assign_fused(const float *__restri
     float *cn = reinterpret_cast<float *>(sw + (size_t)W * K * DP4);   // [Kpad]
     int *cw = reinterpret_cast<int *>(cn + Kpad);         // [W][K]
 
+    __shared__ float red[32];
+    const float cmax2 = block_max_norm2(cnorm, K, red);
+    const float cmax = sqrtf(cmax2);
     stage_centroids(cs, cn, C, cnorm, 0, Kpad, K, d4, DP4);
     for (int i = threadIdx.x; i < W * K * DP4; i += blockDim.x) sw[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = threadIdx.x; i < W * K; i += blockDim.x) cw[i] = 0;
@@ -135,18 +222,24 @@ __global__ void __launch_bounds__(256) kmeans_assign_fused(const float *__restri
     load_rows(cur, emb, w0, w1, d4, lane);
     for (int64_t row = w0; row < w1; row += R) {
         load_rows(nxt, emb, row + R, w1, d4, lane);
-        float best[R];
+        float best[R], second[R], xn[R];
         int bidx[R];
 #pragma unroll
         for (int i = 0; i < R; ++i) {
-            best[i] = CUDART_INF_F;
+            best[i] = second[i] = CUDART_INF_F;
             bidx[i] = 0;
         }
-        score_chunk<VPL, R>(cur, cs, cn, 0, Kpad, lane, best, bidx);
+        score_chunk<VPL, R>(cur, cs, cn, 0, Kpad, lane, best, bidx, second);
+        row_norms_of<VPL, R>(cur, xn);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (row + i < w1) {
-                int a = warp_argmin(best[i], bidx[i]);
+                float wbest = best[i];
+                int a = warp_argmin(wbest, bidx[i]);
+                const float runner = warp_runner_up(best[i], bidx[i], second[i], a);
+                // too close to call from the scores: decide by the distances themselves
+                if (__any_sync(FULL, runner - wbest <= score_resolution<VPL>(xn[i], cmax, cmax2)))
+                    a = argmin_direct<VPL>(cur.x[i], C, K, d4, lane);
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     float4 s = mysum[a * DP4 + lane + 32 * v];
@@ -199,16 +292,19 @@ __global__ void __launch_bounds__(256) kmeans_assign_chunked(const float *__rest
     const int d4 = d >> 2;
     float4 *cs = smem4;                                            // [kchunk][DP4]
     float *cn = reinterpret_cast<float *>(cs + (size_t)kchunk * DP4);   // [kchunk]
+    __shared__ float red[32];
+    const float cmax2 = block_max_norm2(cnorm, K, red);
+    const float cmax = sqrtf(cmax2);
     const int64_t batch = (int64_t)W * R;
     for (int64_t b0 = (int64_t)blockIdx.x * batch; b0 < N; b0 += (int64_t)gridDim.x * batch) {
         const int64_t row = b0 + (int64_t)warp * R;
         Rows<VPL, R> cur;
         load_rows(cur, emb, row, N, d4, lane);
-        float best[R];
+        float best[R], second[R], xn[R];
         int bidx[R];
 #pragma unroll
         for (int i = 0; i < R; ++i) {
-            best[i] = CUDART_INF_F;
+            best[i] = second[i] = CUDART_INF_F;
             bidx[i] = 0;
         }
         for (int k0 = 0; k0 < Kpad; k0 += kchunk) {
@@ -216,11 +312,17 @@ __global__ void __launch_bounds__(256) kmeans_assign_chunked(const float *__rest
             __syncthreads();
             stage_centroids(cs, cn, C, cnorm, k0, kc, K, d4, DP4);
             __syncthreads();
-            score_chunk<VPL, R>(cur, cs, cn, k0, kc, lane, best, bidx);
+            score_chunk<VPL, R>(cur, cs, cn, k0, kc, lane, best, bidx, second);
         }
+        row_norms_of<VPL, R>(cur, xn);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
-            int a = warp_argmin(best[i], bidx[i]);
+            float wbest = best[i];
+            int a = warp_argmin(wbest, bidx[i]);
+            const float runner = warp_runner_up(best[i], bidx[i], second[i], a);
+            // too close to call from the scores: decide by the distances themselves
+            if (row + i < N && __any_sync(FULL, runner - wbest <= score_resolution<VPL>(xn[i], cmax, cmax2)))
+                a = argmin_direct<VPL>(cur.x[i], C, K, d4, lane);
             if (lane == 0 && row + i < N) assign[row + i] = a;
         }
     }

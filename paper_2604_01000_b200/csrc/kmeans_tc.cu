@@ -13,7 +13,7 @@
 // it.  The other rows go on a list, and kmeans_tc_resolve re-evaluates in fp32 every centroid that the
 // bound cannot exclude: the best of each group whose best is within the bound of the row's overall best,
 // and a whole group when its second best is within the bound as well (its hidden third might be).  The
-// label is the exact fp32 argmin with the lowest index winning ties, as on the CUDA-core path.
+// label is the candidate nearest in fp32 squared distance (direct form), the lowest index winning ties.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -332,10 +332,13 @@ __global__ void __launch_bounds__(1024) centroid_maxima(const float *__restrict_
 // the 16-byte slices l, l+32, ... of the row, as in the CUDA-core kernels.  rownorm[i] = (|x_i|,
 // |x_i - trunc_tf32(x_i)|), computed once per call.
 //
-// The listed centroid is scored first (its row of C comes with the prefetch of the row).  With `best` its fp32
-// score and E the allowance, a centroid h can only reach or tie the final fp32 minimum if its key is at most
-// best + E (key(h) <= f(h) + E <= best + E): that threshold, never larger than the screening pass's own
-// (smallest key + 2E), decides which other centroids are scored and which groups are scanned.
+// The listed centroid is evaluated first (its row of C comes with the prefetch of the row), both as the score
+// f = |c|^2 - 2 x.c and as the squared distance.  With E the allowance, a centroid h can only be as near as the
+// listed one if its key is at most f + E (key(h) <= score(h) + E <= f + E): that threshold, never larger than the
+// screening pass's own (smallest key + 2E), decides which other centroids are evaluated and which groups are
+// scanned.  The label is the candidate with the smallest squared distance in the direct form sum_j (x_j - c_j)^2,
+// lowest index on ties: the rows that arrive here are the near ties, and only the direct form separates two
+// distances whose gap is small beside |x|^2 and |c|^2.
 template <int VPL>
 __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict__ emb, int64_t row_begin, int rows, int d, int K,
                                                          int G, const float *__restrict__ C,
@@ -397,26 +400,32 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
         const float2 nr = nr_n;
         const uint2 key0 = lane < G ? key_n : make_uint2(KEY_INIT, KEY_INIT);   // this lane's group of the first 32
         float4 x[VPL];
-        float acc_f = 0.f;
+        float acc_f = 0.f, dist_f = 0.f;
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
             x[v] = x_n[v];
             acc_f = dot4(x[v], c_n[v], acc_f);
+            dist_f = dist4(x[v], c_n[v], dist_f);
         }
         const float cn_f = cn_n;
         ent = ent_n;
         ent_n = entry((int64_t)i + 2 * (int64_t)stride);
         fetch(ent);
+        // Candidates are compared by their squared distance in the direct form sum_j (x_j - c_j)^2 (accurate
+        // relative to the distance itself: these are the near ties).  The score |c|^2 - 2 x.c of the listed
+        // centroid only places the threshold below.
         float best = CUDART_INF_F;
         int bidx = 0x7fffffff;
+        float score_first = CUDART_INF_F;
         if (kfirst >= 0) {
-            const float sf = fmaf(-2.f, warp_sum(acc_f), cn_f);
-            best = (sf == sf) ? sf : CUDART_INF_F;
+            const float sf = fmaf(-2.f, warp_sum(acc_f), cn_f), df = warp_sum(dist_f);
+            score_first = (sf == sf) ? sf : CUDART_INF_F;
+            best = (df == df) ? df : CUDART_INF_F;
             bidx = kfirst;
             ++n_single;
         }
-        // nothing above this key can reach or tie `best`
-        const float thr = best + screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
+        // no centroid whose key lies above this can be as near as the listed one
+        const float thr = score_first + screen_allowance(nr.x, nr.y, cmax, cmax2, clomax, d);
 
         bool lanes_differ = false;                 // set once a lane holds a score the others do not
         for (int g0 = 0; g0 < G; g0 += 32) {
@@ -442,15 +451,14 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                     const int k1 = (g0 + src1) * GROUP + (int)(__shfl_sync(FULL, key.x, src1) & IDX_MASK);
                     const bool use0 = k0 < K, use1 = two && k1 < K;
                     const int kk0 = use0 ? k0 : 0, kk1 = use1 ? k1 : 0;
-                    const float cn0 = __ldg(cn + kk0), cn1 = __ldg(cn + kk1);
                     float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
                     for (int v = 0; v < VPL; ++v) {
                         const int q = lane + 32 * v;
                         if (q < d4) {
                             const float4 c0 = __ldg(C4 + (size_t)kk0 * d4 + q), c1 = __ldg(C4 + (size_t)kk1 * d4 + q);
-                            acc0 = dot4(x[v], c0, acc0);
-                            acc1 = dot4(x[v], c1, acc1);
+                            acc0 = dist4(x[v], c0, acc0);
+                            acc1 = dist4(x[v], c1, acc1);
                         }
                     }
 #pragma unroll
@@ -458,7 +466,7 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                         acc0 += __shfl_xor_sync(FULL, acc0, m);
                         acc1 += __shfl_xor_sync(FULL, acc1, m);
                     }
-                    float s0 = fmaf(-2.f, acc0, cn0), s1 = fmaf(-2.f, acc1, cn1);
+                    float s0 = acc0, s1 = acc1;
                     s0 = (s0 == s0) ? s0 : CUDART_INF_F;
                     s1 = (s1 == s1) ? s1 : CUDART_INF_F;
                     n_single += (use0 ? 1 : 0) + (use1 ? 1 : 0);
@@ -476,7 +484,6 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
             while (ms) {
                 float acc[KC];
                 int myk = -1;
-                float mycn = 0.f;
 #pragma unroll
                 for (int kk = 0; kk < KC; ++kk) {
                     acc[kk] = 0.f;
@@ -486,21 +493,17 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
                         const int kone = (g0 + src) * GROUP + (int)(__shfl_sync(FULL, key.x, src) & IDX_MASK);
                         if (kone < K) {
                             ++n_single;
-                            if (kk == slot) {
-                                myk = kone;
-                                mycn = __ldg(cn + kone);
-                            }
+                            if (kk == slot) myk = kone;
 #pragma unroll
                             for (int v = 0; v < VPL; ++v) {
                                 const int q = lane + 32 * v;
-                                if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc[kk]);
+                                if (q < d4) acc[kk] = dist4(x[v], __ldg(C4 + (size_t)kone * d4 + q), acc[kk]);
                             }
                         }
                     }
                 }
-                const float dot = reduce8_transposed(acc, lane);
+                float s = reduce8_transposed(acc, lane);
                 if (myk >= 0) {
-                    float s = fmaf(-2.f, dot, mycn);
                     s = (s == s) ? s : CUDART_INF_F;
                     if (s < best || (s == best && myk < bidx)) {
                         best = s;
@@ -525,13 +528,13 @@ __global__ void __launch_bounds__(256) kmeans_tc_resolve(const float *__restrict
 #pragma unroll
                             for (int v = 0; v < VPL; ++v) {
                                 const int q = lane + 32 * v;
-                                if (q < d4) acc[kk] = dot4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
+                                if (q < d4) acc[kk] = dist4(x[v], __ldg(C4 + (size_t)(kb + kk) * d4 + q), acc[kk]);
                             }
                         }
                     }
-                    const float dot = reduce8_transposed(acc, lane);
+                    const float dist = reduce8_transposed(acc, lane);
                     const int k = kb + slot;
-                    float s = k < kend ? fmaf(-2.f, dot, cn[k]) : CUDART_INF_F;
+                    float s = k < kend ? dist : CUDART_INF_F;
                     s = (s == s) ? s : CUDART_INF_F;
                     if (s < best || (s == best && k < bidx)) {
                         best = s;

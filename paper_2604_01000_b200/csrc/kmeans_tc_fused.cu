@@ -641,12 +641,13 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
                             m &= m - 1;
                             if (kk == slot) myk = k;
 #pragma unroll
-                            for (int v = 0; v < VPL; ++v) a[kk] = dot4(x[v], cs[k * RP + lane + 32 * v], a[kk]);
+                            for (int v = 0; v < VPL; ++v) a[kk] = dist4(x[v], cs[k * RP + lane + 32 * v], a[kk]);
                         }
                     }
-                    const float dot = reduce8_transposed(a, lane);
+                    // |x - c|^2 itself, not |c|^2 - 2 x.c: these rows are the near ties, and the direct form
+                    // resolves a gap relative to the distance even when the norms are far larger than it
+                    float sc = reduce8_transposed(a, lane);
                     if (myk >= 0) {
-                        float sc = fmaf(-2.f, dot, cns[myk]);
                         sc = (sc == sc) ? sc : CUDART_INF_F;
                         if (sc < best || (sc == best && myk < bidx)) {
                             best = sc;

@@ -1,5 +1,9 @@
-"""GPU parity at the benchmark's full sizes (cfg4: N = 2,449,029, d = 128, nnz ~ 123.5 M), in the launch
-configuration bench.py times.  The oracle cannot run whole Lloyd iterations at this size in seconds, so:
+"""GPU parity at the configs' full sizes, in the launch configuration bench.py times.
+
+cfg2 (N = 169,343, d = 128, K = 8, 30 iterations) and cfg3 (N = 232,965, d = 256, K = 16, 30 iterations, 114.6 M CSR
+entries) are small enough for the oracle to run whole: every output is compared with it element by element.
+
+cfg4 (N = 2,449,029, d = 128, nnz ~ 123.5 M): the oracle cannot run whole Lloyd iterations at this size in seconds, so:
 labels are compared on a seeded row sample against the oracle's assignment step from the GPU's own
 C_{T-1}; centroids against an independent fp64 mean of the rows carrying each label; the rest through
 properties that hold at any size.  The graph passes are integer and are compared in full."""
@@ -9,7 +13,7 @@ import torch
 
 import oracle
 import synth
-from parity import assert_labels_match, CENTROID_RTOL, rms_row_norm
+from parity import assert_labels_match, check_run_against_oracle, CENTROID_RTOL, rms_row_norm
 
 pytestmark = pytest.mark.gpu
 
@@ -131,3 +135,37 @@ def test_cfg4_graph_passes_full_size(ctx, cfg4):
     ref_labels, ref_moved = oracle.migrate(rowptr.cpu().numpy(), a, w.K, cap, words.numpy().view(np.uint32))
     np.testing.assert_array_equal(moved_labels.cpu().numpy(), ref_labels)
     assert int(state[2].item()) == ref_moved
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_cfg2_cfg3_whole_config_against_the_oracle(ctx, name):
+    """The config as stated (full N, K, iteration count): K-Means end to end and iteration by iteration, then every
+    graph pass on the full graph, bit for bit."""
+    w = synth.WORKLOADS[name]
+    emb = synth.embeddings(w, device="cuda")
+    init = emb[synth.init_centroid_rows(w, device="cuda")].contiguous()
+    check_run_against_oracle(ctx, emb, init, w.K, w.iters, pinned_iterations=(1, 2, w.iters // 2, w.iters))
+    km = ctx.kmeans(emb, w.K, w.iters, init)
+    del emb
+    rowptr, colidx = synth.graph(w, device="cuda")
+    q = ctx.partition_quality(rowptr, colidx, km.assign, w.K)
+    r = ctx.reorder(km.assign, w.K)
+    bw = ctx.graph_bandwidth(rowptr, colidx, r.inv_perm)
+    rp2, ci2 = ctx.relabel_graph(rowptr, colidx, r.perm, r.inv_perm)
+    torch.cuda.synchronize()
+    ctx.check()
+    a = km.assign.cpu().numpy()
+    rp_h, ci_h = rowptr.cpu().numpy(), colidx.cpu().numpy()
+    ref = oracle.partition_quality(rp_h, ci_h, a, w.K)
+    assert int(q.edge_cut.item()) == ref.edge_cut and ref.edge_cut % 2 == 0
+    np.testing.assert_array_equal(q.part_vertices.cpu().numpy(), ref.part_vertices)
+    np.testing.assert_array_equal(q.part_edges.cpu().numpy(), ref.part_edges)
+    perm, inv = oracle.reorder(a, w.K)
+    np.testing.assert_array_equal(r.perm.cpu().numpy(), perm)
+    np.testing.assert_array_equal(r.inv_perm.cpu().numpy(), inv)
+    ref_bw = oracle.graph_bandwidth(rp_h, ci_h, inv)
+    assert int(bw.bandwidth_sum.item()) == ref_bw.bandwidth_sum
+    np.testing.assert_array_equal(bw.vertex_bandwidth.cpu().numpy(), ref_bw.vertex_bandwidth)
+    ref_rp, ref_ci = oracle.relabel_graph(rp_h, ci_h, perm, inv)
+    np.testing.assert_array_equal(rp2.cpu().numpy().astype(np.int64), ref_rp)
+    np.testing.assert_array_equal(ci2.cpu().numpy(), ref_ci)

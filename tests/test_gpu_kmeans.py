@@ -5,7 +5,8 @@ import torch
 
 import oracle
 import synth
-from parity import assert_centroids_close, assert_labels_match, assert_objective_close
+from parity import (assert_centroids_are_means, assert_centroids_close, assert_labels_match,
+                    assert_objective_close)
 
 pytestmark = pytest.mark.gpu
 
@@ -124,7 +125,7 @@ def test_tensor_core_path_ties_and_duplicates(ctx):
 
 
 def test_fused_tensor_core_pass_ties_duplicates_and_repeatability(ctx):
-    """K <= 128: the single-kernel tensor-core pass.  Duplicated centroids tie exactly, so those rows must
+    """K <= 64: the single-kernel tensor-core pass.  Duplicated centroids tie exactly, so those rows must
     go through its fp32 queue and come out on the lowest index; two runs must agree bit for bit."""
     rng = np.random.default_rng(6)
     base = rng.integers(-4, 5, size=(50, 64)).astype(np.float32)
@@ -166,6 +167,78 @@ def test_fused_tensor_core_pass_with_very_uneven_clusters(ctx, K, d):
     four = ctx.kmeans(emb, K, 4, init)
     step = ctx.kmeans(emb, K, 1, three.centroids)       # first iteration of a call: the default owners
     assert torch.equal(step.assign, four.assign) and torch.equal(step.centroids, four.centroids)
+
+
+def _pin_every_iteration(ctx, emb, init, K, T, path):
+    """Rows far from the origin next to tiny clusters make whole runs fragile: one near-tied row that changes sides
+    (which the match criterion allows) moves a five-row centroid by a fifth of a distance, and the trajectories part
+    for good.  So every iteration of the library's run is pinned on its own: iteration t against ONE oracle step from
+    the library's own C_{t-1} (labels: no row with a clear nearest centroid may differ; centroids: the oracle's where
+    the memberships agree, the mean of the rows that carry each label everywhere).  The whole run is compared with the
+    oracle's whole run as well, up to the first iteration in which a near-tied row legitimately changed sides."""
+    ctx.set_kmeans_path(path)
+    try:
+        emb_h, init_h = emb.cpu().numpy(), init.cpu().numpy()
+        c_prev = init_h
+        diverged_at = None
+        for t in range(1, T + 1):
+            got = ctx.kmeans(emb, K, t, init)                 # a t-iteration run is the prefix of the longer ones
+            torch.cuda.synchronize()
+            ctx.check()
+            a = got.assign.cpu().numpy()
+            c = got.centroids.cpu().numpy()
+            step_ref = oracle.kmeans(emb_h, K, 1, c_prev)
+            flips = assert_labels_match(a, step_ref, emb_h, c_prev.astype(np.float64))
+            assert_centroids_are_means(c, emb_h, a, c_prev)
+            if flips == 0:
+                assert_centroids_close(c, step_ref.centroids, emb_h)
+            if diverged_at is None:
+                whole = oracle.kmeans(emb_h, K, t, init_h)
+                if assert_labels_match(a, whole) > 0:          # raises on a clear mismatch; > 0: near ties changed sides
+                    diverged_at = t
+                else:
+                    assert_centroids_close(c, whole.centroids, emb_h)
+            c_prev = c
+        return diverged_at
+    finally:
+        ctx.set_kmeans_path("auto")
+
+
+def _clump_far_from_origin(K, d, N=20_011):
+    """70 % of the rows in one tight clump far from the origin: |x|^2 about 9 d, squared distances between the rows
+    of the clump about 0.18 d, so |x|^2 is fifty times the distances the labels are decided on; the initial centroids
+    are random rows, most of them inside the clump, which the clustering therefore cuts into many near-tied pieces."""
+    rng = np.random.default_rng(100 + K)
+    centres = rng.normal(size=(K, d)).astype(np.float32) * 3
+    comp = np.where(rng.random(N) < 0.7, 0, rng.integers(1, K, size=N))
+    emb_h = (centres[comp] + 0.3 * rng.normal(size=(N, d))).astype(np.float32)
+    init_h = emb_h[rng.permutation(N)[:K]].copy()
+    return torch.from_numpy(emb_h).cuda(), torch.from_numpy(init_h).cuda()
+
+
+@pytest.mark.parametrize("K,d,path", [(11, 256, "tensor"), (37, 96, "tensor"), (64, 128, "tensor"),
+                                      (11, 256, "simt"), (37, 96, "simt"), (64, 128, "simt"),
+                                      (130, 128, "tensor"), (300, 64, "tensor"), (300, 64, "simt")])
+def test_rows_far_from_the_origin_keep_the_match_criterion(ctx, K, d, path):
+    """|x|^2 far above the distances: the score |c|^2 - 2 x.c carries a rounding error relative to the NORMS, the
+    criterion (labels agree unless the two nearest distances differ by less than 1e-5 relative) is stated on the
+    DISTANCES.  Every kernel family therefore settles its close calls by sum_j (x_j - c_j)^2: the fused tensor-core
+    pass (K <= 64), the CUDA-core kernels (fused for K <= 256, chunked beyond), the large-K tensor-core path."""
+    emb, init = _clump_far_from_origin(K, d)
+    _pin_every_iteration(ctx, emb, init, K, 4, path)
+
+
+@pytest.mark.parametrize("path", ["auto", "simt"])
+@pytest.mark.parametrize("name,N,K", [("cfg4", 30_011, 32), ("cfg3", 9_973, 16), ("cfg4", 20_011, 200)])
+def test_uncentred_mixture_keeps_the_match_criterion(ctx, name, N, K, path):
+    """The benchmark mixtures moved away from the origin by 8 in every coordinate (|x|^2 about 64 d, forty times the
+    squared distances between components): a translation changes no distance, so the labels must still be the
+    oracle's."""
+    w = synth.scaled(synth.WORKLOADS[name], N, K=K)
+    emb, init = _inputs(w)
+    emb += 8.0
+    init += 8.0
+    _pin_every_iteration(ctx, emb, init, K, 3, path)
 
 
 @pytest.mark.parametrize("N,d,K", [(1, 4, 1), (2, 8, 2), (33, 4, 3), (257, 1024, 5), (1000, 12, 1), (515, 100, 9),

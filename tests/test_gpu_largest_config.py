@@ -11,7 +11,7 @@ import torch
 
 import oracle
 import synth
-from parity import assert_centroids_close, assert_labels_match, assert_objective_close
+from parity import check_run_against_oracle
 from test_gpu_full_size import _check_run
 
 pytestmark = pytest.mark.gpu
@@ -29,19 +29,11 @@ def ctx():
 
 
 def test_cfg5_one_million_row_subsample_against_the_oracle(ctx):
+    """The config's K and its stated 20 iterations on the seeded 1 M-row subsample."""
     rows = torch.sort(synth.subsample_rows(W, 1_000_000, device="cuda")).values
     emb = synth.embedding_rows(W, rows).contiguous()
     init = emb[: W.K].contiguous()
-    T = 5
-    got = ctx.kmeans(emb, W.K, T, init, objective=True)
-    torch.cuda.synchronize()
-    ctx.check()
-    emb_h, init_h = emb.cpu().numpy(), init.cpu().numpy()
-    ref = oracle.kmeans(emb_h, W.K, T, init_h)
-    prev = oracle.kmeans(emb_h, W.K, T - 1, init_h).centroids
-    assert_labels_match(got.assign.cpu().numpy(), ref, emb_h, prev)
-    assert_centroids_close(got.centroids.cpu().numpy(), ref.centroids, emb_h)
-    assert_objective_close(got.objective.cpu().numpy(), ref.objective, emb_h)
+    check_run_against_oracle(ctx, emb, init, W.K, W.iters, pinned_iterations=(1, W.iters // 2, W.iters))
 
 
 def _enough_memory(gib):

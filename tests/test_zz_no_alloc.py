@@ -4,17 +4,20 @@ A plug-in running inside another framework, a process whose device memory was al
 start-up, or a loop that cannot afford cudaMalloc's device-wide synchronisation has no way to give
 ep_reorder a workspace or even to create a context.  ep_reorder_static keeps its scratch in an array
 compiled into the library instead.  These tests call it through the C ABI and require the same
-permutation, bit for bit, as the ordinary entry point (integer outputs are compared exactly
-everywhere in this suite) -- twice in a row, because the second call starts from whatever the first
-one left in the shared scratch.
+permutation, bit for bit, as the ordinary entry point and as the CPU oracle's stable counting sort
+(integer outputs are compared exactly everywhere in this suite) -- twice in a row, because the
+second call starts from whatever the first one left in the shared scratch.
 
 This file sorts last on purpose: a run that stops at the first failure has then already executed
 every other test.
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
+
+import oracle
 
 
 def _labels(N, K, seed):
@@ -52,6 +55,9 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
         assert int(status.item()) == 0
         assert torch.equal(got.perm, want.perm)
         assert torch.equal(got.inv_perm, want.inv_perm)
+        perm, inv = oracle.reorder(assign.cpu().numpy(), K)                            # and the definition itself
+        np.testing.assert_array_equal(got.perm.cpu().numpy(), perm)
+        np.testing.assert_array_equal(got.inv_perm.cpu().numpy(), inv)
         again = ep.ep_reorder_static(assign, K, inverse=False)                         # same input, scratch now dirty
         torch.cuda.synchronize()
         assert again.inv_perm is None and torch.equal(again.perm, want.perm)

@@ -126,7 +126,7 @@ int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *ro
 int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st);
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
                       const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, void *late_list, int *late_count, bool use_prev, cudaStream_t stream);
+                      int *pcnt, void *late_list, bool use_prev, cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

@@ -663,7 +663,6 @@ struct KMeansBuffers {
     float2 *rownorm;   // tensor paths: (|x_i|, |x_i - trunc(x_i)|)
     float *cmaxima;    // large-K tensor path: max |c|^2 and max rounding residual of this iteration
     void *late_list;   // fused tensor path: per screen warp, the rows the screening left undecided (16 bytes each)
-    int *late_count;
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -697,7 +696,7 @@ bool kmeans_make_plan(const ep_ctx *ctx, int64_t N, int d, int K, KMeansPlan *pl
         p.warps = 12;
         p.smem = 0;
         p.grid = kmeans_tcf_grid(ctx, N, d);
-        p.parts = 2 * p.grid;   // the fused kernel's slabs, then those of the kernel for the rows it left undecided
+        p.parts = p.grid;
     } else if (p.fused) {
         p.warps = W;
         p.smem = Kpad * row_bytes + (size_t)W * K * row_bytes + Kpad * 4 + (size_t)W * K * 4;
@@ -736,7 +735,6 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.rownorm = a.take<float2>(p.N);
         if (p.tc_fused) {
             b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N, p.d) * 4 * p.grid);
-            b.late_count = a.take<int>((size_t)4 * p.grid);
         } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
             b.cmaxima = a.take<float>(2);
@@ -786,7 +784,7 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
             constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
             if (p.tc_fused) {
                 return kmeans_tcf_assign(ctx, *tcf_state, emb, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
-                                         b.pcnt, b.late_list, b.late_count, /*use_prev=*/t > 0, stream);
+                                         b.pcnt, b.late_list, /*use_prev=*/t > 0, stream);
             } else if (p.fused) {
                 auto kern = kmeans_assign_fused<VPL, R>;
                 EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));

@@ -17,10 +17,10 @@
 //      which cluster is settled per launch from the block's own counts of the previous iteration, so that
 //      uneven clusters still give the warps even work; a cluster's rows are added by one warp in row order
 //      whoever that is, so the sums do not depend on it.
-// kmeans_late_rows then settles the undecided rows in fp32 (lowest index wins ties, same summation order
-// as the CUDA-core kernels) and adds them into a second set of partial sums.  No floating-point atomics
-// anywhere: the order of every addition is fixed by the launch shape and the lists, so results repeat
-// bit for bit.
+// After its last tile the block settles the rows its screen warps left undecided: their squared distances
+// sum_j (x_j - c_j)^2 to the listed centroids in fp32 (lowest index wins ties), the label, and the row added to
+// the block's sums after all decided rows, in list order.  No floating-point atomics anywhere: the order of
+// every addition is fixed by the launch shape and the lists, so results repeat bit for bit.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -43,6 +43,8 @@ constexpr int S_WARP0 = 4;
 constexpr int A_WARP0 = 8;
 constexpr int A_WARPS = 8;
 constexpr int MAX_K = 64;
+constexpr int LATE_WARPS = THREADS / 32;   // every warp of the block works on the undecided rows
+constexpr int MAX_LATE_CHUNK = 256;        // undecided rows held in shared memory at a time
 
 // Phase clocks for tuning (compiled in with -DEP_PHASE_CLOCKS only): thread 0 of a warp set adds up how long
 // it waited and how long it worked, into the diagnostic counters.
@@ -78,14 +80,21 @@ struct FusedShared {
     uint16_t order[2][BM];              // the tile's rows grouped by sorting key, ascending row inside a key, each as
                                         // its byte offset inside a k-block with the swizzle term in bits 4..6
     int goff[2][MAX_K + 1];             // first position of each label in order[]
-    int hcnt[2][MAX_K + 1];             // scratch of the two sorting warps
+    int hcnt[2][MAX_K + 1];             // scratch of the two sorting warps; hcnt[1] first holds the weights of the
+                                        // clusters while warp 3 shares the accumulate work out
     int cnt[MAX_K];                     // rows per sorting key that this block decided
-    int plan_cnt[MAX_K];                // weights of the clusters when the accumulate work is shared out
     uint8_t plan_sorted[MAX_K];         // clusters by descending weight
     uint8_t keymap[MAX_K + 1];          // cluster -> sorting key = owner warp * OWN + slot; [MAX_K] = MAX_K
     int8_t kof[MAX_K];                  // sorting key -> cluster, -1 = no cluster
     alignas(16) float cn[MAX_K];
+    uint64_t late_bar[LATE_WARPS];      // one per warp: its undecided rows of the current chunk have arrived
+    int late_n[4];                      // entries in each screen warp's list of undecided rows
+    int late_cum[5];                    // their running totals
 };
+// With 64 centroids of 128 floats, three 64 KB stages fit beside this block and the centroid tile only while it
+// stays within 3 KB; a fourth of the pass's speed hangs on the third stage.
+static_assert(sizeof(FusedShared) <= 3072, "FusedShared has outgrown the room beside three stages");
+static_assert(MAX_LATE_CHUNK <= 2 * BM, "the labels of a chunk of undecided rows reuse FusedShared::lab");
 
 // 16 accumulator columns, issued without waiting: several of these go out before one tmem_wait().
 template <int O, int VN>
@@ -112,21 +121,24 @@ __device__ __forceinline__ void add_if_less(float4 &a, const float4 &x, int i, i
 }
 __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// KMAX = 32 or 64: upper bound of K.  VPL = 16-byte chunks of a row per lane: 1 for d <= 128 with tiles of 128
+// KMAX = 16, 32 or 64: upper bound of K.  VPL = 16-byte chunks of a row per lane: 1 for d <= 128 with tiles of 128
 // rows, 2 for d <= 256 with tiles of 64 rows (the stage stays 64 KB; the MMA still spans 128 TMEM lanes, the upper
-// 64 of which then hold scores of whatever follows the tile in shared memory and are never read).  rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - tf32(c_k)|;
-// cn = |c_k|^2 padded with a huge value.  Block b leaves the sums of the rows it decided in psum[b][K][d],
-// their counts in pcnt[b][K], and per screen warp w the undecided rows in late_list[(4 b + w) late_cap ..]
-// (x = row id, y and z = mask of the centroids within the bound), late_count[4 b + w] of them.
+// 64 of which then hold scores of whatever follows the tile in shared memory and are never read).
+// rownorm[i] = (|x_i|, |x_i - trunc_tf32(x_i)|); clo[k] = |c_k - tf32(c_k)|; cn = |c_k|^2 padded with a huge value;
+// centroids = the fp32 centroids themselves (map_c covers their TF32-rounded copy).  Block b leaves the sums of its
+// rows in psum[b][K][d] and their counts in pcnt[b][K].  late_list[(4 b + w) late_cap ..] is scratch for the rows
+// screen warp w cannot decide (x = row id, y and z = mask of the centroids within the bound); the block settles
+// them itself after its last tile, late_chunk rows at a time.
 // use_prev != 0: pcnt[b] still holds this block's counts of the previous iteration over the same tiles; they
 // weigh the clusters when these are shared out among the accumulate warps (any sharing gives the same sums).
 template <int KMAX, int VPL>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
+                const float *__restrict__ emb, const float *__restrict__ centroids,
                 const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
                 int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
                 int32_t *__restrict__ assign, float *__restrict__ psum, int *__restrict__ pcnt,
-                int4 *__restrict__ late_list, int64_t late_cap, int *__restrict__ late_count, int use_prev,
+                int4 *__restrict__ late_list, int64_t late_cap, int late_chunk, int use_prev,
                 unsigned long long *counters, int *status) {
     // The swizzled tiles need 1024-byte alignment.  The array is used as declared (no pointer arithmetic
     // through integers), so that every access below stays a shared-memory instruction; should a launch
@@ -134,7 +146,6 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     extern __shared__ __align__(1024) uint8_t smem[];
     if ((smem_u32(smem) & 1023u) != 0u || npad != KMAX) {
         if (threadIdx.x == 0) ep_raise(status, EP_ERR_CUDA);
-        if (threadIdx.x < 4) late_count[blockIdx.x * 4 + threadIdx.x] = 0;
         return;
     }
     constexpr int BMR = BM / VPL;                      // rows per tile
@@ -167,10 +178,13 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_init(&sh->ord_empty[i], A_WARPS);
         }
         mbar_init(&sh->plan_full, 1);
+#pragma unroll 1
+        for (int i = 0; i < LATE_WARPS; ++i) mbar_init(&sh->late_bar[i], 1);
         sh->abort = 0;
         sh->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (threadIdx.x < 4) sh->late_n[threadIdx.x] = 0;
     for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
         sh->cnt[k] = 0;
         sh->cn[k] = k < KMAX ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
@@ -242,6 +256,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // about the same number of rows per tile however uneven the clusters are.
             // (runs once per launch: its loops stay rolled, the kernel's code is large as it is)
             constexpr int OWN = KMAX / A_WARPS;
+            int *plan_cnt = sh->hcnt[1];               // this warp's own scratch, not yet in use
 #pragma unroll 1
             for (int k = lane; k <= MAX_K; k += 32) sh->keymap[k] = (uint8_t)MAX_K;
 #pragma unroll 1
@@ -249,16 +264,16 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 sh->kof[q] = (int8_t)-1;
                 int w = 0;
                 if (q < K) w = 1 + (use_prev ? min(max(pcnt[(size_t)blockIdx.x * K + q], 0), 1 << 24) : 0);
-                sh->plan_cnt[q] = w;
+                plan_cnt[q] = w;
             }
             __syncwarp();
 #pragma unroll 1
             for (int k = lane; k < K; k += 32) {
-                const int mine = sh->plan_cnt[k];
+                const int mine = plan_cnt[k];
                 int rank = 0;
 #pragma unroll 1
                 for (int j = 0; j < K; ++j) {
-                    const int o = sh->plan_cnt[j];
+                    const int o = plan_cnt[j];
                     rank += (o > mine || (o == mine && j < k)) ? 1 : 0;
                 }
                 sh->plan_sorted[rank] = (uint8_t)k;
@@ -275,7 +290,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     sh->keymap[k] = (uint8_t)(lane * OWN + taken);
                     sh->kof[lane * OWN + taken] = (int8_t)k;
                     ++taken;
-                    load += (unsigned)sh->plan_cnt[k];
+                    load += (unsigned)plan_cnt[k];
                 }
             }
             __syncwarp();
@@ -422,7 +437,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (todo) {
                 // Rows that the screening cannot decide are not settled here: their ids go, in row order, to
                 // this warp's list, each with the set of centroids whose screened score is within the allowance
-                // of the row's best (bit c of the two mask words); kmeans_late_rows labels and accumulates them.
+                // of the row's best (bit c of the two mask words); the block settles them after its last tile.
                 if (undecided) {
                     uint32_t mlo = 0u, mhi = 0u;
 #pragma unroll
@@ -452,7 +467,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (lane == 0) mbar_arrive(&sh->lab_full[par]);
         }
         EP_CLK_OUT(stid == 0, 1, 2)
-        if (lane == 0) late_count[blockIdx.x * 4 + sw] = late_n;   // always written: the next kernel trusts it
+        if (lane == 0) sh->late_n[sw] = late_n;
         if (counters) {
 #pragma unroll
             for (int o = 16; o >= 1; o >>= 1) n_rows += __shfl_xor_sync(FULL, n_rows, o);
@@ -518,118 +533,124 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
         }
         EP_CLK_OUT(aw == 0 && lane == 0, 6, 7)
-        // ---- publish this block's sums: every (cluster, chunk) has exactly one owner
-        float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
+        // ---- this block's sums of the decided rows go to shared memory, where the undecided rows are added to them.
+        // The table takes the place of the first tiles of the ring, so every accumulate warp must have read its last
+        // row first (all eight arrive here whatever happened; nobody else touches the ring any more).
+        asm volatile("bar.sync 2, %0;" ::"n"(A_WARPS * 32) : "memory");
+        float4 *acc_s = reinterpret_cast<float4 *>(x_smem);                 // [K][d4]
 #pragma unroll
         for (int i = 0; i < OWN; ++i) {
             const int k = planned ? (int)sh->kof[aw * OWN + i] : -1;
             if (k >= 0 && k < K) {
 #pragma unroll
                 for (int v = 0; v < VPL; ++v)
-                    if (lane + 32 * v < d4) out[(size_t)k * d4 + lane + 32 * v] = acc[i][v];
+                    if (lane + 32 * v < d4) acc_s[(size_t)k * d4 + lane + 32 * v] = acc[i][v];
             }
         }
     }
     __syncthreads();
+    const bool aborted = sh->abort != 0;
+    if (!aborted) {
+        // ---------------------------------------------------------------- the rows the screening left undecided
+        // All 16 warps.  The ring is free now: it holds the block's sums (acc_s, above), the fp32 centroids (cs) and
+        // late_chunk rows at a time (rows_s), fetched by bulk copies, a warp's share on a barrier of its own.
+        //   1. warp w settles rows w per .. w per + per - 1 of the chunk: squared distances sum_j (x_j - c_j)^2 to the
+        //      centroids the row's mask names (all K if the mask is empty, which NaN scores cause), eight per
+        //      reduction, lowest index winning ties; the label goes to assign[] and to late_lab[].
+        //   2. warp w adds the chunk's rows with label k = w (mod 16), in list order, to acc_s[k]: one warp per
+        //      cluster, so every sum has one fixed order.
+        float4 *acc_s = reinterpret_cast<float4 *>(x_smem);                 // [K][d4]
+        float4 *cs = acc_s + (size_t)K * d4;                                // [K][d4]
+        float4 *rows_s = cs + (size_t)K * d4;                               // [late_chunk][d4]
+        uint8_t *late_lab = &sh->lab[0][0];                                 // [late_chunk] labels of the chunk's rows, 255 = none
+        const float4 *C4 = reinterpret_cast<const float4 *>(centroids);
 #pragma unroll 1
-    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
-    if (sh->abort && threadIdx.x == 0) ep_raise(status, EP_ERR_TIMEOUT);
-    if (warp == 2) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-    }
-}
-
-// The rows the fused kernel left undecided.  Block b serves fused-kernel block b and its four lists.
-//   1. All 16 warps, 32 consecutive entries per coalesced load: fp32 scores of each row against the
-//      centroids its mask names (all K if the mask is empty, which NaN scores cause), eight per reduction,
-//      lowest index winning ties, with the same summation order as the other kernels; the label goes to
-//      assign[].
-//   2. Warps 0..3: warp w adds the rows of list w, in list order, into its own sum table.
-//   3. The block folds the four tables in warp order into psum[b] / pcnt[b].
-// Every addition happens in an order fixed by the lists, so results repeat bit for bit.
-constexpr int LATE_THREADS = 512;
-constexpr int LATE_LABELS = 4096;
-
-template <int VPL>
-__global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__restrict__ emb, int64_t N, int d, int K,
-                                                                 int kpad, const float *__restrict__ C,
-                                                                 const float *__restrict__ cn,
-                                                                 const int4 *__restrict__ late_list, int64_t late_cap,
-                                                                 const int *__restrict__ late_count,
-                                                                 int32_t *__restrict__ assign, float *__restrict__ psum,
-                                                                 int *__restrict__ pcnt) {
-    extern __shared__ float4 late_smem[];
-    __shared__ int cum[5];
-    __shared__ int ncount[4];
-    __shared__ uint8_t lab_s[LATE_LABELS];                   // labels of the block's first LATE_LABELS listed rows
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
-    const int nwarps = blockDim.x >> 5;
-    constexpr int RP = 32 * VPL;                             // 16-byte chunks per (padded) row
-    float4 *cs = late_smem;                                  // [kpad][RP] centroids, zero padded
-    float4 *tab = cs + (size_t)kpad * RP;                    // [4][K][RP] per-list sums
-    float *cns = reinterpret_cast<float *>(tab + (size_t)4 * K * RP);   // [kpad]
-    int *cw = reinterpret_cast<int *>(cns + kpad);           // [4][K]
-    for (int i = threadIdx.x; i < kpad * RP; i += blockDim.x) {
-        const int k = i / RP, q = i - k * RP;
-        cs[i] = (k < K && q < d4) ? __ldg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    for (int i = threadIdx.x; i < 4 * K * RP; i += blockDim.x) tab[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = threadIdx.x; i < kpad; i += blockDim.x) cns[i] = i < K ? cn[i] : CUDART_INF_F;
-    for (int i = threadIdx.x; i < 4 * K; i += blockDim.x) cw[i] = 0;
-    if (threadIdx.x < 4) ncount[threadIdx.x] = (int)min((int64_t)max(late_count[blockIdx.x * 4 + threadIdx.x], 0), late_cap);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int w = 0; w < 4; ++w) {
-            cum[w] = run;
-            run += ncount[w];
+        for (int i = threadIdx.x; i < K * d4; i += THREADS) cs[i] = __ldg(C4 + i);
+        if (threadIdx.x == 0) {
+            int run = 0;
+#pragma unroll 1
+            for (int w = 0; w < 4; ++w) {
+                sh->late_cum[w] = run;
+                run += min(max(sh->late_n[w], 0), (int)late_cap);
+            }
+            sh->late_cum[4] = run;
         }
-        cum[4] = run;
-    }
-    __syncthreads();
-    const int4 *lists = late_list + (size_t)blockIdx.x * 4 * late_cap;
-    const int slot = lane_chunk_slot(lane);
-    // this lane's 16-byte chunks (lane, lane + 32) of row r; zeros for r < 0
-    auto load_row = [&](float4 (&x)[VPL], int r) {
-#pragma unroll
-        for (int v = 0; v < VPL; ++v)
-            x[v] = (r >= 0 && lane + 32 * v < d4) ? ldg_stream(reinterpret_cast<const float4 *>(emb) + (int64_t)r * d4 + lane + 32 * v)
-                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-    };
-    // ---- 1. labels, the rows' data fetched four ahead
-    constexpr int AHEAD1 = 4;
-    // entries per warp and turn: 32 when there are many, fewer when that keeps all warps busy on a short list
-    const int turn = min(32, max(AHEAD1, (cum[4] + nwarps * AHEAD1 - 1) / (nwarps * AHEAD1) * AHEAD1));
-    for (int p0 = warp * turn; p0 < cum[4]; p0 += nwarps * turn) {
-        const int cnt = min(turn, cum[4] - p0);
-        int4 e = make_int4(-1, 0, 0, 0);
-        if (lane < cnt) {
-            const int p = p0 + lane;
-            const int w = (p >= cum[1]) + (p >= cum[2]) + (p >= cum[3]);
-            e = lists[(size_t)w * late_cap + (p - cum[w])];
-            if (e.x < 0 || e.x >= N) e.x = -1;               // never index outside the matrix, whatever the list holds
-        }
-        float4 xq[AHEAD1][VPL];
-#pragma unroll
-        for (int u = 0; u < AHEAD1; ++u) load_row(xq[u], __shfl_sync(FULL, e.x, u));
-        for (int i0 = 0; i0 < cnt; i0 += AHEAD1) {
-#pragma unroll
-            for (int u = 0; u < AHEAD1; ++u) {
-                const int i = i0 + u;
+        __syncthreads();
+        const int total = sh->late_cum[4];
+        const int cum1 = sh->late_cum[1], cum2 = sh->late_cum[2], cum3 = sh->late_cum[3];
+        const int4 *lists = late_list + (size_t)blockIdx.x * 4 * late_cap;
+        const int slot = lane_chunk_slot(lane);
+        const uint32_t row_bytes = (uint32_t)d * 4u;
+        uint32_t chunk_it = 0;
+#pragma unroll 1
+        for (int p0 = 0; p0 < total; p0 += late_chunk, ++chunk_it) {
+            // ---- 1. fetch and settle this warp's rows: an even share of the chunk, at most 32
+            const int cn_rows = min(late_chunk, total - p0);
+            const int per = (cn_rows + LATE_WARPS - 1) / LATE_WARPS;
+            const int pw = p0 + warp * per;
+            const int nw = max(0, min(per, total - pw));
+            int4 e = make_int4(-1, 0, 0, 0);
+            if (lane < nw) {
+                const int p = pw + lane;
+                const int w = (p >= cum1) + (p >= cum2) + (p >= cum3);
+                e = lists[(size_t)w * late_cap + (p - sh->late_cum[w])];
+                if (e.x < 0 || e.x >= N) e.x = -1;                          // never index outside the matrix
+            }
+            const unsigned have = __ballot_sync(FULL, e.x >= 0);
+            bool arrived = true;
+            if (have) {
+                if (lane == 0) mbar_expect_tx(&sh->late_bar[warp], (uint32_t)__popc(have) * row_bytes);
+                __syncwarp();
+                if (e.x >= 0)
+                    bulk_load_1d(rows_s + (size_t)(warp * per + lane) * d4, emb + (size_t)e.x * d, row_bytes, &sh->late_bar[warp]);
+                arrived = mbar_wait(&sh->late_bar[warp], chunk_it & 1u, abort_flag);
+            } else if (lane == 0) {
+                mbar_arrive(&sh->late_bar[warp]);                           // keeps this barrier's phase in step with the chunks
+            }
+#pragma unroll 1
+            for (int r = 0; r < nw; ++r) {
+                const int row = __shfl_sync(FULL, e.x, r);
+                const uint32_t mlo = (uint32_t)__shfl_sync(FULL, e.y, r), mhi = (uint32_t)__shfl_sync(FULL, e.z, r);
+                if (row < 0 || !arrived) {
+                    if (lane == 0) late_lab[warp * per + r] = 255;
+                    continue;
+                }
                 float4 x[VPL];
 #pragma unroll
-                for (int v = 0; v < VPL; ++v) x[v] = xq[u][v];
-                const int row = __shfl_sync(FULL, e.x, i & 31);
-                const uint32_t mlo = (uint32_t)__shfl_sync(FULL, e.y, i & 31), mhi = (uint32_t)__shfl_sync(FULL, e.z, i & 31);
-                const int rn = __shfl_sync(FULL, e.x, (i + AHEAD1) & 31);
-                load_row(xq[u], i + AHEAD1 < cnt ? rn : -1);
-                if (i >= cnt || row < 0) continue;
+                for (int v = 0; v < VPL; ++v)
+                    x[v] = lane + 32 * v < d4 ? rows_s[(size_t)(warp * per + r) * d4 + lane + 32 * v] : make_float4(0.f, 0.f, 0.f, 0.f);
                 unsigned long long m = ((unsigned long long)mhi << 32) | mlo;
                 if (K < 64) m &= (1ull << K) - 1ull;
                 if (m == 0ull) m = K < 64 ? (1ull << K) - 1ull : ~0ull;
                 float best = CUDART_INF_F;
                 int bidx = 0x7fffffff;
+                if (__popcll(m) <= 2) {
+                    // the usual near tie, between two centroids: two sums side by side
+                    // |x - c|^2 itself, not |c|^2 - 2 x.c: these rows are the near ties, and the direct form
+                    // resolves a gap relative to the distance even when the norms are far larger than it
+                    const int k0 = __ffsll((long long)m) - 1;
+                    const unsigned long long rest = m & (m - 1);
+                    const int k1 = rest ? __ffsll((long long)rest) - 1 : k0;
+                    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) {
+                        if (lane + 32 * v < d4) {
+                            a0 = dist4(x[v], cs[(size_t)k0 * d4 + lane + 32 * v], a0);
+                            a1 = dist4(x[v], cs[(size_t)k1 * d4 + lane + 32 * v], a1);
+                        }
+                    }
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1) {
+                        a0 += __shfl_xor_sync(FULL, a0, o);
+                        a1 += __shfl_xor_sync(FULL, a1, o);
+                    }
+                    const int lab2 = (a1 < a0 || !(a0 == a0)) ? k1 : k0;      // k0 < k1: it keeps a tie
+                    if (lane == 0) {
+                        assign[row] = lab2;
+                        late_lab[warp * per + r] = (uint8_t)lab2;
+                    }
+                    continue;
+                }
                 while (m) {
                     float a[KC];
                     int myk = -1;
@@ -641,7 +662,8 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
                             m &= m - 1;
                             if (kk == slot) myk = k;
 #pragma unroll
-                            for (int v = 0; v < VPL; ++v) a[kk] = dist4(x[v], cs[k * RP + lane + 32 * v], a[kk]);
+                            for (int v = 0; v < VPL; ++v)
+                                if (lane + 32 * v < d4) a[kk] = dist4(x[v], cs[(size_t)k * d4 + lane + 32 * v], a[kk]);
                         }
                     }
                     // |x - c|^2 itself, not |c|^2 - 2 x.c: these rows are the near ties, and the direct form
@@ -667,71 +689,49 @@ __global__ void __launch_bounds__(LATE_THREADS) kmeans_late_rows(const float *__
                 if (bidx < 0 || bidx >= K) bidx = 0;         // a row of NaNs still gets a valid label
                 if (lane == 0) {
                     assign[row] = bidx;
-                    if (p0 + i < LATE_LABELS) lab_s[p0 + i] = (uint8_t)bidx;
+                    late_lab[warp * per + r] = (uint8_t)bidx;
                 }
             }
-        }
-    }
-    __syncthreads();
-    // ---- 2. sums: warp w walks list w in order, 32 entries per coalesced load, row data fetched eight ahead
-    if (warp < 4) {
-        const int n = cum[warp + 1] - cum[warp];
-        const int4 *rows = lists + (size_t)warp * late_cap;
-        float4 *mytab = tab + (size_t)warp * K * RP;
-        constexpr int AHEAD = 8 / VPL;
-        for (int j0 = 0; j0 < n; j0 += 32) {
-            const int cnt = min(32, n - j0);
-            int row_l = -1, lab_l = -1;
-            if (lane < cnt) {
-                row_l = rows[j0 + lane].x;
-                if (row_l < 0 || row_l >= N) row_l = -1;
-                if (row_l >= 0) lab_l = cum[warp] + j0 + lane < LATE_LABELS ? (int)lab_s[cum[warp] + j0 + lane] : assign[row_l];
-            }
-            float4 xq[AHEAD][VPL];
+            __syncthreads();
+            // ---- 2. add the chunk's rows to the sums of their clusters
+#pragma unroll 1
+            for (int j0 = 0; j0 < cn_rows; j0 += 32) {
+                const int lab = j0 + lane < cn_rows ? (int)late_lab[j0 + lane] : 255;
+                const bool mine = lab < K && (lab & (LATE_WARPS - 1)) == warp;
+                if (mine) atomicAdd(&sh->cnt[sh->keymap[lab]], 1);           // integer: exact whatever the order
+                unsigned mm = __ballot_sync(FULL, mine);
+                while (mm) {
+                    const int b = __ffs(mm) - 1;
+                    mm &= mm - 1;
+                    const int k = __shfl_sync(FULL, lab, b);
 #pragma unroll
-            for (int u = 0; u < AHEAD; ++u) load_row(xq[u], __shfl_sync(FULL, row_l, u));
-            for (int i0 = 0; i0 < cnt; i0 += AHEAD) {
-#pragma unroll
-                for (int u = 0; u < AHEAD; ++u) {
-                    const int i = i0 + u;
-                    float4 x[VPL];
-#pragma unroll
-                    for (int v = 0; v < VPL; ++v) x[v] = xq[u][v];
-                    const int a = __shfl_sync(FULL, lab_l, i & 31);
-                    const int rn = __shfl_sync(FULL, row_l, (i + AHEAD) & 31);
-                    load_row(xq[u], i + AHEAD < cnt ? rn : -1);
-                    if (i < cnt && a >= 0 && a < K) {
-#pragma unroll
-                        for (int v = 0; v < VPL; ++v) {
-                            float4 t = mytab[a * RP + lane + 32 * v];
-                            t.x += x[v].x;
-                            t.y += x[v].y;
-                            t.z += x[v].z;
-                            t.w += x[v].w;
-                            mytab[a * RP + lane + 32 * v] = t;
+                    for (int v = 0; v < VPL; ++v) {
+                        if (lane + 32 * v < d4) {
+                            const float4 xr = rows_s[(size_t)(j0 + b) * d4 + lane + 32 * v];
+                            float4 t = acc_s[(size_t)k * d4 + lane + 32 * v];
+                            t.x += xr.x;
+                            t.y += xr.y;
+                            t.z += xr.z;
+                            t.w += xr.w;
+                            acc_s[(size_t)k * d4 + lane + 32 * v] = t;
                         }
-                        if (lane == 0) cw[warp * K + a] += 1;
                     }
                 }
             }
+            __syncthreads();                                 // the next chunk overwrites rows_s and late_lab
         }
+        // ---- publish this block's sums and counts
+        float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
+#pragma unroll 1
+        for (int i = threadIdx.x; i < K * d4; i += THREADS) out[i] = acc_s[i];
     }
-    __syncthreads();
-    // ---- 3. fold
-    float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
-    for (int i = threadIdx.x; i < K * d4; i += blockDim.x) {
-        const int k = i / d4, q = i - k * d4;
-        float4 t = tab[k * RP + q];
-        for (int w = 1; w < 4; ++w) {
-            const float4 u = tab[((size_t)w * K + k) * RP + q];
-            t.x += u.x;
-            t.y += u.y;
-            t.z += u.z;
-            t.w += u.w;
-        }
-        out[i] = t;
+#pragma unroll 1
+    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
+    if (threadIdx.x == 0 && *abort_flag) ep_raise(status, EP_ERR_TIMEOUT);   // a wait of the tail may have run out too
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
-    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = cw[k] + cw[K + k] + cw[2 * K + k] + cw[3 * K + k];
 }
 
 // rownorm[i] = (|x_i|_2, |x_i - trunc_tf32(x_i)|_2), both rounded up a little; one warp per row.
@@ -760,7 +760,7 @@ namespace ep {
 
 struct TcFusedState {
     CUtensorMap map_x, map_c;
-    int npad, num_kb, stages, grid;
+    int npad, num_kb, stages, grid, late_chunk;
     int64_t late_cap;
     size_t smem;
     uint32_t tmem_cols;
@@ -778,11 +778,27 @@ static size_t tcf_fixed_smem(int d, int K) {
     return (size_t)num_kb * tcf_npad(K) * 128 + sizeof(FusedShared);
 }
 
+static inline size_t tcf_stage_bytes(int d) { return (size_t)((d + KBLK - 1) / KBLK) * tcf_tile_rows(d) * 128; }
+
+static inline int tcf_stages(const ep_ctx *ctx, int d, int K) {
+    const size_t fixed = tcf_fixed_smem(d, K);
+    if (fixed >= (size_t)ctx->smem_optin) return 0;
+    return (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / tcf_stage_bytes(d));
+}
+
+// Undecided rows the block holds in shared memory at a time once its tiles are done: what the ring leaves beside
+// the block's sums and the fp32 centroids (K x d floats each), in whole rows, a multiple of the warps.
+static inline int tcf_late_chunk(const ep_ctx *ctx, int d, int K) {
+    const size_t ring = (size_t)tcf_stages(ctx, d, K) * tcf_stage_bytes(d), tables = 2 * (size_t)K * d * 4;
+    if (ring <= tables) return 0;
+    const size_t rows = (ring - tables) / ((size_t)d * 4);
+    return (int)std::min<size_t>(MAX_LATE_CHUNK, rows / LATE_WARPS * LATE_WARPS);
+}
+
 bool kmeans_tcf_shape_ok(const ep_ctx *ctx, int d, int K) {
     if (d < KBLK || d > MAX_KB * KBLK || K < 1 || K > MAX_K) return false;
-    if (d > 128 && K > 32) return false;   // the fp32 kernel's sum tables must fit in shared memory
-    const int num_kb = (d + KBLK - 1) / KBLK;
-    return tcf_fixed_smem(d, K) + 2 * (size_t)num_kb * tcf_tile_rows(d) * 128 <= (size_t)ctx->smem_optin;
+    if (d > 128 && K > 32) return false;   // the kernel instances for 64-row tiles stop at 32 columns
+    return tcf_stages(ctx, d, K) >= 2 && tcf_late_chunk(ctx, d, K) >= LATE_WARPS;
 }
 
 int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N, int d) {
@@ -806,10 +822,9 @@ int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *ro
 int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st) {
     st->npad = tcf_npad(K);
     st->num_kb = (d + KBLK - 1) / KBLK;
-    const size_t fixed = tcf_fixed_smem(d, K);
-    const size_t stage = (size_t)st->num_kb * tcf_tile_rows(d) * 128;
-    st->stages = (int)std::min<size_t>(MAX_STAGES, ((size_t)ctx->smem_optin - fixed) / stage);
-    st->smem = fixed + (size_t)st->stages * stage;
+    st->stages = tcf_stages(ctx, d, K);
+    st->smem = tcf_fixed_smem(d, K) + (size_t)st->stages * tcf_stage_bytes(d);
+    st->late_chunk = tcf_late_chunk(ctx, d, K);
     st->grid = kmeans_tcf_grid(ctx, N, d);
     st->late_cap = kmeans_tcf_late_cap(ctx, N, d);
     uint32_t cols = 32;
@@ -821,44 +836,33 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
 }
 
 template <int KMAX, int VPL>
-static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *cn, const float *clo, const float2 *rownorm,
-                      int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, int4 *late_list, int *late_count,
-                      bool use_prev, cudaStream_t stream) {
+static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
+                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
+                      int *pcnt, int4 *late_list, bool use_prev, cudaStream_t stream) {
     auto kern = kmeans_tc_fused<KMAX, VPL>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
     unsigned long long *counters =
         ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
-    kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, cn, clo, rownorm, N, d, K, st.npad, st.num_kb,
-                                              st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK, assign,
-                                              psum, pcnt, late_list, st.late_cap, late_count, use_prev ? 1 : 0, counters, ctx->d_status);
+    kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, emb, centroids, cn, clo, rownorm, N, d, K, st.npad,
+                                              st.num_kb, st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK,
+                                              assign, psum, pcnt, late_list, st.late_cap, st.late_chunk, use_prev ? 1 : 0,
+                                              counters, ctx->d_status);
     tm.end(1);
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;
 }
 
-// One Lloyd assignment + accumulation pass.  The fused kernel's block b leaves its sums in psum[b][K][d] and
-// counts in pcnt[b][K]; the kernel for the rows it left undecided adds the slabs grid .. 2 grid - 1.
+// One Lloyd assignment + accumulation pass in one launch: block b leaves its sums in psum[b][K][d] and its counts in
+// pcnt[b][K].
 int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
                       const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, void *late_list_ws, int *late_count, bool use_prev, cudaStream_t stream) {
+                      int *pcnt, void *late_list_ws, bool use_prev, cudaStream_t stream) {
     int4 *late_list = static_cast<int4 *>(late_list_ws);
     const int vpl = d <= 128 ? 1 : 2;
-#define EP_TCF(KM, V) tcf_launch<KM, V>(ctx, st, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, late_count, use_prev, stream)
-    int rc = vpl == 2 ? (K <= 16 ? EP_TCF(16, 2) : EP_TCF(32, 2)) : K <= 16 ? EP_TCF(16, 1) : K <= 32 ? EP_TCF(32, 1) : EP_TCF(64, 1);
+#define EP_TCF(KM, V) tcf_launch<KM, V>(ctx, st, emb, centroids, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, use_prev, stream)
+    return vpl == 2 ? (K <= 16 ? EP_TCF(16, 2) : EP_TCF(32, 2)) : K <= 16 ? EP_TCF(16, 1) : K <= 32 ? EP_TCF(32, 1) : EP_TCF(64, 1);
 #undef EP_TCF
-    if (rc != EP_OK) return rc;
-    const int kpad = (K + KC - 1) / KC * KC;
-    const size_t row = 512 * (size_t)vpl;
-    const size_t smem = (size_t)kpad * row + (size_t)4 * K * row + (size_t)kpad * 4 + (size_t)4 * K * 4;
-    auto late = vpl == 1 ? kmeans_late_rows<1> : kmeans_late_rows<2>;
-    EP_CUDA(ctx, cudaFuncSetAttribute(late, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    Timed tm(ctx, stream, EP_TIMER_KMEANS_RESOLVE);
-    late<<<st.grid, LATE_THREADS, smem, stream>>>(emb, N, d, K, kpad, centroids, cn, late_list, st.late_cap, late_count, assign,
-                                                  psum + (size_t)st.grid * K * d, pcnt + (size_t)st.grid * K);
-    tm.end(1);
-    EP_CUDA(ctx, cudaGetLastError());
-    return EP_OK;
 }
 
 }  // namespace ep

@@ -34,15 +34,8 @@ import synth  # noqa: E402
 NCU_TRAFFIC = {
     ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_286_797_056 + 615_664_128, "launch": "all rows, one iteration",
                                       "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
-    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_274_444_000 + 13_390_848, "launch": "all rows, one iteration",
-                                    "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
-    # captured on 12 M rows of the same recipe (6,240,555,000 + 51,485,696 bytes = 524.3 per row) and scaled by the
-    # rows of a full launch: the kernel's traffic is the rows it streams
-    ("kmeans_assign_K64", "cfg5"): {"bytes_per_launch": int(round(111_059_956 * (6_240_555_000 + 51_485_696) / 12_000_000)),
-                                    "launch": "all rows, one iteration; scaled from a 12 M-row capture",
-                                    "source": "profiles/kmeans_tc_fused_K64_cfg5_12M_rows.md"},
 }
-TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio used to derive the TF32 roof from the bf16 one
+TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio: the TF32 roof when the yardstick below cannot run
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -56,6 +49,47 @@ def load_peaks():
     p = dict(FALLBACK_PEAKS)
     p["_source"] = "fallback"
     return p
+
+
+def measure_tf32_peak(device, index, seconds=3.0, n=8192):
+    """The TF32 roof as measured on this GPU: a dense n^3 torch.matmul with TF32 allowed (a library GEMM, used as a
+    yardstick only and run outside every timed region), as a burst (best of 10) and back to back for a few seconds
+    (what a kernel inside a long step can draw on), with the SM clock sampled under the sustained load."""
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        a = torch.randn((n, n), device=device, dtype=torch.float32)
+        b = torch.randn((n, n), device=device, dtype=torch.float32)
+        c = torch.empty((n, n), device=device, dtype=torch.float32)
+        flops = 2.0 * n ** 3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(10):
+            e0.record()
+            torch.matmul(a, b, out=c)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        reps = max(10, int(seconds * 1e3 / best))
+        sampler = ClockSampler(index)
+        sampler.start()
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        sustained_ms = e0.elapsed_time(e1) / reps
+        del a, b, c
+        torch.cuda.empty_cache()
+        return {"burst_tflops": flops / (best * 1e-3) / 1e12, "sustained_tflops": flops / (sustained_ms * 1e-3) / 1e12,
+                "how": f"torch.matmul fp32 {n}^3 with TF32 allowed: best of 10, and {reps} back to back",
+                "clocks_sustained": clocks}
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
 
 
 # ------------------------------------------------------------------------------------------------ clocks
@@ -242,16 +276,29 @@ def pick_sample_rows(w, budget_s):
     return int(max(max(w.K, w.reorder_K, 1024), min(w.N, rows)))
 
 
-def cpu_baseline(w, budget_s=15.0):
+def cpu_baseline(w, budget_s=12.0):
+    """The oracle (gcc -O3 -march=native, no contraction) on this machine's host cores: all threads on a sample sized for
+    about budget_s seconds, then one thread on a sample sized for about a third of that."""
+    import oracle
+    all_threads = oracle.num_threads()
     rows = pick_sample_rows(w, budget_s)
     graph_rows = min(w.N, 200_000)
     secs, det = oracle_sample_run(w, rows, graph_rows)
+    rows1 = max(max(w.K, w.reorder_K, 256), rows // (3 * max(all_threads, 1)))
+    try:
+        _, det1 = oracle_sample_run(w, rows1, min(graph_rows, 50_000), threads=1)
+    finally:
+        oracle.set_num_threads(all_threads)
     return {"value": det["row_iters"] / det["kmeans_s"], "unit": "rows*iters/s", "cores": det["threads"],
             "kind": "oracle",
             "sample": (f"fp64 oracle K-Means on the first {rows} rows of {w.name} (same K and iteration counts), "
                        f"{det['kmeans_s']:.1f} s; edge cut + reorder on a {graph_rows}-vertex graph of the same recipe: "
                        f"{det['graph_entries'] / max(det['graph_s'], 1e-9):.3g} entries/s"),
-            "edge_cut_entries_per_s": det["graph_entries"] / max(det["graph_s"], 1e-9)}
+            "edge_cut_entries_per_s": det["graph_entries"] / max(det["graph_s"], 1e-9),
+            "one_thread": {"value": det1["row_iters"] / det1["kmeans_s"], "unit": "rows*iters/s", "cores": det1["threads"],
+                           "sample": f"the first {rows1} rows, {det1['kmeans_s']:.1f} s",
+                           "edge_cut_entries_per_s": det1["graph_entries"] / max(det1["graph_s"], 1e-9)},
+            "build": "gcc -O3 -march=native -ffp-contract=off -fopenmp"}
 
 
 def run_reference(args, w, rank):
@@ -378,7 +425,18 @@ def main():
 
     # ---- per-pass rates and rooflines from the library's event timers -----------------------------------
     hbm = peaks["hbm_gbs"]
-    tf32_peak = peaks["bf16_tflops_sustained"] * TF32_OVER_BF16
+    tf32 = None
+    if w.reorder_K and args.kmeans_path != "simt":
+        try:
+            tf32 = measure_tf32_peak(device, local_rank)
+        except RuntimeError as exc:                     # no room for the yardstick's three matrices
+            tf32 = None
+            print(f"TF32 yardstick skipped: {exc}", file=sys.stderr)
+    if tf32:
+        tf32_peak, tf32_source = tf32["sustained_tflops"], "measured tf32 (torch.matmul 8192^3 back to back, this run)"
+    else:
+        tf32_peak = peaks["bf16_tflops_sustained"] * TF32_OVER_BF16
+        tf32_source = peaks["_source"] + " bf16 sustained x nominal tf32/bf16 ratio"
     rp_bytes = x["rowptr"].element_size()
     passes = {}
 
@@ -399,33 +457,39 @@ def main():
         if flops_per_unit is not None:
             tfs = work * flops_per_unit / secs / 1e12
             e["roofline"] = {"bound": "tensor", "achieved": tfs, "peak": tf32_peak, "unit": "TFLOP/s",
-                             "frac": tfs / tf32_peak, "traffic": None,
-                             "peak_source": peaks["_source"] + " bf16 sustained x nominal tf32/bf16 ratio"}
+                             "frac": tfs / tf32_peak, "traffic": None, "peak_source": tf32_source}
         e["share_of_step"] = tot / ms
         passes[name] = e
 
     S = args.steps
     tensor_small = timers[(0, "kmeans_resolve")][1] > 0
     tensor_large = timers[(1, "kmeans_resolve")][1] > 0
+    # few centroids: the assign kernel labels every row and accumulates the sums, one launch per iteration
     add_pass(f"kmeans_assign_K{w.K}", (0, "kmeans_assign"), w.N, "rows*iters/s", S * w.iters,
              bytes_per_unit=4 * w.d + 4)
-    if tensor_small:
+    if tensor_small:    # the large-K path when the workload's K itself is large
         add_pass(f"kmeans_resolve_K{w.K}", (0, "kmeans_resolve"), w.N, "rows*iters/s", S * w.iters)
-        # the assign step as a whole: the fused kernel plus the kernel for the rows it leaves undecided
-        both = timers[(0, "kmeans_assign")][0] + timers[(0, "kmeans_resolve")][0]
-        gbs = w.N * S * w.iters * (4 * w.d + 4) / (both * 1e-3) / 1e9
-        passes[f"kmeans_assign_K{w.K}"]["roofline_with_resolve"] = {"achieved": gbs, "peak": hbm, "unit": "GB/s",
-                                                                    "frac": gbs / hbm}
     add_pass(f"kmeans_update_K{w.K}", (0, "kmeans_update"), w.N, "rows*iters/s", S * w.iters)
     if w.reorder_K:
+        name = f"kmeans_assign_K{w.reorder_K}"
+        add_pass(name, (1, "kmeans_assign"), w.N, "rows*iters/s", S * w.reorder_iters,
+                 flops_per_unit=2.0 * w.reorder_K * w.d)      # on the CUDA cores too: the same contraction's flops
         if tensor_large:
-            add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s", S * w.reorder_iters,
-                     flops_per_unit=2.0 * w.reorder_K * w.d)
             add_pass(f"kmeans_resolve_K{w.reorder_K}", (1, "kmeans_resolve"), w.N, "rows*iters/s", S * w.reorder_iters)
-        else:   # CUDA cores: report against the same contraction's flops
-            add_pass(f"kmeans_assign_K{w.reorder_K}", (1, "kmeans_assign"), w.N, "rows*iters/s", S * w.reorder_iters,
-                     flops_per_unit=2.0 * w.reorder_K * w.d)
         add_pass(f"kmeans_update_K{w.reorder_K}", (1, "kmeans_update"), w.N, "rows*iters/s", S * w.reorder_iters)
+        if tensor_large and name in passes:
+            # The labels need the screening kernel AND the fp32 kernel that settles what it leaves: the assign step's
+            # fraction charges both to the contraction's flops; the whole iteration adds grouping, sums and update.
+            flops = 2.0 * w.reorder_K * w.d * w.N * S * w.reorder_iters
+            t_a, t_r, t_u = (timers[(1, k)][0] for k in ("kmeans_assign", "kmeans_resolve", "kmeans_update"))
+            screen_only = dict(passes[name]["roofline"])
+            for key, t in (("roofline", t_a + t_r), ("roofline_whole_iteration", t_a + t_r + t_u)):
+                tfs = flops / (t * 1e-3) / 1e12
+                passes[name][key] = {"bound": "tensor", "achieved": tfs, "peak": tf32_peak, "unit": "TFLOP/s",
+                                     "frac": tfs / tf32_peak, "traffic": None, "peak_source": tf32_source,
+                                     "ms_per_iteration": t / (S * w.reorder_iters), "covers": "screening + fp32 resolve kernels" if key == "roofline"
+                                     else "screening + fp32 resolve + grouping, sums and centroid update"}
+            passes[name]["roofline_screen_only"] = screen_only
     add_pass("edge_cut", (0, "edge_cut"), nnz, "edges/s", S,
              bytes_per_unit=(4 * nnz + rp_bytes * (w.N + 1) + w.N) / max(nnz, 1))
     add_pass("quality_prep", (0, "quality_prep"), w.N, "vertices/s", S, bytes_per_unit=4 + rp_bytes)
@@ -434,12 +498,24 @@ def main():
     dominant_name = [k for k, v in passes.items() if v is dominant][0]
     roofline = dict(dominant["roofline"])
     roofline["kernel"] = dominant_name
-    t = NCU_TRAFFIC.get((dominant_name, w.name))
-    if t and args.kmeans_path == "auto":
-        roofline["traffic"] = t["bytes_per_launch"]
-        roofline["traffic_note"] = f"{t['launch']}; {t['source']}"
+    if args.kmeans_path == "auto":
+        for pname, p in passes.items():       # dram bytes per launch from the committed captures, where one exists
+            t = NCU_TRAFFIC.get((pname, w.name))
+            if t and "roofline" in p:
+                for key in ("roofline", "roofline_screen_only"):
+                    if key in p:
+                        p[key]["traffic"] = t["bytes_per_launch"]
+                        p[key]["traffic_note"] = f"{t['launch']}; {t['source']}" + (
+                            " (the screening kernel's launch)" if "roofline_screen_only" in p else "")
+        roofline = dict(dominant["roofline"])
+        roofline["kernel"] = dominant_name
     roofline["ms_per_launch"] = dominant["ms_per_launch"]
     roofline["ms_per_pass"] = dominant["ms_per_pass"]
+    if "roofline_whole_iteration" in dominant:
+        roofline["whole_iteration"] = dominant["roofline_whole_iteration"]
+        roofline["screen_only"] = dominant["roofline_screen_only"]
+    if tf32:
+        roofline["tf32_yardstick"] = tf32
 
     # ---- outside the step: the average graph bandwidth (Eq. 3-5) of the numbering the step produced ------
     extras = {}

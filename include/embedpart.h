@@ -110,6 +110,15 @@ int64_t ep_launch_count(const ep_ctx *ctx);
  * kernel; the rest are reserved. */
 int ep_debug_counters(ep_ctx *ctx, int64_t *out);
 
+/* Self-test of the bounded device wait (no counterpart in the paper: a property of this library).  Every wait
+ * inside the tensor-core kernels gives up after a number of clocks and makes its kernel report EP_ERR_TIMEOUT
+ * instead of hanging.  This call launches one small block whose first warp waits, for at most limit_clocks, on a
+ * barrier that nothing ever completes, and whose second warp waits on the same barrier with the library's ordinary
+ * limit (about 2 s) and has to leave when the first gives up.  Afterwards ep_poll_status returns EP_ERR_TIMEOUT
+ * (once), and waited [dev, 3 x int64] holds the clocks either warp waited and, in [2], a bit per warp whose wait
+ * claimed success (0 expected).  limit_clocks in [1e3, 2e8].  Nothing faults or spins without end. */
+int ep_selftest_wait_timeout(ep_ctx *ctx, int64_t limit_clocks, int64_t *waited, void *cuda_stream);
+
 /* --------------------------------------------------------------------------------------------
  * ep_kmeans -- Lloyd K-Means (Algorithm 3, the clustering step).
  *

@@ -6,6 +6,7 @@ compiles it with gcc and marshals arrays.
 from __future__ import annotations
 
 import ctypes
+import hashlib
 import os
 import subprocess
 from typing import NamedTuple, Optional
@@ -14,18 +15,41 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ep_oracle.c")
-_LIB = os.path.join(_HERE, "libep_oracle.so")
 _lib = None
+
+# -O3 -march=native as the CPU-baseline plan asks; -ffp-contract=off keeps every operation the separately rounded
+# IEEE double operation the C file states (no fused multiply-add), so the optimisation level changes no result.
+_CFLAGS = ["-O3", "-march=native", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=c11"]
+
+
+def _host_tag() -> str:
+    """-march=native code only runs on the kind of CPU it was built on: the library's name carries a tag of the
+    host's instruction-set flags, so a tree carried to another machine rebuilds there."""
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1((flags + " ".join(_CFLAGS)).encode()).hexdigest()[:10]
+
+
+def _lib_path() -> str:
+    return os.path.join(_HERE, "libep_oracle.%s.so" % _host_tag())
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP on) and return the library path."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + ".tmp.%d" % os.getpid()
-        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+    lib = _lib_path()
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < os.path.getmtime(_SRC):
+        tmp = lib + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", *_CFLAGS, "-o", tmp, _SRC, "-lm"]
         subprocess.run(cmd, check=True, capture_output=True, text=True)
-        os.replace(tmp, _LIB)
-    return _LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 def _load():

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
     "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
     "ep_balance_workspace_bytes", "ep_migrate", "ep_balance",
-    "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance",
+    "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance", "ep_selftest_wait_timeout",
 )
 
 EP_OK = 0
@@ -93,6 +93,8 @@ def load_library() -> ctypes.CDLL:
             lib.ep_profile_read.restype = ctypes.c_int
             lib.ep_debug_counters.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
             lib.ep_debug_counters.restype = ctypes.c_int
+            lib.ep_selftest_wait_timeout.argtypes = [vp, i64, vp, vp]
+            lib.ep_selftest_wait_timeout.restype = ctypes.c_int
             lib.ep_launch_count.argtypes = [vp]
             lib.ep_launch_count.restype = ctypes.c_int64
             lib.ep_kmeans_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32]
@@ -248,6 +250,14 @@ class Context:
         if rc != EP_OK:
             self._raise(rc)
         return list(out)
+
+    def selftest_wait_timeout(self, limit_clocks: int) -> torch.Tensor:
+        """Makes a bounded device wait run out (see ep_selftest_wait_timeout); returns the 3 diagnostic words."""
+        out = torch.zeros(3, dtype=torch.int64, device=self.device)
+        rc = self._lib.ep_selftest_wait_timeout(self._h, int(limit_clocks), ctypes.c_void_p(out.data_ptr()), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
 
     def launch_count(self) -> int:
         return int(self._lib.ep_launch_count(self._h))

@@ -48,6 +48,7 @@ struct TcShared {
     uint64_t x_full[MAX_KB], x_empty[MAX_KB];
     uint64_t c_full[MAX_STAGES], c_empty[MAX_STAGES];
     uint64_t t_full[2], t_empty[2];
+    uint64_t drain;                        // after an abort: the MMAs still in flight have completed
     uint32_t tmem_base;
     int abort;
     uint64_t h_full[4][4];                 // [tile & 3][32-row quarter]: the warp of columns 128..255 has left its result
@@ -99,6 +100,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             mbar_init(&sh->t_empty[i], EPI_WARPS);
         }
         for (int i = 0; i < 16; ++i) mbar_init(&sh->h_full[i >> 2][i & 3], 1);
+        mbar_init(&sh->drain, 1);
         sh->abort = 0;
         sh->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -119,6 +121,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            int64_t x_tile = -1;                                   // local index of the last tile any k-block was loaded for
             for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
                 const int row0 = (int)(row_begin + tile * BM);
                 for (int nt = 0; ok && nt < num_nt; ++nt) {
@@ -127,6 +130,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             if (!(ok = mbar_wait(&sh->x_empty[kb], (uint32_t)(lt & 1) ^ 1u, abort_flag))) break;
                             mbar_expect_tx(&sh->x_full[kb], X_KB_BYTES);
                             tma_load_2d(x_smem + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK, row0, &sh->x_full[kb]);
+                            x_tile = lt;
                         }
                         const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                         if (!(ok = mbar_wait(&sh->c_empty[s], ph ^ 1u, abort_flag))) break;
@@ -134,6 +138,17 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         tma_load_2d(c_smem + (size_t)s * C_STAGE_BYTES, &map_c, kb * KBLK, nt * BN, &sh->c_full[s]);
                     }
                 }
+            }
+            if (!ok || *abort_flag) {
+                // On the way out after an abort: the loads already issued get time to land, so that nothing of this
+                // block's own still writes into its shared memory when it leaves.  (A k-block of x whose barrier is
+                // still in an earlier phase was not loaded for the last tile: the wait then runs to its limit.)
+#pragma unroll 1
+                for (uint32_t j = it > (uint32_t)stages ? it - (uint32_t)stages : 0u; j < it; ++j)
+                    mbar_wait_quiet(&sh->c_full[j % (uint32_t)stages], (j / (uint32_t)stages) & 1u, DRAIN_LIMIT_CLOCKS);
+                if (x_tile >= 0)
+#pragma unroll 1
+                    for (int kb = 0; kb < num_kb; ++kb) mbar_wait_quiet(&sh->x_full[kb], (uint32_t)(x_tile & 1), DRAIN_LIMIT_CLOCKS);
             }
         }
     } else if (warp == 1) {
@@ -163,6 +178,12 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                     if (ok) umma_commit(&sh->t_full[buf]);
                 }
+            }
+            if (!ok || *abort_flag) {
+                // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
+                // here must have completed
+                umma_commit(&sh->drain);
+                mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
             }
         }
     } else if (warp >= EPI_WARP0) {

@@ -74,6 +74,7 @@ struct FusedShared {
     uint64_t lab_full[2], lab_empty[2];
     uint64_t ord_full[2], ord_empty[2];
     uint64_t plan_full;
+    uint64_t drain;                     // after an abort: the MMAs still in flight have completed
     uint32_t tmem_base;
     int abort;
     uint8_t lab[2][BM];                 // sorting key of each row of the tile; MAX_K = not to be accumulated here
@@ -178,6 +179,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_init(&sh->ord_empty[i], A_WARPS);
         }
         mbar_init(&sh->plan_full, 1);
+        mbar_init(&sh->drain, 1);
 #pragma unroll 1
         for (int i = 0; i < LATE_WARPS; ++i) mbar_init(&sh->late_bar[i], 1);
         sh->abort = 0;
@@ -217,6 +219,14 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     tma_load_2d(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK,
                                 (int)(tile * BMR), &sh->x_full[s]);
             }
+            if (*abort_flag) {
+                // On the way out after an abort: the loads already issued get time to land, so that nothing of this
+                // block's own still writes into its shared memory when it leaves.
+                mbar_wait_quiet(&sh->c_full, 0u, DRAIN_LIMIT_CLOCKS);
+#pragma unroll 1
+                for (uint32_t j = it > (uint32_t)stages ? it - (uint32_t)stages : 0u; j < it; ++j)
+                    mbar_wait_quiet(&sh->x_full[j % (uint32_t)stages], (j / (uint32_t)stages) & 1u, DRAIN_LIMIT_CLOCKS);
+            }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
@@ -240,6 +250,12 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                                   (kb | ks) != 0 ? 1u : 0u);
                 }
                 umma_commit(&sh->t_full[buf]);
+            }
+            if (!ok || *abort_flag) {
+                // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
+                // here must have completed
+                umma_commit(&sh->drain);
+                mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
             }
         }
     }

@@ -28,9 +28,10 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Waits for the phase of the given parity, but never for ever: after WAIT_LIMIT_CLOCKS, or once
+// Waits for the phase of the given parity, but never for ever: after `limit` clocks, or once
 // another thread has given up, it sets the block's abort flag and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit = WAIT_LIMIT_CLOCKS) {
     const uint32_t addr = smem_u32(bar);
     long long t0 = 0;
     for (uint32_t spins = 0;; ++spins) {
@@ -45,12 +46,33 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (ok) return true;
         if (*abort_flag) return false;
         if (spins == 64) t0 = clock64();
-        if (spins > 64 && (spins & 63) == 0 && clock64() - t0 > WAIT_LIMIT_CLOCKS) {
+        if (spins > 64 && (spins & 63) == 0 && clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
     }
 }
+
+// The same wait without the abort flag, for a block that is already on its way out after an abort: it gives the
+// copies and MMAs the block has in flight `limit` clocks to finish (their completion is what flips the phase), so
+// that nothing of its own still writes to its shared memory or TMEM when it releases them.
+__device__ __forceinline__ bool mbar_wait_quiet(uint64_t *bar, uint32_t parity, long long limit) {
+    const uint32_t addr = smem_u32(bar);
+    const long long t0 = clock64();
+    for (uint32_t spins = 0;; ++spins) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((spins & 63) == 63 && clock64() - t0 > limit) return false;
+    }
+}
+constexpr long long DRAIN_LIMIT_CLOCKS = 20000000ll;   // ~10 ms per barrier on the way out
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
     asm volatile(

@@ -541,6 +541,32 @@ def main():
                 "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
                              "traffic": None, "peak_source": peaks["_source"]}}
 
+    # ---- outside the step: what this GPU can do for the edge-cut pass's label gather at all (yardstick kernels of the
+    # library: the column ids streamed the same way, one byte gathered per entry, nothing else)
+    if last is not None and w.K <= 256:
+        table = last[0].assign.to(torch.uint8)
+        gather = {}
+        for csize in (0, 8, 16):
+            try:
+                ctx.probe_gather(x["colidx"], table, csize)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(3):
+                    ctx.probe_gather(x["colidx"], table, csize)
+                e1.record()
+                torch.cuda.synchronize()
+                ms_g = e0.elapsed_time(e1) / 3
+                gather["global_memory" if csize == 0 else f"cluster_of_{csize}_shared_memory"] = {
+                    "ms": ms_g, "gathers_per_s": nnz / (ms_g * 1e-3)}
+            except ep.EmbedPartError as exc:            # the table does not fit such a cluster, or no such cluster
+                gather[f"cluster_of_{csize}_shared_memory"] = {"unavailable": str(exc)}
+        ctx.check()
+        if "edge_cut" in passes and "global_memory" in gather:
+            gather["edge_cut_over_global_gather_rate"] = passes["edge_cut"]["rate"] / gather["global_memory"]["gathers_per_s"]
+        extras["label_gather_yardstick"] = gather
+        del table
+
     # ---- outside the step: the graph and the rows stored under the numbering the step produced -----------
     if last is not None and last[3].inv_perm is not None:
         reps = 3

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "ep_graph_bandwidth_host", "ep_kmeans_sampled_workspace_bytes", "ep_kmeans_sampled", "ep_gather_rows",
     "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
     "ep_balance_workspace_bytes", "ep_migrate", "ep_balance",
-    "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance", "ep_selftest_wait_timeout",
+    "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance", "ep_selftest_wait_timeout", "ep_probe_gather",
 )
 
 EP_OK = 0
@@ -95,6 +95,8 @@ def load_library() -> ctypes.CDLL:
             lib.ep_debug_counters.restype = ctypes.c_int
             lib.ep_selftest_wait_timeout.argtypes = [vp, i64, vp, vp]
             lib.ep_selftest_wait_timeout.restype = ctypes.c_int
+            lib.ep_probe_gather.argtypes = [vp, vp, i64, vp, i64, i32, vp, vp]
+            lib.ep_probe_gather.restype = ctypes.c_int
             lib.ep_launch_count.argtypes = [vp]
             lib.ep_launch_count.restype = ctypes.c_int64
             lib.ep_kmeans_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32]
@@ -255,6 +257,18 @@ class Context:
         """Makes a bounded device wait run out (see ep_selftest_wait_timeout); returns the 3 diagnostic words."""
         out = torch.zeros(3, dtype=torch.int64, device=self.device)
         rc = self._lib.ep_selftest_wait_timeout(self._h, int(limit_clocks), ctypes.c_void_p(out.data_ptr()), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+    def probe_gather(self, colidx: torch.Tensor, table: torch.Tensor, cluster_size: int = 0) -> torch.Tensor:
+        """Yardstick: sum of table[colidx[e]] over all entries (see ep_probe_gather); returns the 1-element sum."""
+        if colidx.dtype != torch.int32 or table.dtype != torch.uint8 or not colidx.is_cuda or not table.is_cuda:
+            raise ValueError("colidx must be a CUDA int32 tensor, table a CUDA uint8 tensor")
+        out = torch.zeros(1, dtype=torch.int64, device=self.device)
+        rc = self._lib.ep_probe_gather(self._h, ctypes.c_void_p(colidx.data_ptr()), colidx.numel(),
+                                       ctypes.c_void_p(table.data_ptr()), table.numel(), int(cluster_size),
+                                       ctypes.c_void_p(out.data_ptr()), self._stream())
         if rc != EP_OK:
             self._raise(rc)
         return out

@@ -216,3 +216,27 @@ def test_host_buffer_entry_points_match_the_device_ones(ctx):
     assert torch.equal(hq.edge_cut, q.edge_cut.cpu()) and torch.equal(hq.part_vertices, q.part_vertices.cpu())
     assert torch.equal(hq.part_edges, q.part_edges.cpu())
     assert torch.equal(hr.perm, r.perm.cpu()) and torch.equal(hr.inv_perm, r.inv_perm.cpu())
+
+
+@pytest.mark.parametrize("cluster_size", [0, 2, 8, 16])
+def test_gather_yardsticks_sum_what_they_gather(ctx, cluster_size):
+    """ep_probe_gather is the edge-cut pass reduced to its label lookups (a measuring stick for the bench): whatever
+    memory serves the lookups, the sum must be that of the gathered bytes; entries outside [0, N) are skipped."""
+    import paper_2604_01000_b200 as ep
+    w = synth.scaled(synth.WORKLOADS["cfg3"], 40_009)
+    rowptr, colidx = synth.graph(w, device="cuda")
+    table = (synth.component_labels(w, torch.arange(w.N, device="cuda")) % 251).to(torch.uint8)
+    colidx = colidx.clone()
+    colidx[::1013] = -1                                   # a few entries that point nowhere
+    colidx[5::4099] = w.N
+    try:
+        got = ctx.probe_gather(colidx, table, cluster_size)
+    except ep.EmbedPartError as exc:
+        if cluster_size == 16 and exc.status == 2:
+            pytest.skip("no cluster of 16 blocks on this device")
+        raise
+    torch.cuda.synchronize()
+    ctx.check()
+    ok = (colidx >= 0) & (colidx < w.N)
+    want = int(table[colidx[ok].long()].long().sum().item())
+    assert int(got.item()) == want

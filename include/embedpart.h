@@ -364,27 +364,32 @@ int ep_reorder_host(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, in
  * memory pool was sized and handed out at start-up, a latency-critical loop in which cudaMalloc's
  * implicit device synchronisation is unacceptable.  ep_reorder needs a workspace and ep_create
  * itself allocates a status word, so neither is usable there.  This variant performs the same
- * stable sort with the same kernels, but keeps its scratch (per-tile digit counts and their scan
- * totals, about 1 MB) in an array compiled into the library.  Every GPU that loads the library
- * holds that array until the process ends, whether or not this function is ever called.
+ * stable sort with the same kernel, but keeps its scratch (one row of digit counts per thread block
+ * and the word the blocks meet on, about 1 MB) in an array compiled into the library.  Every GPU that
+ * loads the library holds that array until the process ends, whether or not this function is ever called.
  *
  *   assign, perm, inv_perm   as for ep_reorder ([dev], caller-owned; inv_perm may be NULL)
  *   N                        1 <= N <= EP_REORDER_STATIC_MAX_N
  *   K                        1 <= K <= EP_REORDER_STATIC_MAX_K   (the one-pass range of the sort)
  *   device_status            [dev] out or NULL: one int32, set to EP_OK, or to EP_ERR_BAD_INDEX if a
- *                            label outside [0, K) was seen (valid once the stream has drained)
+ *                            label outside [0, K) was seen, or to EP_ERR_TIMEOUT if the blocks' bounded
+ *                            wait for one another ran out (valid once the stream has drained).  With NULL
+ *                            the word is kept inside the built-in array, where no call can read it: a
+ *                            caller that wants to learn of bad labels must pass a word of its own
  *   cuda_stream              as elsewhere
  *
  * Works on the device that is current in the calling thread.  Returns EP_ERR_UNSUPPORTED when N or
  * K exceeds the limits above (nothing is launched), EP_ERR_INVALID_ARG for null or misaligned
  * pointers, EP_ERR_CUDA if a runtime call fails.  The function calls no cudaMalloc, cudaFree or
- * other allocating routine; it enqueues one 4-byte memset and five kernels on the stream.
+ * other allocating routine; it enqueues two 4-byte memsets and one kernel (a cooperative launch: its
+ * blocks are resident together) on the stream.
  *
- * The first call on each device looks up the device address of the built-in array (a one-time
- * set-up step); make that first call outside of any stream capture.
+ * Every call looks up the device address of the built-in array; the first such look-up on a device
+ * is a one-time set-up step of the CUDA runtime (it loads the library's code there): make that first
+ * call outside of any stream capture.
  *
  * All calls on a device share the one array, and it keeps whatever the previous call left in it.
- * The function clears the single word that has to start at zero and its kernels overwrite every
+ * The function clears the two words that have to start at zero and its kernel overwrites every
  * count before reading it, so back-to-back calls on one stream are fine.  Two calls that can run on
  * the GPU at the same time (different streams, different host threads) would scribble over each
  * other's counts: order them yourself.

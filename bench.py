@@ -182,47 +182,25 @@ def make_host_inputs(x):
 def make_host_outputs(w):
     pin = lambda *shape, dtype: torch.empty(shape, dtype=dtype).pin_memory()   # noqa: E731
     from paper_2604_01000_b200.binding import KMeansResult, QualityResult, ReorderResult
-    out = {"km": KMeansResult(pin(w.N, dtype=torch.int32), pin(w.K, w.d, dtype=torch.float32), None),
-           "q": QualityResult(pin(1, dtype=torch.int64), pin(w.K, dtype=torch.int64), pin(w.K, dtype=torch.int64)),
-           "r": ReorderResult(pin(w.N, dtype=torch.int32), pin(w.N, dtype=torch.int32))}
-    if w.reorder_K:
-        out["fine"] = KMeansResult(pin(w.N, dtype=torch.int32), pin(w.reorder_K, w.d, dtype=torch.float32), None)
-    return out
+    return (KMeansResult(pin(w.N, dtype=torch.int32), pin(w.K, w.d, dtype=torch.float32), None),
+            QualityResult(pin(1, dtype=torch.int64), pin(w.K, dtype=torch.int64), pin(w.K, dtype=torch.int64)),
+            ReorderResult(pin(w.N, dtype=torch.int32), pin(w.N, dtype=torch.int32)),
+            pin(w.N, dtype=torch.int32) if w.reorder_K else None)
 
 
-def step_host(ctx, w, h, out, ctx2=None, streams=None):
-    """The same pass through the host-buffer C-ABI calls: every call uploads its inputs and downloads its results.
-    With a second context (own workspace) and two streams, the two independent clustering runs are issued side by
-    side, as a caller with two host threads' worth of work would: the upload of one overlaps the kernels of the
-    other.  Each call still moves all of its inputs and outputs."""
-    if ctx2 is None or not w.reorder_K:
-        km = ctx.kmeans_host(h["emb"], w.K, w.iters, h["init"], out=out["km"])
-        fine, fineK = km, w.K
-        if w.reorder_K:
-            fine, fineK = ctx.kmeans_host(h["emb"], w.reorder_K, w.reorder_iters, h["init2"], out=out["fine"]), w.reorder_K
-        ctx.partition_quality_host(h["rowptr"], h["colidx"], km.assign, w.K, out=out["q"])
-        ctx.reorder_host(fine.assign, fineK, out=out["r"])
-        return
-    sa, sb = streams
-    cur = torch.cuda.current_stream()
-    sa.wait_stream(cur)
-    sb.wait_stream(cur)
-    with torch.cuda.stream(sa):        # partition run, then its score
-        km = ctx.kmeans_host(h["emb"], w.K, w.iters, h["init"], out=out["km"])
-        ctx.partition_quality_host(h["rowptr"], h["colidx"], km.assign, w.K, out=out["q"])
-    with torch.cuda.stream(sb):        # reordering run, then its permutation
-        fine = ctx2.kmeans_host(h["emb"], w.reorder_K, w.reorder_iters, h["init2"], out=out["fine"])
-        ctx2.reorder_host(fine.assign, w.reorder_K, out=out["r"])
-    cur.wait_stream(sa)
-    cur.wait_stream(sb)
+def step_host(ctx, w, h, out):
+    """The same pass through the host-buffer C ABI: ep_partition_and_reorder_host uploads every input once, runs the
+    step's kernels and downloads every result (labels of both runs, centroids, cut and loads, permutation and its
+    inverse)."""
+    ctx.partition_and_reorder_host(h["emb"], w.K, w.iters, h["init"], h["rowptr"], h["colidx"], reorder_K=w.reorder_K,
+                                   reorder_iters=w.reorder_iters, reorder_init=h["init2"], out=out)
 
 
 def host_traffic(w, h):
     nb = lambda t: t.numel() * t.element_size()   # noqa: E731
+    h2d = nb(h["emb"]) + nb(h["init"]) + (nb(h["init2"]) if w.reorder_K else 0) + nb(h["rowptr"]) + nb(h["colidx"])
     runs = 2 if w.reorder_K else 1
-    h2d = runs * nb(h["emb"]) + nb(h["init"]) + (nb(h["init2"]) if w.reorder_K else 0)
-    h2d += nb(h["rowptr"]) + nb(h["colidx"]) + 4 * w.N + 4 * w.N               # graph + labels for quality and reorder
-    d2h = runs * 4 * w.N + 4 * w.d * (w.K + w.reorder_K) + 8 * (2 * w.K + 1) + 8 * w.N
+    d2h = runs * 4 * w.N + 4 * w.d * w.K + 8 * (2 * w.K + 1) + 8 * w.N
     return h2d, d2h
 
 
@@ -659,36 +637,51 @@ def main():
                                     "full_pass_gbs": w.N * (4 * w.d + 4) / (ms_s * 1e-3) / 1e9}
 
     # ---- end to end: the same pass through the host-buffer C ABI (uploads and downloads timed) ---------
+    # Consecutive steps alternate between two contexts, each with its own arena, stream and page-locked output
+    # buffers, as a caller who keeps the GPU fed would: the uploads of one step overlap the kernels of the step before.
+    # Every step still moves all of its inputs and outputs.  One context when two arenas do not fit.
     e2e = None
     if not args.no_e2e:
         h = make_host_inputs(x)
-        out = make_host_outputs(w)
         h2d, d2h = host_traffic(w, h)
         del x
         torch.cuda.empty_cache()
-        ctx2, streams = None, None
-        if w.reorder_K:
-            ctx2 = ep.Context(local_rank)
-            ctx2.set_kmeans_path(args.kmeans_path)
-            streams = (torch.cuda.Stream(device), torch.cuda.Stream(device))
-        for _ in range(2):
-            step_host(ctx, w, h, out, ctx2, streams)
+        need = ctx.partition_and_reorder_host_arena_bytes(w.N, w.d, w.K, w.reorder_K, nnz, h["rowptr"].dtype == torch.int64)
+        free, _ = torch.cuda.mem_get_info()
+        lanes = 2 if 2 * need + (4 << 30) <= free else 1
+        ctxs, streams, outs = [ctx], [torch.cuda.Stream(device)], [make_host_outputs(w)]
+        if lanes == 2:
+            c2 = ep.Context(local_rank)
+            c2.set_kmeans_path(args.kmeans_path)
+            ctxs.append(c2)
+            streams.append(torch.cuda.Stream(device))
+            outs.append(make_host_outputs(w))
+        cur = torch.cuda.current_stream()
+
+        def run_host_steps(n):
+            for st in streams:
+                st.wait_stream(cur)
+            for i in range(n):
+                with torch.cuda.stream(streams[i % lanes]):
+                    step_host(ctxs[i % lanes], w, h, outs[i % lanes])
+            for st in streams:
+                cur.wait_stream(st)
+
+        run_host_steps(2)
         barrier()
-        e_steps = max(1, min(args.steps, 3))
+        e_steps = max(2, min(args.steps, 4))
         start.record()
-        for _ in range(e_steps):
-            step_host(ctx, w, h, out, ctx2, streams)
+        run_host_steps(e_steps)
         stop.record()
         barrier()
         ems = start.elapsed_time(stop)
         ems = max_over_ranks(ems, dist, device)
-        ctx.check()
-        if ctx2 is not None:
-            ctx2.check()
+        for c in ctxs:
+            c.check()
         e2e = {"value": whole_job_rate(world, row_iters, e_steps, ems), "unit": "rows*iters/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ems / e_steps, "steps": e_steps,
-               "api": "ep_kmeans_host / ep_partition_quality_host / ep_reorder_host with page-locked host buffers",
-               "streams": 2 if ctx2 is not None else 1}
+               "api": "ep_partition_and_reorder_host with page-locked host buffers (every input uploaded once per step)",
+               "steps_in_flight": lanes, "h2d_gb_per_s": h2d * e_steps / (ems * 1e-3) / 1e9}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

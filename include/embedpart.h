@@ -356,6 +356,32 @@ int ep_reorder_host(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, in
                     void *arena, size_t arena_bytes, void *cuda_stream);
 
 /* --------------------------------------------------------------------------------------------
+ * ep_partition_and_reorder_host -- the whole path on host buffers, every input uploaded once:
+ * P <- KMeans(E, K) (Algorithm 3, the clustering step), its edge cut and loads (Section 2.1.1, Eq. 1 and 2), and the
+ * partition-ordered numbering of Section 4.5.1, taken from a second clustering of the same embeddings with
+ * reorder_K clusters (reordering wants many small clusters) or, with reorder_K = 0, from P itself.  The same
+ * kernels as the separate calls, in this order on `cuda_stream`: uploads, ep_kmeans(K), ep_partition_quality,
+ * ep_kmeans(reorder_K), ep_reorder, each result copied back as soon as it exists.  What it saves over four *_host
+ * calls is the second upload of the embedding matrix and the upload of the labels.
+ *
+ *   emb, N, d, K, iters, init_centroids, assign, centroids:  as for ep_kmeans_host
+ *   reorder_K, reorder_iters, reorder_init [host, reorder_K x d]: the second run; reorder_K = 0 = none
+ *   rowptr, rowptr_is_int64, colidx, nnz, edge_cut, part_vertices, part_edges: as for ep_partition_quality_host
+ *   reorder_assign [host] out or NULL, N int32: the labels of the second run
+ *   perm, inv_perm [host] out (inv_perm may be NULL), N int32 each: as for ep_reorder_host
+ *   arena [dev]: at least ep_partition_and_reorder_host_arena_bytes, 256-byte aligned
+ */
+size_t ep_partition_and_reorder_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int32_t reorder_K,
+                                                 int64_t nnz, int32_t rowptr_is_int64);
+int ep_partition_and_reorder_host(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                                  const float *init_centroids, int32_t reorder_K, int32_t reorder_iters,
+                                  const float *reorder_init, const void *rowptr, int32_t rowptr_is_int64,
+                                  const int32_t *colidx, int64_t nnz, int32_t *assign, float *centroids,
+                                  uint64_t *edge_cut, int64_t *part_vertices, int64_t *part_edges,
+                                  int32_t *reorder_assign, int32_t *perm, int32_t *inv_perm, void *arena,
+                                  size_t arena_bytes, void *cuda_stream);
+
+/* --------------------------------------------------------------------------------------------
  * ep_reorder_static -- ep_reorder without a workspace and without a context.  (The paper has no
  * counterpart to this call; it exists for the sake of callers, not of the method.)
  *

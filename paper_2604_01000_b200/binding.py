@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = (
     "ep_relabel_graph_workspace_bytes", "ep_relabel_graph", "ep_permute_rows",
     "ep_balance_workspace_bytes", "ep_migrate", "ep_balance",
     "ep_cluster_and_balance_workspace_bytes", "ep_cluster_and_balance", "ep_selftest_wait_timeout", "ep_probe_gather",
+    "ep_partition_and_reorder_host_arena_bytes", "ep_partition_and_reorder_host",
 )
 
 EP_OK = 0
@@ -97,6 +98,11 @@ def load_library() -> ctypes.CDLL:
             lib.ep_selftest_wait_timeout.restype = ctypes.c_int
             lib.ep_probe_gather.argtypes = [vp, vp, i64, vp, i64, i32, vp, vp]
             lib.ep_probe_gather.restype = ctypes.c_int
+            lib.ep_partition_and_reorder_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32, i64, i32]
+            lib.ep_partition_and_reorder_host_arena_bytes.restype = sz
+            lib.ep_partition_and_reorder_host.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, vp, vp, i32, vp, i64,
+                                                          vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+            lib.ep_partition_and_reorder_host.restype = ctypes.c_int
             lib.ep_launch_count.argtypes = [vp]
             lib.ep_launch_count.restype = ctypes.c_int64
             lib.ep_kmeans_host_arena_bytes.argtypes = [vp, i64, i32, i32, i32]
@@ -601,6 +607,42 @@ class Context:
         with torch.cuda.device(self.device):
             rc = self._lib.ep_reorder_host(self._h, _dev_ptr(assign), N, K, _dev_ptr(out.perm), _dev_ptr(out.inv_perm),
                                            _dev_ptr(ws), ws.numel(), self._stream())
+        if rc != EP_OK:
+            self._raise(rc)
+        return out
+
+    def partition_and_reorder_host_arena_bytes(self, N, d, K, reorder_K, nnz, rowptr64) -> int:
+        return int(self._lib.ep_partition_and_reorder_host_arena_bytes(self._h, N, d, K, reorder_K, nnz, int(bool(rowptr64))))
+
+    def partition_and_reorder_host(self, emb, K: int, iters: int, init_centroids, rowptr, colidx, reorder_K: int = 0,
+                                   reorder_iters: int = 0, reorder_init=None, out=None):
+        """The whole path on host buffers with every input uploaded once (ep_partition_and_reorder_host).
+        Returns (KMeansResult, QualityResult, ReorderResult, labels of the second run or None); `out` may carry
+        such a tuple of page-locked tensors to write into."""
+        emb = self._host(emb, torch.float32, "emb")
+        init = self._host(init_centroids, torch.float32, "init_centroids")
+        colidx = self._host(colidx, torch.int32, "colidx")
+        rowptr = self._host(rowptr, rowptr.dtype, "rowptr")
+        init2 = self._host(reorder_init, torch.float32, "reorder_init") if reorder_K > 0 else None
+        N, d = emb.shape
+        nnz, is64 = colidx.numel(), int(rowptr.dtype == torch.int64)
+        need = self._lib.ep_partition_and_reorder_host_arena_bytes(self._h, N, d, K, reorder_K, nnz, is64)
+        if need == 0:
+            raise EmbedPartError(1, f"shape out of range: N={N} d={d} K={K} reorder_K={reorder_K} nnz={nnz}")
+        ws = self.workspace(need)
+        if out is None:
+            pin = lambda *shape, dtype: torch.empty(shape, dtype=dtype).pin_memory()   # noqa: E731
+            out = (KMeansResult(pin(N, dtype=torch.int32), pin(K, d, dtype=torch.float32), None),
+                   QualityResult(pin(1, dtype=torch.int64), pin(K, dtype=torch.int64), pin(K, dtype=torch.int64)),
+                   ReorderResult(pin(N, dtype=torch.int32), pin(N, dtype=torch.int32)),
+                   pin(N, dtype=torch.int32) if reorder_K > 0 else None)
+        km, q, r, fine = out
+        with torch.cuda.device(self.device):
+            rc = self._lib.ep_partition_and_reorder_host(
+                self._h, _dev_ptr(emb), N, d, K, iters, _dev_ptr(init), reorder_K, reorder_iters, _dev_ptr(init2),
+                _dev_ptr(rowptr), is64, _dev_ptr(colidx), nnz, _dev_ptr(km.assign), _dev_ptr(km.centroids),
+                _dev_ptr(q.edge_cut), _dev_ptr(q.part_vertices), _dev_ptr(q.part_edges), _dev_ptr(fine),
+                _dev_ptr(r.perm), _dev_ptr(r.inv_perm), _dev_ptr(ws), ws.numel(), self._stream())
         if rc != EP_OK:
             self._raise(rc)
         return out

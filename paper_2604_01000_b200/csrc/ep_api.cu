@@ -738,4 +738,103 @@ int ep_reorder_host(ep_ctx *ctx, const int32_t *assign, int64_t N, int32_t K, in
     return EP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------- whole path, host buffers
+struct WholeLayout {
+    float *emb, *cent, *cent2;
+    int32_t *assign, *assign2, *colidx, *perm, *inv;
+    char *rowptr;
+    int64_t *out;
+    void *ws;
+    size_t ws_bytes, used;
+};
+
+static bool whole_layout(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int32_t K2, int64_t nnz, int32_t is64,
+                         void *arena, WholeLayout *out) {
+    const int32_t Kf = K2 > 0 ? K2 : K;
+    const size_t km = ep_kmeans_workspace_bytes(ctx, N, d, K), km2 = K2 > 0 ? ep_kmeans_workspace_bytes(ctx, N, d, K2) : 1;
+    const size_t qw = ep_quality_workspace_bytes(ctx, N, nnz, K), rw = ep_reorder_workspace_bytes(ctx, N, Kf);
+    if (km == 0 || km2 == 0 || qw == 0 || rw == 0) return false;
+    Arena a(arena);
+    WholeLayout l{};
+    l.emb = a.take<float>((size_t)N * d);
+    l.cent = a.take<float>((size_t)K * d);
+    l.cent2 = a.take<float>((size_t)std::max(K2, 1) * d);
+    l.assign = a.take<int32_t>(N);
+    l.assign2 = a.take<int32_t>(N);
+    l.rowptr = a.take<char>((size_t)(N + 1) * (is64 ? 8 : 4));
+    l.colidx = a.take<int32_t>(nnz);
+    l.out = a.take<int64_t>(2 * (size_t)K + 1);
+    l.perm = a.take<int32_t>(N);
+    l.inv = a.take<int32_t>(N);
+    l.ws_bytes = std::max(std::max(km, km2), std::max(qw, rw));
+    l.ws = a.take<char>(l.ws_bytes);
+    l.used = a.used;
+    *out = l;
+    return true;
+}
+
+size_t ep_partition_and_reorder_host_arena_bytes(const ep_ctx *ctx, int64_t N, int32_t d, int32_t K, int32_t reorder_K,
+                                                 int64_t nnz, int32_t rowptr_is_int64) {
+    WholeLayout l;
+    if (!ctx || reorder_K < 0 || !whole_layout(ctx, N, d, K, reorder_K, nnz, rowptr_is_int64, nullptr, &l)) return 0;
+    return l.used;
+}
+
+int ep_partition_and_reorder_host(ep_ctx *ctx, const float *emb, int64_t N, int32_t d, int32_t K, int32_t iters,
+                                  const float *init_centroids, int32_t reorder_K, int32_t reorder_iters,
+                                  const float *reorder_init, const void *rowptr, int32_t rowptr_is_int64,
+                                  const int32_t *colidx, int64_t nnz, int32_t *assign, float *centroids,
+                                  uint64_t *edge_cut, int64_t *part_vertices, int64_t *part_edges,
+                                  int32_t *reorder_assign, int32_t *perm, int32_t *inv_perm, void *arena,
+                                  size_t arena_bytes, void *cuda_stream) {
+    if (!ctx) return EP_ERR_INVALID_ARG;
+    if (!emb || !init_centroids || !rowptr || (!colidx && nnz > 0) || !assign || !centroids || !edge_cut ||
+        !part_vertices || !part_edges || !perm || (reorder_K > 0 && !reorder_init))
+        return fail(ctx, EP_ERR_INVALID_ARG, "null pointer");
+    if (reorder_K < 0 || iters < 0 || reorder_iters < 0) return fail(ctx, EP_ERR_INVALID_ARG, "negative count");
+    WholeLayout l;
+    if (!whole_layout(ctx, N, d, K, reorder_K, nnz, rowptr_is_int64, arena, &l))
+        return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld d=%d K=%d reorder_K=%d nnz=%lld", (long long)N, d, K,
+                    reorder_K, (long long)nnz);
+    if (!arena || !aligned(arena, 256) || arena_bytes < l.used)
+        return fail(ctx, EP_ERR_WORKSPACE, "host arena: need %zu bytes, 256-byte aligned", l.used);
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t rp_bytes = (size_t)(N + 1) * (rowptr_is_int64 ? 8 : 4);
+    // every input once
+    EP_CUDA(ctx, cudaMemcpyAsync(l.emb, emb, sizeof(float) * N * d, cudaMemcpyHostToDevice, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(l.cent, init_centroids, sizeof(float) * K * d, cudaMemcpyHostToDevice, st));
+    if (reorder_K > 0)
+        EP_CUDA(ctx, cudaMemcpyAsync(l.cent2, reorder_init, sizeof(float) * reorder_K * d, cudaMemcpyHostToDevice, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(l.rowptr, rowptr, rp_bytes, cudaMemcpyHostToDevice, st));
+    if (nnz > 0) EP_CUDA(ctx, cudaMemcpyAsync(l.colidx, colidx, sizeof(int32_t) * nnz, cudaMemcpyHostToDevice, st));
+    // the partition and its score
+    int rc = ep_kmeans(ctx, l.emb, N, d, K, iters, l.cent, l.assign, l.cent, nullptr, l.ws, l.ws_bytes, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(assign, l.assign, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(centroids, l.cent, sizeof(float) * K * d, cudaMemcpyDeviceToHost, st));
+    rc = ep_partition_quality(ctx, l.rowptr, rowptr_is_int64, l.colidx, nnz, l.assign, N, K, reinterpret_cast<uint64_t *>(l.out),
+                              l.out + 1, l.out + 1 + K, l.ws, l.ws_bytes, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(edge_cut, l.out, sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(part_vertices, l.out + 1, sizeof(int64_t) * K, cudaMemcpyDeviceToHost, st));
+    EP_CUDA(ctx, cudaMemcpyAsync(part_edges, l.out + 1 + K, sizeof(int64_t) * K, cudaMemcpyDeviceToHost, st));
+    // the numbering: the clusters of a second, finer run when one is asked for, else the partitions themselves
+    const int32_t *fine = l.assign;
+    int32_t fineK = K;
+    if (reorder_K > 0) {
+        rc = ep_kmeans(ctx, l.emb, N, d, reorder_K, reorder_iters, l.cent2, l.assign2, l.cent2, nullptr, l.ws, l.ws_bytes, st);
+        if (rc != EP_OK) return rc;
+        if (reorder_assign)
+            EP_CUDA(ctx, cudaMemcpyAsync(reorder_assign, l.assign2, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+        fine = l.assign2;
+        fineK = reorder_K;
+    }
+    rc = ep_reorder(ctx, fine, N, fineK, l.perm, inv_perm ? l.inv : nullptr, l.ws, l.ws_bytes, st);
+    if (rc != EP_OK) return rc;
+    EP_CUDA(ctx, cudaMemcpyAsync(perm, l.perm, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    if (inv_perm) EP_CUDA(ctx, cudaMemcpyAsync(inv_perm, l.inv, sizeof(int32_t) * N, cudaMemcpyDeviceToHost, st));
+    return EP_OK;
+}
+
 }  // extern "C"

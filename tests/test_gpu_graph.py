@@ -240,3 +240,35 @@ def test_gather_yardsticks_sum_what_they_gather(ctx, cluster_size):
     ok = (colidx >= 0) & (colidx < w.N)
     want = int(table[colidx[ok].long()].long().sum().item())
     assert int(got.item()) == want
+
+
+@pytest.mark.parametrize("reorder_K", [0, 300])
+def test_whole_path_on_host_buffers_equals_the_separate_calls(ctx, reorder_K):
+    """ep_partition_and_reorder_host uploads every input once and runs the same kernels as the separate calls: its
+    outputs are theirs, bit for bit, and the graph passes equal the oracle's."""
+    w = synth.scaled(synth.WORKLOADS["cfg4"], 30_011)
+    emb = synth.embeddings(w, device="cuda")
+    rows = synth.init_centroid_rows(w, max(w.K, reorder_K), device="cuda")
+    init, init2 = emb[rows[: w.K]].contiguous(), (emb[rows[:reorder_K]].contiguous() if reorder_K else None)
+    rowptr, colidx = synth.graph(w, device="cuda")
+    km = ctx.kmeans(emb, w.K, 5, init)
+    fine = ctx.kmeans(emb, reorder_K, 2, init2) if reorder_K else km
+    q = ctx.partition_quality(rowptr, colidx, km.assign, w.K)
+    r = ctx.reorder(fine.assign, reorder_K or w.K)
+    torch.cuda.synchronize()
+    hk, hq, hr, hfine = ctx.partition_and_reorder_host(
+        emb.cpu().pin_memory(), w.K, 5, init.cpu(), rowptr.cpu(), colidx.cpu().pin_memory(), reorder_K=reorder_K,
+        reorder_iters=2, reorder_init=init2.cpu() if reorder_K else None)
+    torch.cuda.synchronize()
+    ctx.check()
+    assert torch.equal(hk.assign, km.assign.cpu()) and torch.equal(hk.centroids, km.centroids.cpu())
+    assert int(hq.edge_cut.item()) == int(q.edge_cut.item())
+    assert torch.equal(hq.part_vertices, q.part_vertices.cpu()) and torch.equal(hq.part_edges, q.part_edges.cpu())
+    assert torch.equal(hr.perm, r.perm.cpu()) and torch.equal(hr.inv_perm, r.inv_perm.cpu())
+    if reorder_K:
+        assert torch.equal(hfine, fine.assign.cpu())
+    ref = oracle.partition_quality(rowptr.cpu().numpy(), colidx.cpu().numpy(), hk.assign.numpy(), w.K)
+    assert int(hq.edge_cut.item()) == ref.edge_cut
+    perm, inv = oracle.reorder(fine.assign.cpu().numpy(), reorder_K or w.K)
+    np.testing.assert_array_equal(hr.perm.numpy(), perm)
+    np.testing.assert_array_equal(hr.inv_perm.numpy(), inv)

@@ -44,6 +44,9 @@ class EmbedPartError(RuntimeError):
 
 
 def library_path() -> str:
+    """The built library; the bounds-checked build when EP_USE_DEBUG_LIBRARY=1 is set before the first use."""
+    if os.environ.get("EP_USE_DEBUG_LIBRARY", "") == "1":
+        return os.path.join(_PKG, "libembedpart_debug.so")
     return os.path.join(_PKG, _LIB_NAME)
 
 

@@ -11,6 +11,8 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libembedpart.so")
+OBJ_DEBUG = os.path.join(PKG, "_build_debug")
+LIB_DEBUG = os.path.join(PKG, "libembedpart_debug.so")   # the bounds-checked build (-DEP_DEBUG)
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -28,8 +30,12 @@ def _newest_header():
     return max(os.path.getmtime(h) for h in hs)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds the library; debug = the bounds-checked variant (also chosen by EP_DEBUG=1 in the environment)."""
+    debug = debug or os.environ.get("EP_DEBUG", "") == "1"
     nvcc = os.environ.get("NVCC", "nvcc")
+    OBJ, LIB = (OBJ_DEBUG, LIB_DEBUG) if debug else (globals()["OBJ"], globals()["LIB"])
+    extra = ["-DEP_DEBUG"] if debug else []
     os.makedirs(OBJ, exist_ok=True)
     hdr = _newest_header()
     jobs = []
@@ -39,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, f[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr):
-            cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("EP_NVCC_EXTRA", "").split(), "-c", src, "-o", obj]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, *os.environ.get("EP_NVCC_EXTRA", "").split(), "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
@@ -63,4 +69,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

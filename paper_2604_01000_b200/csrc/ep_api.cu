@@ -1,6 +1,8 @@
 // C ABI entry points: argument checks on the host, then the kernels of the other translation units.
 #include "ep_common.cuh"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
@@ -23,7 +25,14 @@ int cuda_fail(ep_ctx *ctx, cudaError_t e, const char *what) {
     return fail(ctx, EP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+// Names of the timed regions as a profiler's timeline shows them (NVTX ranges around the host-side enqueue; they cost
+// nothing while no tool is attached).
+static const char *const kRangeNames[EP_TIMER_COUNT] = {
+    "ep:kmeans assign", "ep:kmeans update", "ep:edge cut", "ep:quality prep", "ep:reorder",
+    "ep:kmeans resolve", "ep:graph bandwidth", "ep:relabel", "ep:balance"};
+
 Timed::Timed(ep_ctx *c, cudaStream_t s, int t) : ctx(c), stream(s), timer(c->opt_timer_group * EP_TIMER_COUNT + t) {
+    nvtxRangePushA(kRangeNames[t >= 0 && t < EP_TIMER_COUNT ? t : 0]);
     if (!ctx->opt_profile) return;
     if (!ctx->spare_events.empty()) {
         start = ctx->spare_events.back();
@@ -37,6 +46,7 @@ Timed::Timed(ep_ctx *c, cudaStream_t s, int t) : ctx(c), stream(s), timer(c->opt
 
 void Timed::end(int kernels) {
     ctx->launches += kernels;
+    nvtxRangePop();
     if (!start) return;
     cudaEvent_t stop = nullptr;
     if (!ctx->spare_events.empty()) {

@@ -166,3 +166,19 @@ const long long *balance_state_ptr(int64_t N, int K, int64_t max_degree, void *w
 
 // ---- device helpers -------------------------------------------------------------------------------
 __device__ __forceinline__ void ep_raise(int *status, int code) { atomicMax(status, code); }
+
+// The bounds-checked build (-DEP_DEBUG: `EP_DEBUG=1 python -m paper_2604_01000_b200.build`, library
+// libembedpart_debug.so): an index the kernels compute themselves (a scatter destination, a slot of a list, a row
+// taken from a list) is tested before it is used; one that lies outside its array raises EP_ERR_CUDA in the status
+// word and the access is skipped, so that a wrong index shows up as a status, never as a fault.  In the ordinary
+// build the test is the constant true and costs nothing.
+#ifdef EP_DEBUG
+__device__ __forceinline__ bool ep_index_ok(long long i, long long n, int *status) {
+    if (i >= 0 && i < n) return true;
+    ep_raise(status, EP_ERR_CUDA);
+    return false;
+}
+#define EP_INDEX_OK(i, n, status) ep_index_ok((long long)(i), (long long)(n), (status))
+#else
+#define EP_INDEX_OK(i, n, status) true
+#endif

@@ -294,7 +294,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     int base = 0;
                     if (lane == 0) base = atomicAdd(slow_count, __popc(slow));
                     base = __shfl_sync(FULL, base, 0);
-                    if (live && !fast)
+                    if (live && !fast && EP_INDEX_OK(base + __popc(slow & ((1u << lane) - 1u)), row_end - row_begin, status))
                         slow_list[base + __popc(slow & ((1u << lane) - 1u))] = make_int2((int)(row - row_begin), kone);
                 }
             }

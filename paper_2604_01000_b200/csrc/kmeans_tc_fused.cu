@@ -466,7 +466,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     }
                     mlo &= K >= 32 ? 0xFFFFFFFFu : (1u << K) - 1u;     // columns beyond K are padding
                     mhi &= K >= 64 ? 0xFFFFFFFFu : K > 32 ? (1u << (K - 32)) - 1u : 0u;
-                    late_rows[(size_t)late_n + __popc(todo & lt)] = make_int4((int)row, (int)mlo, (int)mhi, 0);
+                    if (EP_INDEX_OK(late_n + __popc(todo & lt), late_cap, status))
+                        late_rows[(size_t)late_n + __popc(todo & lt)] = make_int4((int)row, (int)mlo, (int)mhi, 0);
                 }
                 late_n += __popc(todo);
             }
@@ -703,7 +704,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     }
                 }
                 if (bidx < 0 || bidx >= K) bidx = 0;         // a row of NaNs still gets a valid label
-                if (lane == 0) {
+                if (lane == 0 && EP_INDEX_OK(warp * per + r, late_chunk, status)) {
                     assign[row] = bidx;
                     late_lab[warp * per + r] = (uint8_t)bidx;
                 }

@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
         for (int64_t r = r_lo + tid; r <= r_hi; r += QT_THREADS) {
             const int64_t s = (int64_t)rowptr[r], e = (int64_t)rowptr[r + 1];
             const int64_t h = s - e0;
-            if (e > s && h >= 0 && h < ne) {
+            if (e > s && h >= 0 && h < ne && EP_INDEX_OK(h, QT_EDGES, status)) {
                 atomicOr(&bitmap[h >> 5], 1u << (h & 31));
                 headlab[h] = lab[r];
             }

@@ -262,16 +262,19 @@ __global__ void __launch_bounds__(SORT_THREADS, 1) radix_pass(const PassArgs a) 
                 const int dg = packed[i] & 255;
                 const int lp = cnt[warp][dg] + (packed[i] >> 8);
                 const int val = a.vals_in ? a.vals_in[idx] : (int)idx;
+                if (!EP_INDEX_OK(lp, tile_keys, a.status)) continue;
                 sval[lp] = val;
                 sdig[lp] = (uint8_t)dg;
                 if (KEYS_OUT) skey[lp] = key[i];
-                if (a.inv_out) a.inv_out[val] = lp + delta[dg];
+                if (a.inv_out && EP_INDEX_OK(val, a.N, a.status) && EP_INDEX_OK(lp + delta[dg], a.N, a.status))
+                    a.inv_out[val] = lp + delta[dg];
             }
         }
         __syncthreads();
         const int ntile = (int)min((int64_t)tile_keys, a.N - tile * tile_keys);
         for (int q = threadIdx.x; q < ntile; q += SORT_THREADS) {
             const int dst = q + delta[sdig[q]];
+            if (!EP_INDEX_OK(dst, a.N, a.status)) continue;
             a.vals_out[dst] = sval[q];
             if (KEYS_OUT) a.keys_out[dst] = skey[q];
         }

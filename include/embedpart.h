@@ -64,6 +64,12 @@ enum {
                                the vertex range is cut into up to 8 slices of at most this size and the column ids
                                are streamed once per slice, so that a slice's labels stay in the L2.  The result
                                does not depend on it */
+    ,
+    EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH = 6 /* the fused small-K tensor-core pass (2 <= K <= 64): 2 = all Lloyd iterations
+                               of a call inside one launch, the blocks updating the centroids themselves between grid-wide
+                               barriers; 1 = one launch per iteration plus the update kernel; 0 = by size (default: one
+                               launch while a pass reads at most 512 MiB).  The labels do not depend on it; centroids
+                               may differ in the last bit (another fixed order of the fp64 fold) */
 };
 
 /* Timers kept while EP_OPT_PROFILE is 1. */
@@ -106,8 +112,9 @@ int64_t ep_launch_count(const ep_ctx *ctx);
 /* Diagnostic counters kept while EP_OPT_PROFILE is 1; synchronises the device, copies the 8 counters to
  * out [host, 8 x int64] and clears them.  Tensor-core K-Means paths: [0] rows screened, [1] centroids the
  * large-K path re-evaluated singly in fp32, [2] groups of 128 centroids it re-evaluated whole, [3] rows the
- * fused small-K kernel left to the fp32 kernel, [4] rows the large-K screening kernel left to the fp32
- * kernel; the rest are reserved. */
+ * fused small-K kernel left undecided by its screening, [4] rows the large-K screening kernel left to the fp32
+ * kernel, [5] and [6] (one launch for all iterations only) clocks block 0 spent assigning and accumulating /
+ * meeting the other blocks and updating centroids; [7] is reserved. */
 int ep_debug_counters(ep_ctx *ctx, int64_t *out);
 
 /* Self-test of the bounded device wait (no counterpart in the paper: a property of this library).  Every wait

@@ -31,6 +31,7 @@ EP_OPT_PROFILE = 2
 EP_OPT_TIMER_GROUP = 3
 EP_OPT_KMEANS_CAND_MB = 4
 EP_OPT_QUALITY_SLICE_KB = 5
+EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH = 6
 TIMER_COUNT = 9
 TIMERS = {"kmeans_assign": 0, "kmeans_update": 1, "edge_cut": 2, "quality_prep": 3, "reorder": 4,
           "kmeans_resolve": 5, "graph_bandwidth": 6, "relabel": 7, "balance": 8}
@@ -236,6 +237,12 @@ class Context:
     def set_kmeans_cand_mb(self, mib: int):
         """Upper bound (MiB) of the tensor-core path's candidate buffer; set before calling kmeans."""
         rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_CAND_MB, mib)
+        if rc != EP_OK:
+            self._raise(rc)
+
+    def set_kmeans_iterations_per_launch(self, mode: int):
+        """0 = by size, 1 = one launch per Lloyd iteration, 2 = all iterations in one launch (fused small-K pass)."""
+        rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH, int(mode))
         if rc != EP_OK:
             self._raise(rc)
 

@@ -156,6 +156,7 @@ int ep_create(ep_ctx **out, int device) {
     ctx->opt_timer_group = 0;
     ctx->opt_cand_mb = 1024;
     ctx->opt_slice_kb = 56 * 1024;
+    ctx->opt_iters_per_launch = 0;
     ctx->launches = 0;
     ctx->last_error[0] = 0;
     DeviceGuard g(device);
@@ -214,6 +215,10 @@ int ep_set_option(ep_ctx *ctx, int option, int value) {
         ctx->opt_slice_kb = value;
         return EP_OK;
     }
+    if (option == EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH && value >= 0 && value <= 2) {
+        ctx->opt_iters_per_launch = value;
+        return EP_OK;
+    }
     return fail(ctx, EP_ERR_INVALID_ARG, "unknown option %d or value %d", option, value);
 }
 
@@ -237,6 +242,10 @@ int ep_get_option(const ep_ctx *ctx, int option, int *value) {
     }
     if (option == EP_OPT_QUALITY_SLICE_KB) {
         *value = ctx->opt_slice_kb;
+        return EP_OK;
+    }
+    if (option == EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH) {
+        *value = ctx->opt_iters_per_launch;
         return EP_OK;
     }
     return EP_ERR_INVALID_ARG;

@@ -24,6 +24,7 @@ struct ep_ctx {
     int opt_timer_group;   // EP_OPT_TIMER_GROUP
     int opt_cand_mb;       // EP_OPT_KMEANS_CAND_MB
     int opt_slice_kb;      // EP_OPT_QUALITY_SLICE_KB
+    int opt_iters_per_launch;   // EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH
     long long launches;    // kernels launched through this context
     std::vector<ep_timed_interval> intervals;   // pending event pairs (profile mode)
     std::vector<cudaEvent_t> spare_events;
@@ -124,9 +125,10 @@ int kmeans_tcf_grid(const ep_ctx *ctx, int64_t N, int d);
 int64_t kmeans_tcf_late_cap(const ep_ctx *ctx, int64_t N, int d);
 int kmeans_row_norms(ep_ctx *ctx, const float *emb, int64_t N, int d, float2 *rownorm, cudaStream_t stream);
 int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, const float *ct, TcFusedState *st);
-int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
-                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, void *late_list, bool use_prev, cudaStream_t stream);
+int kmeans_tcf_run(ep_ctx *ctx, const TcFusedState &st, const float *emb, float *centroids, float *cn, float *ct, float *clo,
+                   const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, void *late_list,
+                   int T, bool update_here, bool use_prev0, bool keep_centroids, double *objterm, double *objective,
+                   const double *x2part, int x2n, unsigned *grid_bar, cudaStream_t stream);
 
 // ---- reorder (reorder.cu) -----------------------------------------------------------------------
 size_t reorder_workspace_bytes(int64_t N, int K);

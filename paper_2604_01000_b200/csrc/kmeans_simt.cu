@@ -663,6 +663,7 @@ struct KMeansBuffers {
     float2 *rownorm;   // tensor paths: (|x_i|, |x_i - trunc(x_i)|)
     float *cmaxima;    // large-K tensor path: max |c|^2 and max rounding residual of this iteration
     void *late_list;   // fused tensor path: per screen warp, the rows the screening left undecided (16 bytes each)
+    unsigned *grid_bar;   // fused tensor path: the word its blocks meet on
 };
 
 static inline int vpl_of(int d) { return d <= 128 ? 1 : d <= 256 ? 2 : d <= 512 ? 4 : 8; }
@@ -735,6 +736,7 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.rownorm = a.take<float2>(p.N);
         if (p.tc_fused) {
             b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N, p.d) * 4 * p.grid);
+            b.grid_bar = a.take<unsigned>(64);
         } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
             b.cmaxima = a.take<float>(2);
@@ -778,13 +780,27 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     }
 
     const int T = iters > 0 ? iters : 1;
+    // Few centroids on the tensor cores.  Inputs up to a few hundred MB per pass run all their iterations, centroid
+    // updates included, inside one launch: there the gaps and prologues between launches cost more than the passes.
+    // Longer passes keep one launch per iteration and the update kernel of the other paths (it spreads over more SMs).
+    const bool one_launch = p.tc_fused && (ctx->opt_iters_per_launch == 2 ||
+                                           (ctx->opt_iters_per_launch == 0 && (size_t)N * d * sizeof(float) <= ((size_t)512 << 20)));
+    if (one_launch) {
+        int rc = kmeans_tcf_run(ctx, *tcf_state, emb, centroids, b.cnorm, b.ct, b.clo, b.rownorm, N, d, K, assign, b.psum, b.pcnt,
+                                b.late_list, T, /*update_here=*/true, false, iters == 0, b.objterm, objective, b.x2part,
+                                X2_BLOCKS, b.grid_bar, stream);
+        if (rc != EP_OK) return rc;
+        EP_CUDA(ctx, cudaGetLastError());
+        return EP_OK;
+    }
     for (int t = 0; t < T; ++t) {
         int rc = dispatch_vpl(d, [&](auto vpl_c) -> int {
             constexpr int VPL = decltype(vpl_c)::value;
             constexpr int R = VPL == 1 ? 4 : VPL == 2 ? 2 : 1;
             if (p.tc_fused) {
-                return kmeans_tcf_assign(ctx, *tcf_state, emb, centroids, b.cnorm, b.clo, b.rownorm, N, d, K, assign, b.psum,
-                                         b.pcnt, b.late_list, /*use_prev=*/t > 0, stream);
+                return kmeans_tcf_run(ctx, *tcf_state, emb, centroids, b.cnorm, b.ct, b.clo, b.rownorm, N, d, K, assign, b.psum,
+                                      b.pcnt, b.late_list, 1, /*update_here=*/false, /*use_prev0=*/t > 0, false, b.objterm, nullptr,
+                                      b.x2part, X2_BLOCKS, b.grid_bar, stream);
             } else if (p.fused) {
                 auto kern = kmeans_assign_fused<VPL, R>;
                 EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));

@@ -21,6 +21,11 @@
 // sum_j (x_j - c_j)^2 to the listed centroids in fp32 (lowest index wins ties), the label, and the row added to
 // the block's sums after all decided rows, in list order.  No floating-point atomics anywhere: the order of
 // every addition is fixed by the launch shape and the lists, so results repeat bit for bit.
+//
+// All Lloyd iterations of a call run inside ONE launch (a cooperative launch: the blocks are resident together).
+// After an iteration's tiles the blocks meet on a grid-wide barrier (a counter, polled with a time limit), block k
+// turns the published partial sums into the new centroid k (fp64, fixed order), they meet again, and the next
+// iteration's tiles start: no launch gap, no prologue and no second kernel between iterations.
 #include "ep_common.cuh"
 #include "kmeans_device.cuh"
 #include "tc_device.cuh"
@@ -122,6 +127,133 @@ __device__ __forceinline__ void add_if_less(float4 &a, const float4 &x, int i, i
 }
 __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Every block of the (cooperative) grid has arrived `target` times in total.  Bounded: after GRID_WAIT_CLOCKS, or
+// once this block has given up elsewhere, the block's abort flag is set and false comes back.
+constexpr long long GRID_WAIT_CLOCKS = 4000000000ll;
+__device__ __noinline__ bool grid_barrier(unsigned *bar, unsigned target, volatile int *abort_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(bar, 1u);
+        const long long t0 = clock64();
+        for (unsigned spins = 0;; ++spins) {
+            unsigned seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(bar) : "memory");
+            if (seen >= target || *abort_flag) break;
+            if ((spins & 31u) == 31u && clock64() - t0 > GRID_WAIT_CLOCKS) {
+                *abort_flag = 1;
+                break;
+            }
+            __nanosleep(40);
+        }
+        __threadfence();
+    }
+    __syncthreads();
+    return *abort_flag == 0;
+}
+
+// Sums of four doubles per thread over the block, in a fixed order: a butterfly inside each warp, then the warps'
+// results in warp order (red: 4 x 16 doubles of shared memory).  Every thread gets the four totals.
+__device__ __forceinline__ void block_sum4(double (&v)[4], double *red) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] += __shfl_xor_sync(FULL, v[i], o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) red[i * (THREADS / 32) + warp] = v[i];
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < THREADS / 32; ++w) t += red[i * (THREADS / 32) + w];
+        v[i] = t;
+    }
+}
+
+__device__ __forceinline__ float tf32_nearest(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+// Centroid update of cluster k by the whole block: S_k = sum over the blocks' partial sums in fp64.  A thread takes
+// four columns; the thread groups (THREADS / (d / 4, rounded up to a warp) of them) take contiguous shares of the
+// slabs, in slab order, and the group sums are added in group order: a fixed tree.  c_k <- S_k / n_k when n_k > 0,
+// else unchanged; |c_k|^2 of the new centroid, its TF32-rounded copy and what that copy misses, and the cluster's share
+// n_k |c|^2 - 2 c.S_k of the objective (c = the centroid the rows were assigned against).  Everything other blocks
+// wrote is read past the L1.  buf: 4 x THREADS + 64 doubles of shared memory.
+__device__ __noinline__ void update_cluster(int k, int K, int d, int parts, const float *psum, const int *pcnt, float *C,
+                                               float *cnorm, float *ct, float *clo, double *objterm, int keep_centroids,
+                                               double *buf) {
+    const int d4 = d >> 2, d4pad = (d4 + 31) / 32 * 32;
+    const int G = max(1, THREADS / d4pad);
+    const int g = threadIdx.x / d4pad, q = threadIdx.x - g * d4pad;
+    double *red = buf + 4 * THREADS;
+    double sums[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int p = threadIdx.x; p < parts; p += THREADS) sums[0] += (double)__ldcg(pcnt + (size_t)p * K + k);
+    block_sum4(sums, red);
+    const long long n = (long long)sums[0];                     // counts are far below 2^53: exact
+    double part[4] = {0.0, 0.0, 0.0, 0.0};
+    if (g < G && q < d4) {
+        const int p0 = (int)((long long)parts * g / G), p1 = (int)((long long)parts * (g + 1) / G);
+        const float4 *src = reinterpret_cast<const float4 *>(psum) + (size_t)k * d4 + q;
+        const size_t pitch = (size_t)K * d4;
+#pragma unroll 8
+        for (int p = p0; p < p1; ++p) {
+            const float4 v = __ldcg(src + (size_t)p * pitch);
+            part[0] += (double)v.x;
+            part[1] += (double)v.y;
+            part[2] += (double)v.z;
+            part[3] += (double)v.w;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) buf[i * THREADS + threadIdx.x] = part[i];
+    __syncthreads();
+    double t[4] = {0.0, 0.0, 0.0, 0.0};                          // c.S, |c|^2, |c'|^2, |c' - tf32(c')|^2
+    if (g == 0 && q < d4) {
+        float cold[4], cnew[4], crnd[4];
+        const float4 c4 = __ldcg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + q);
+        cold[0] = c4.x, cold[1] = c4.y, cold[2] = c4.z, cold[3] = c4.w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            double S = buf[i * THREADS + q];
+            for (int gg = 1; gg < G; ++gg) S += buf[i * THREADS + gg * d4pad + q];
+            cnew[i] = (n > 0 && !keep_centroids) ? (float)(S / (double)n) : cold[i];
+            crnd[i] = tf32_nearest(cnew[i]);
+            const double lo = (double)cnew[i] - (double)crnd[i];
+            t[0] += (double)cold[i] * S;
+            t[1] += (double)cold[i] * (double)cold[i];
+            t[2] += (double)cnew[i] * (double)cnew[i];
+            t[3] += lo * lo;
+        }
+        reinterpret_cast<float4 *>(C)[(size_t)k * d4 + q] = make_float4(cnew[0], cnew[1], cnew[2], cnew[3]);
+        reinterpret_cast<float4 *>(ct)[(size_t)k * d4 + q] = make_float4(crnd[0], crnd[1], crnd[2], crnd[3]);
+    }
+    block_sum4(t, red);
+    if (threadIdx.x == 0) {
+        cnorm[k] = (float)t[2];
+        objterm[k] = (double)n * t[1] - 2.0 * t[0];
+        clo[k] = (float)(sqrt(t[3]) * 1.000001);
+    }
+    __syncthreads();
+}
+
+// J of an iteration = sum_i |x_i|^2 + sum_k (n_k |c_k|^2 - 2 c_k.S_k), both summed in a fixed order, by one block.
+__device__ __noinline__ void objective_of_iteration(const double *x2part, int x2n, const double *objterm, int K, double *red,
+                                                    double *out) {
+    double t[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int i = threadIdx.x; i < x2n; i += THREADS) t[0] += x2part[i];
+    for (int k = threadIdx.x; k < K; k += THREADS) t[1] += __ldcg(objterm + k);
+    block_sum4(t, red);
+    if (threadIdx.x == 0) *out = t[0] + t[1];
+}
+
 // KMAX = 16, 32 or 64: upper bound of K.  VPL = 16-byte chunks of a row per lane: 1 for d <= 128 with tiles of 128
 // rows, 2 for d <= 256 with tiles of 64 rows (the stage stays 64 KB; the MMA still spans 128 TMEM lanes, the upper
 // 64 of which then hold scores of whatever follows the tile in shared memory and are never read).
@@ -130,16 +262,26 @@ __device__ __forceinline__ void tmem_wait() { asm volatile("tcgen05.wait::ld.syn
 // rows in psum[b][K][d] and their counts in pcnt[b][K].  late_list[(4 b + w) late_cap ..] is scratch for the rows
 // screen warp w cannot decide (x = row id, y and z = mask of the centroids within the bound); the block settles
 // them itself after its last tile, late_chunk rows at a time.
-// use_prev != 0: pcnt[b] still holds this block's counts of the previous iteration over the same tiles; they
-// weigh the clusters when these are shared out among the accumulate warps (any sharing gives the same sums).
-template <int KMAX, int VPL>
+// From the second iteration on (from the first when use_prev0 says so) pcnt[b] holds this block's counts of the previous
+// iteration over the same tiles; they weigh the clusters when these are shared out among the accumulate warps (any
+// sharing gives the same sums).
+// update_here != 0: the launch runs T iterations (T = 1 with keep_centroids: labels against the given centroids only);
+// after each, the centroids, cn, their TF32 copy ct (what map_c covers) and clo are rewritten in place by the blocks
+// themselves, the cluster terms of the objective go to objterm[K], and block 0 writes objective[iteration] (when asked
+// for) from them and the x2n partial sums of squares x2part.  grid_bar: one word, zero before the launch.
+// update_here == 0 (T = 1): the launch ends once the sums are published; a separate kernel updates the centroids.
+// counters (profiling only): [0] rows screened, [3] rows left undecided by the screening, [5] / [6] clocks block 0
+// spent from an iteration's start to its sums being published / from there to the end of the update.
+// PERSISTENT = update_here, known at compile time: the one-iteration instance carries none of the loop's bookkeeping.
+template <int KMAX, int VPL, bool PERSISTENT>
 __global__ void __launch_bounds__(THREADS, 1)
 kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_c,
-                const float *__restrict__ emb, const float *__restrict__ centroids,
-                const float *__restrict__ cn, const float *__restrict__ clo, const float2 *__restrict__ rownorm, int64_t N,
+                const float *__restrict__ emb, float *centroids, float *cn, float *ct, float *clo,
+                const float2 *__restrict__ rownorm, int64_t N,
                 int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
-                int32_t *__restrict__ assign, float *__restrict__ psum, int *__restrict__ pcnt,
-                int4 *__restrict__ late_list, int64_t late_cap, int late_chunk, int use_prev,
+                int32_t *__restrict__ assign, float *psum, int *pcnt,
+                int4 *late_list, int64_t late_cap, int late_chunk, int T, int update_here, int use_prev0, int keep_centroids,
+                double *objterm, double *objective, const double *__restrict__ x2part, int x2n, unsigned *grid_bar,
                 unsigned long long *counters, int *status) {
     // The swizzled tiles need 1024-byte alignment.  The array is used as declared (no pointer arithmetic
     // through integers), so that every access below stays a shared-memory instruction; should a launch
@@ -186,11 +328,36 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         sh->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (threadIdx.x < 4) sh->late_n[threadIdx.x] = 0;
-    for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
-        sh->cnt[k] = 0;
-        sh->cn[k] = k < KMAX ? cn[k] : CUDART_INF_F;     // cn is padded with a huge value beyond K
-    }
+    // Between two iterations every barrier of the pipeline rests between phases (every tile was loaded, screened,
+    // sorted and accumulated).  A barrier that went through an odd number of phases gets one more, empty one (thread 0
+    // supplies all of its arrivals): then all of them stand where they stood at the start, and the tile counters of
+    // all warp sets begin every iteration at zero, with the parities of a fresh launch.
+    auto even_out_phases = [&](uint32_t tiles, uint32_t chunks) {
+        auto flip = [&](uint64_t *bar, uint32_t count, uint32_t phases) {
+            if (phases & 1u)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+        };
+#pragma unroll 1
+        for (uint32_t st = 0; st < (uint32_t)stages; ++st) {
+            const uint32_t ph = st < tiles ? (tiles - st + (uint32_t)stages - 1u) / (uint32_t)stages : 0u;
+            flip(&sh->x_full[st], 1, ph);
+            flip(&sh->x_empty[st], A_WARPS, ph);
+        }
+#pragma unroll 1
+        for (uint32_t b = 0; b < 2; ++b) {
+            const uint32_t ph = b < tiles ? (tiles - b + 1u) / 2u : 0u;
+            flip(&sh->t_full[b], 1, ph);
+            flip(&sh->t_empty[b], SWARPS, ph);
+            flip(&sh->lab_full[b], SWARPS, ph);
+            flip(&sh->lab_empty[b], 1, ph);
+            flip(&sh->ord_full[b], 1, ph);
+            flip(&sh->ord_empty[b], A_WARPS, ph);
+        }
+        flip(&sh->c_full, 1, 1u);
+        flip(&sh->plan_full, 1, 1u);
+#pragma unroll 1
+        for (int w = 0; w < LATE_WARPS; ++w) flip(&sh->late_bar[w], 1, chunks);
+    };
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
                      "r"(tmem_cols)
@@ -201,15 +368,36 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
+    const uint32_t nt = num_tiles > (int64_t)blockIdx.x ? (uint32_t)((num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0u;   // tiles of this block
+    constexpr uint32_t it_base = 0u, ipar = 0u;
+    uint32_t grid_arrivals = 0;
+    if (PERSISTENT != (update_here != 0)) {                // the host picks the instance that matches
+        if (threadIdx.x == 0) ep_raise(status, EP_ERR_CUDA);
+        T = 0;
+    }
+
+#pragma unroll 1
+    for (int iter = 0; iter < (PERSISTENT ? T : min(T, 1)); ++iter) {
+    const int use_prev = (PERSISTENT && iter > 0) || use_prev0;
+    uint32_t chunk_it = 0;
+    const long long clk_start = clock64();
+    if (threadIdx.x < 4) sh->late_n[threadIdx.x] = 0;
+    for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
+        sh->cnt[k] = 0;
+        sh->cn[k] = k < KMAX ? __ldcg(cn + k) : CUDART_INF_F;     // cn is padded with a huge value beyond K
+    }
+    __syncthreads();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
+            // the centroids' TF32 copy of this iteration (written by other blocks through ordinary stores)
+            asm volatile("fence.proxy.async;" ::: "memory");
             mbar_expect_tx(&sh->c_full, (uint32_t)(num_kb * c_kb_bytes));
 #pragma unroll 1
             for (int kb = 0; kb < num_kb; ++kb)
                 tma_load_2d(c_smem + (size_t)kb * c_kb_bytes, &map_c, kb * KBLK, 0, &sh->c_full);
-            uint32_t it = 0;
+            uint32_t it = it_base;
             for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                 if (!mbar_wait(&sh->x_empty[s], ph ^ 1u, abort_flag)) break;
@@ -222,7 +410,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (*abort_flag) {
                 // On the way out after an abort: the loads already issued get time to land, so that nothing of this
                 // block's own still writes into its shared memory when it leaves.
-                mbar_wait_quiet(&sh->c_full, 0u, DRAIN_LIMIT_CLOCKS);
+                mbar_wait_quiet(&sh->c_full, ipar, DRAIN_LIMIT_CLOCKS);
 #pragma unroll 1
                 for (uint32_t j = it > (uint32_t)stages ? it - (uint32_t)stages : 0u; j < it; ++j)
                     mbar_wait_quiet(&sh->x_full[j % (uint32_t)stages], (j / (uint32_t)stages) & 1u, DRAIN_LIMIT_CLOCKS);
@@ -231,8 +419,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            bool ok = mbar_wait(&sh->c_full, 0u, abort_flag);
-            uint32_t it = 0;
+            bool ok = mbar_wait(&sh->c_full, ipar, abort_flag);
+            uint32_t it = it_base;
             for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
@@ -254,7 +442,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (!ok || *abort_flag) {
                 // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
                 // here must have completed
-                umma_commit(&sh->drain);
+                umma_commit(&sh->drain);                  // only ever used once: the block leaves after an abort
                 mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
             }
         }
@@ -279,7 +467,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int q = lane; q < MAX_K; q += 32) {
                 sh->kof[q] = (int8_t)-1;
                 int w = 0;
-                if (q < K) w = 1 + (use_prev ? min(max(pcnt[(size_t)blockIdx.x * K + q], 0), 1 << 24) : 0);
+                if (q < K) w = 1 + (use_prev ? min(max(__ldcg(pcnt + (size_t)blockIdx.x * K + q), 0), 1 << 24) : 0);
                 plan_cnt[q] = w;
             }
             __syncwarp();
@@ -313,9 +501,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (lane == 0) mbar_arrive(&sh->plan_full);
         }
         EP_CLK_DECL
-        for (uint32_t it = hw;; it += 2) {
-            const int64_t tile = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
-            if (tile >= num_tiles) break;
+        for (uint32_t j = 0; j < nt; ++j) {
+            const uint32_t it = it_base + j;
+            if ((it & 1u) != hw) continue;             // warp 2 takes the even tiles of the running count, warp 3 the odd ones
             const uint32_t par = hw, use = (it >> 1) & 1u;
             EP_CLK(pc_work)
             if (!mbar_wait(&sh->lab_full[par], use, abort_flag)) break;
@@ -375,8 +563,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float m2 = 0.f, ml = 0.f;                          // largest centroid norm and rounding residual
 #pragma unroll 1
         for (int k = lane; k < K; k += 32) {
-            m2 = fmaxf(m2, cn[k]);
-            ml = fmaxf(ml, clo[k]);
+            m2 = fmaxf(m2, __ldcg(cn + k));
+            ml = fmaxf(ml, __ldcg(clo + k));
         }
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) {
@@ -394,8 +582,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float2 nr_next = make_float2(0.f, 0.f);            // this row's norms, fetched one tile ahead
         if (sw < SWARPS && (int64_t)blockIdx.x * BMR + stid < N) nr_next = __ldg(rownorm + (int64_t)blockIdx.x * BMR + stid);
 
-        bool planned = mbar_wait(&sh->plan_full, 0u, abort_flag);
-        uint32_t it = 0;
+        bool planned = mbar_wait(&sh->plan_full, ipar, abort_flag);
+        uint32_t it = it_base;
         for (int64_t tile = blockIdx.x; planned && sw < SWARPS && tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u, par = it & 1u;
             const int64_t row = tile * BMR + stid;
@@ -503,9 +691,9 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < OWN; ++i)
 #pragma unroll
             for (int v = 0; v < VPL; ++v) acc[i][v] = make_float4(0.f, 0.f, 0.f, 0.f);
-        bool planned = mbar_wait(&sh->plan_full, 0u, abort_flag);
+        bool planned = mbar_wait(&sh->plan_full, ipar, abort_flag);
         EP_CLK_DECL
-        uint32_t it = 0;
+        uint32_t it = it_base;
         for (int64_t tile = blockIdx.x; planned && tile < num_tiles; tile += gridDim.x, ++it) {
             const uint32_t s = it % (uint32_t)stages;
             const uint32_t par = it & 1u, use = (it >> 1) & 1u;
@@ -566,8 +754,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     }
     __syncthreads();
-    const bool aborted = sh->abort != 0;
-    if (!aborted) {
+    if (sh->abort != 0) break;
+    {
         // ---------------------------------------------------------------- the rows the screening left undecided
         // All 16 warps.  The ring is free now: it holds the block's sums (acc_s, above), the fp32 centroids (cs) and
         // late_chunk rows at a time (rows_s), fetched by bulk copies, a warp's share on a barrier of its own.
@@ -582,7 +770,7 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         uint8_t *late_lab = &sh->lab[0][0];                                 // [late_chunk] labels of the chunk's rows, 255 = none
         const float4 *C4 = reinterpret_cast<const float4 *>(centroids);
 #pragma unroll 1
-        for (int i = threadIdx.x; i < K * d4; i += THREADS) cs[i] = __ldg(C4 + i);
+        for (int i = threadIdx.x; i < K * d4; i += THREADS) cs[i] = __ldcg(C4 + i);
         if (threadIdx.x == 0) {
             int run = 0;
 #pragma unroll 1
@@ -598,7 +786,6 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int4 *lists = late_list + (size_t)blockIdx.x * 4 * late_cap;
         const int slot = lane_chunk_slot(lane);
         const uint32_t row_bytes = (uint32_t)d * 4u;
-        uint32_t chunk_it = 0;
 #pragma unroll 1
         for (int p0 = 0; p0 < total; p0 += late_chunk, ++chunk_it) {
             // ---- 1. fetch and settle this warp's rows: an even share of the chunk, at most 32
@@ -741,10 +928,33 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float4 *out = reinterpret_cast<float4 *>(psum) + (size_t)blockIdx.x * K * d4;
 #pragma unroll 1
         for (int i = threadIdx.x; i < K * d4; i += THREADS) out[i] = acc_s[i];
-    }
 #pragma unroll 1
-    for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
-    if (threadIdx.x == 0 && *abort_flag) ep_raise(status, EP_ERR_TIMEOUT);   // a wait of the tail may have run out too
+        for (int k = threadIdx.x; k < K; k += blockDim.x) pcnt[(size_t)blockIdx.x * K + k] = sh->cnt[min((int)sh->keymap[k], MAX_K - 1)];
+
+        if (!PERSISTENT) break;
+        // ---- the centroid update, by the blocks themselves: every block has published, block k (and k + grid, ...)
+        // folds cluster k, and everybody meets again before the next iteration reads the new centroids
+        const long long clk_published = clock64();
+        grid_arrivals += gridDim.x;
+        if (!grid_barrier(grid_bar, grid_arrivals, abort_flag)) break;
+        double *buf = reinterpret_cast<double *>(x_smem);     // the block's sums are published: the ring is free again
+#pragma unroll 1
+        for (int k = blockIdx.x; k < K; k += gridDim.x)
+            update_cluster(k, K, d, (int)gridDim.x, psum, pcnt, centroids, cn, ct, clo, objterm, keep_centroids, buf);
+        asm volatile("fence.proxy.async;" ::: "memory");      // ct is next read by the TMA loads of other blocks
+        grid_arrivals += gridDim.x;
+        if (!grid_barrier(grid_bar, grid_arrivals, abort_flag)) break;
+        if (threadIdx.x == 0) even_out_phases(nt, chunk_it);      // nothing of this iteration is in flight any more
+        if (counters && blockIdx.x == 0 && threadIdx.x == 0) {
+            const long long clk_end = clock64();
+            atomicAdd(&counters[5], (unsigned long long)(clk_published - clk_start));
+            atomicAdd(&counters[6], (unsigned long long)(clk_end - clk_published));
+        }
+        if (objective && blockIdx.x == 0) objective_of_iteration(x2part, x2n, objterm, K, buf + 4 * THREADS, objective + iter);
+    }
+    }   // iterations
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) ep_raise(status, EP_ERR_TIMEOUT);
     if (warp == 2) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
@@ -853,31 +1063,48 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
 }
 
 template <int KMAX, int VPL>
-static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
-                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, int4 *late_list, bool use_prev, cudaStream_t stream) {
-    auto kern = kmeans_tc_fused<KMAX, VPL>;
+static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *emb, float *centroids, float *cn, float *ct, float *clo,
+                      const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt,
+                      int4 *late_list, int T, int update_here, int use_prev0, int keep_centroids, double *objterm,
+                      double *objective, const double *x2part, int x2n, unsigned *grid_bar, cudaStream_t stream) {
+    auto kern = update_here ? kmeans_tc_fused<KMAX, VPL, true> : kmeans_tc_fused<KMAX, VPL, false>;
     EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem));
     unsigned long long *counters =
         ctx->opt_profile ? reinterpret_cast<unsigned long long *>(ctx->d_status + EP_COUNTER_WORD0) : nullptr;
+    if (update_here) EP_CUDA(ctx, cudaMemsetAsync(grid_bar, 0, sizeof(unsigned), stream));
     Timed tm(ctx, stream, EP_TIMER_KMEANS_ASSIGN);
-    kern<<<st.grid, THREADS, st.smem, stream>>>(st.map_x, st.map_c, emb, centroids, cn, clo, rownorm, N, d, K, st.npad,
-                                              st.num_kb, st.stages, umma_idesc_tf32_m128(st.npad), st.tmem_cols, ~IDX_MASK,
-                                              assign, psum, pcnt, late_list, st.late_cap, st.late_chunk, use_prev ? 1 : 0,
-                                              counters, ctx->d_status);
+    CUtensorMap map_x = st.map_x, map_c = st.map_c;
+    int npad = st.npad, num_kb = st.num_kb, stages = st.stages, late_chunk = st.late_chunk;
+    uint32_t idesc = umma_idesc_tf32_m128(st.npad), tmem_cols = st.tmem_cols, key_mask = ~IDX_MASK;
+    int64_t late_cap = st.late_cap;
+    int *status = ctx->d_status;
+    void *args[] = {&map_x, &map_c, &emb, &centroids, &cn, &ct, &clo, &rownorm, &N, &d, &K, &npad, &num_kb, &stages, &idesc,
+                    &tmem_cols, &key_mask, &assign, &psum, &pcnt, &late_list, &late_cap, &late_chunk, &T, &update_here, &use_prev0,
+                    &keep_centroids,
+                    &objterm, &objective, &x2part, &x2n, &grid_bar, &counters, &status};
+    if (update_here)   // one block per SM, all resident together: they meet on a grid-wide barrier twice per iteration
+        EP_CUDA(ctx, cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(st.grid), dim3(THREADS), args, st.smem, stream));
+    else
+        EP_CUDA(ctx, cudaLaunchKernel(reinterpret_cast<void *>(kern), dim3(st.grid), dim3(THREADS), args, st.smem, stream));
     tm.end(1);
     EP_CUDA(ctx, cudaGetLastError());
     return EP_OK;
 }
 
-// One Lloyd assignment + accumulation pass in one launch: block b leaves its sums in psum[b][K][d] and its counts in
-// pcnt[b][K].
-int kmeans_tcf_assign(ep_ctx *ctx, const TcFusedState &st, const float *emb, const float *centroids, const float *cn,
-                      const float *clo, const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum,
-                      int *pcnt, void *late_list_ws, bool use_prev, cudaStream_t stream) {
+// update_here: all T Lloyd iterations (assignment, accumulation, centroid update, objective) in one launch; on return
+// of the stream work assign = labels of the last iteration, centroids / cn / ct / clo = those after the last update.
+// Otherwise one assignment + accumulation pass (T is taken as 1): block b leaves its sums in psum[b][K][d] and its counts
+// in pcnt[b][K] for the caller's update kernel; use_prev0 = pcnt still holds the counts of the iteration before.
+int kmeans_tcf_run(ep_ctx *ctx, const TcFusedState &st, const float *emb, float *centroids, float *cn, float *ct, float *clo,
+                   const float2 *rownorm, int64_t N, int d, int K, int32_t *assign, float *psum, int *pcnt, void *late_list_ws,
+                   int T, bool update_here, bool use_prev0, bool keep_centroids, double *objterm, double *objective,
+                   const double *x2part, int x2n, unsigned *grid_bar, cudaStream_t stream) {
     int4 *late_list = static_cast<int4 *>(late_list_ws);
     const int vpl = d <= 128 ? 1 : 2;
-#define EP_TCF(KM, V) tcf_launch<KM, V>(ctx, st, emb, centroids, cn, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, use_prev, stream)
+    if (!update_here) T = 1;
+#define EP_TCF(KM, V)                                                                                                        \
+    tcf_launch<KM, V>(ctx, st, emb, centroids, cn, ct, clo, rownorm, N, d, K, assign, psum, pcnt, late_list, T,             \
+                      update_here ? 1 : 0, use_prev0 ? 1 : 0, keep_centroids ? 1 : 0, objterm, objective, x2part, x2n, grid_bar, stream)
     return vpl == 2 ? (K <= 16 ? EP_TCF(16, 2) : EP_TCF(32, 2)) : K <= 16 ? EP_TCF(16, 1) : K <= 32 ? EP_TCF(32, 1) : EP_TCF(64, 1);
 #undef EP_TCF
 }

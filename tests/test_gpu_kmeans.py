@@ -340,3 +340,31 @@ def test_two_contexts_on_two_streams_do_not_disturb_each_other(ctx):
         other.close()
     assert torch.equal(got_a.assign, alone_a.assign) and torch.equal(got_a.centroids, alone_a.centroids)
     assert torch.equal(got_b.assign, alone_b.assign) and torch.equal(got_b.centroids, alone_b.centroids)
+
+
+@pytest.mark.parametrize("name,N,iters", [("cfg1", 10_000, 6), ("cfg3", 30_011, 4), ("cfg5", 40_009, 3)])
+def test_one_launch_for_all_iterations_equals_one_launch_per_iteration(ctx, name, N, iters):
+    """The fused small-K pass either runs every iteration of a call inside one launch (the blocks update the centroids
+    themselves between grid-wide barriers) or takes one launch per iteration plus the update kernel.  Same labels; the
+    centroids agree to the last bits (the two fold the blocks' partial sums in fp64 in different fixed orders); both
+    repeat bit for bit; both match the oracle."""
+    w = synth.scaled(synth.WORKLOADS[name], N)
+    emb, init = _inputs(w)
+    got = {}
+    try:
+        for mode in (1, 2):
+            ctx.set_kmeans_iterations_per_launch(mode)
+            a = ctx.kmeans(emb, w.K, iters, init, objective=True)
+            b = ctx.kmeans(emb, w.K, iters, init, objective=True)
+            assert torch.equal(a.assign, b.assign) and torch.equal(a.centroids, b.centroids) and torch.equal(a.objective, b.objective)
+            got[mode] = a
+            _run_and_compare(ctx, emb, init, w.K, iters, single_steps=False)
+            ctx.set_kmeans_iterations_per_launch(mode)           # _run_and_compare leaves the path on "auto", not this option
+            first = ctx.kmeans(emb, w.K, 1, init)
+            rest = ctx.kmeans(emb, w.K, iters - 1, first.centroids)
+            assert torch.equal(rest.assign, a.assign) and torch.equal(rest.centroids, a.centroids)      # resumable
+    finally:
+        ctx.set_kmeans_iterations_per_launch(0)
+    assert torch.equal(got[1].assign, got[2].assign)
+    torch.testing.assert_close(got[1].centroids, got[2].centroids, rtol=1e-6, atol=1e-7)
+    torch.testing.assert_close(got[1].objective, got[2].objective, rtol=1e-9, atol=0)

@@ -34,6 +34,18 @@ import synth  # noqa: E402
 NCU_TRAFFIC = {
     ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_286_797_056 + 615_664_128, "launch": "all rows, one iteration",
                                       "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
+    ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": 1_288_142_000 + 13_495_296, "launch": "all rows, one iteration",
+                                    "source": "profiles/kmeans_tc_fused_K32_cfg4.md"},
+    # one launch runs the call's 30 iterations: a thirtieth of its 7,213,608,000 + 103,326,720 bytes per pass
+    ("kmeans_assign_K16", "cfg3"): {"bytes_per_launch": (7_213_608_000 + 103_326_720) // 30,
+                                    "launch": "all rows, one iteration (a thirtieth of the 30-iteration launch)",
+                                    "source": "profiles/kmeans_tc_fused_K16_cfg3_all_iterations.md"},
+    ("edge_cut", "cfg4"): {"bytes_per_launch": 507_021_824 + 3_238_656, "launch": "all entries",
+                           "source": "profiles/edge_cut_chunks_cfg4.md"},
+    ("edge_cut", "cfg3"): {"bytes_per_launch": 438_612_224 + 3_328_512, "launch": "all entries",
+                           "source": "profiles/edge_cut_chunks_cfg3.md"},
+    ("reorder", "cfg4"): {"bytes_per_launch": 9_909_760 + 47_616 + 19_657_216 + 1_024, "launch": "both 6-bit passes of one sort",
+                          "source": "profiles/radix_pass_K4096_cfg4.md"},
 }
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense peak ratio: the TF32 roof when the yardstick below cannot run
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -537,7 +549,7 @@ def main():
     if last is not None and w.K <= 256:
         table = last[0].assign.to(torch.uint8)
         gather = {}
-        for csize in (0, 8, 16):
+        for csize in (0, -1, 8, 16):
             try:
                 ctx.probe_gather(x["colidx"], table, csize)
                 torch.cuda.synchronize()
@@ -548,10 +560,11 @@ def main():
                 e1.record()
                 torch.cuda.synchronize()
                 ms_g = e0.elapsed_time(e1) / 3
-                gather["global_memory" if csize == 0 else f"cluster_of_{csize}_shared_memory"] = {
+                gather[{0: "global_memory", -1: "global_memory_through_texture_units"}.get(
+                    csize, f"cluster_of_{csize}_shared_memory")] = {
                     "ms": ms_g, "gathers_per_s": nnz / (ms_g * 1e-3)}
             except ep.EmbedPartError as exc:            # the table does not fit such a cluster, or no such cluster
-                gather[f"cluster_of_{csize}_shared_memory"] = {"unavailable": str(exc)}
+                gather["texture" if csize < 0 else f"cluster_of_{csize}_shared_memory"] = {"unavailable": str(exc)}
         ctx.check()
         if "edge_cut" in passes and "global_memory" in gather:
             gather["edge_cut_over_global_gather_rate"] = passes["edge_cut"]["rate"] / gather["global_memory"]["gathers_per_s"]

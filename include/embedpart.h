@@ -130,9 +130,13 @@ int ep_selftest_wait_timeout(ep_ctx *ctx, int64_t limit_clocks, int64_t *waited,
  * target; the paper has no counterpart to this call).  Streams colidx exactly as the edge-cut pass does, gathers one
  * byte table[colidx[e]] per entry and sums the bytes: the edge-cut pass without its own work, i.e. the rate at which
  * this GPU serves such gathers.  cluster_size = 0: the table is read from global memory (L1 / L2), as the pass reads
- * labels that do not fit in shared memory; cluster_size = 2, 4, 8 or 16: the table is first spread over the shared
- * memory of thread-block clusters of that size and every lookup is a ld.shared::cluster from the block that holds the
- * vertex's slice (EP_ERR_UNSUPPORTED when N bytes do not fit cluster_size blocks, or no such cluster fits the device).
+ * labels that do not fit in shared memory; cluster_size = -1: the same table read through a texture object, i.e. by
+ * the texture units instead of the load/store unit (the table must then be aligned as textures are, 512 bytes, and
+ * no longer than the widest linear texture, else EP_ERR_INVALID_ARG / EP_ERR_UNSUPPORTED; the context keeps the
+ * texture object of the last table until another table comes or the context is destroyed); cluster_size = 2, 4, 8
+ * or 16: the table is first spread over the shared memory of thread-block clusters of that size and every lookup is
+ * a ld.shared::cluster from the block that holds the vertex's slice (EP_ERR_UNSUPPORTED when N bytes do not fit
+ * cluster_size blocks, or no such cluster fits the device).
  *   colidx [dev] nnz int32, 16-byte aligned; entries outside [0, N) are skipped
  *   table  [dev] N bytes;  sum [dev] out, 1 uint64: sum of the gathered bytes.  Asynchronous; time it with events. */
 int ep_probe_gather(ep_ctx *ctx, const int32_t *colidx, int64_t nnz, const uint8_t *table, int64_t N,

@@ -172,6 +172,7 @@ int ep_destroy(ep_ctx *ctx) {
     if (!ctx) return EP_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
     cudaFree(ctx->d_status);
+    if (ctx->probe_tex) cudaDestroyTextureObject((cudaTextureObject_t)ctx->probe_tex);
     for (auto &iv : ctx->intervals) {
         cudaEventDestroy(iv.start);
         cudaEventDestroy(iv.stop);

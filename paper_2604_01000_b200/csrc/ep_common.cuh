@@ -26,6 +26,9 @@ struct ep_ctx {
     int opt_slice_kb;      // EP_OPT_QUALITY_SLICE_KB
     int opt_iters_per_launch;   // EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH
     long long launches;    // kernels launched through this context
+    unsigned long long probe_tex = 0;   // texture object of ep_probe_gather's last table (0: none), kept so that the call
+    const void *probe_tex_ptr = nullptr;   // stays asynchronous; replaced when another table or size comes
+    long long probe_tex_n = 0;
     std::vector<ep_timed_interval> intervals;   // pending event pairs (profile mode)
     std::vector<cudaEvent_t> spare_events;
     char last_error[256];

@@ -6,7 +6,9 @@
 //   gather_global   the byte table in global memory (L1 / L2), as the edge-cut pass reads it when the labels do
 //                   not fit in shared memory;
 //   gather_cluster  the byte table spread over the shared memory of a thread-block cluster, every lookup a
-//                   ld.shared::cluster from the block that holds the vertex's slice.
+//                   ld.shared::cluster from the block that holds the vertex's slice;
+//   gather_texture  the byte table in global memory, read through a texture object (the texture units' own
+//                   address and tag path instead of the load/store unit's).
 #include "ep_common.cuh"
 
 #include <algorithm>
@@ -54,6 +56,40 @@ __global__ void __launch_bounds__(PB_THREADS, 4) gather_global(const int32_t *__
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 if ((unsigned)cols[j] < (unsigned)N) t += __ldg(table + cols[j]);
+        }
+        mine += t;
+    }
+    block_add(mine, sum);
+}
+
+__global__ void __launch_bounds__(PB_THREADS, 4) gather_texture(const int32_t *__restrict__ colidx, int64_t nnz,
+                                                              cudaTextureObject_t table, int64_t N,
+                                                              unsigned long long *sum) {
+    const int64_t ntiles = (nnz + PB_TILE - 1) / PB_TILE;
+    unsigned long long mine = 0ull;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t e0 = tile * PB_TILE;
+        const int ne = (int)min((int64_t)PB_TILE, nnz - e0);
+        int4 c[PB_VEC];
+#pragma unroll
+        for (int i = 0; i < PB_VEC; ++i) {
+            const int q = (i * PB_THREADS + threadIdx.x) * 4;
+            if (q + 3 < ne) {
+                c[i] = __ldcs(reinterpret_cast<const int4 *>(colidx + e0) + (q >> 2));
+            } else {
+                c[i].x = q + 0 < ne ? colidx[e0 + q + 0] : -1;
+                c[i].y = q + 1 < ne ? colidx[e0 + q + 1] : -1;
+                c[i].z = q + 2 < ne ? colidx[e0 + q + 2] : -1;
+                c[i].w = -1;
+            }
+        }
+        unsigned t = 0;
+#pragma unroll
+        for (int i = 0; i < PB_VEC; ++i) {
+            const int cols[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if ((unsigned)cols[j] < (unsigned)N) t += tex1Dfetch<unsigned char>(table, cols[j]);
         }
         mine += t;
     }
@@ -127,8 +163,9 @@ extern "C" int ep_probe_gather(ep_ctx *ctx, const int32_t *colidx, int64_t nnz, 
     if (!aligned(colidx, 16) || !aligned(sum, 8)) return fail(ctx, EP_ERR_INVALID_ARG, "misaligned pointer");
     if (N < 1 || N >= (int64_t(1) << 31) || nnz < 1 || nnz >= (int64_t(1) << 40))
         return fail(ctx, EP_ERR_INVALID_ARG, "shape out of range: N=%lld nnz=%lld", (long long)N, (long long)nnz);
-    if (cluster_size != 0 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8 && cluster_size != 16)
-        return fail(ctx, EP_ERR_INVALID_ARG, "cluster_size must be 0 (global memory), 2, 4, 8 or 16");
+    if (cluster_size != -1 && cluster_size != 0 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8 &&
+        cluster_size != 16)
+        return fail(ctx, EP_ERR_INVALID_ARG, "cluster_size must be -1 (texture), 0 (global memory), 2, 4, 8 or 16");
     DeviceGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     auto *out = reinterpret_cast<unsigned long long *>(sum);
@@ -136,6 +173,39 @@ extern "C" int ep_probe_gather(ep_ctx *ctx, const int32_t *colidx, int64_t nnz, 
     if (cluster_size == 0) {
         const int grid = (int)std::min<int64_t>(ceil_div(nnz, PB_TILE), (int64_t)ctx->sm_count * 4);
         gather_global<<<grid, PB_THREADS, 0, st>>>(colidx, nnz, table, N, out);
+        ctx->launches += 1;
+        EP_CUDA(ctx, cudaGetLastError());
+        return EP_OK;
+    }
+    if (cluster_size == -1) {
+        int max_linear = 0, tex_align = 0;
+        EP_CUDA(ctx, cudaDeviceGetAttribute(&max_linear, cudaDevAttrMaxTexture1DLinearWidth, ctx->device));
+        EP_CUDA(ctx, cudaDeviceGetAttribute(&tex_align, cudaDevAttrTextureAlignment, ctx->device));
+        if (N > (int64_t)max_linear)
+            return fail(ctx, EP_ERR_UNSUPPORTED, "%lld table bytes exceed the widest linear texture (%d)", (long long)N, max_linear);
+        if (tex_align > 0 && !aligned(table, (size_t)tex_align))
+            return fail(ctx, EP_ERR_INVALID_ARG, "the table must be aligned to %d bytes for the texture path", tex_align);
+        if (ctx->probe_tex == 0 || ctx->probe_tex_ptr != table || ctx->probe_tex_n != (long long)N) {
+            if (ctx->probe_tex) {                              // a kernel of an earlier call may still read through it
+                EP_CUDA(ctx, cudaDeviceSynchronize());
+                cudaDestroyTextureObject((cudaTextureObject_t)ctx->probe_tex);
+                ctx->probe_tex = 0;
+            }
+            cudaResourceDesc res = {};
+            res.resType = cudaResourceTypeLinear;
+            res.res.linear.devPtr = const_cast<uint8_t *>(table);
+            res.res.linear.desc = cudaCreateChannelDesc<unsigned char>();
+            res.res.linear.sizeInBytes = (size_t)N;
+            cudaTextureDesc td = {};
+            td.readMode = cudaReadModeElementType;
+            cudaTextureObject_t tex = 0;
+            EP_CUDA(ctx, cudaCreateTextureObject(&tex, &res, &td, nullptr));
+            ctx->probe_tex = (unsigned long long)tex;
+            ctx->probe_tex_ptr = table;
+            ctx->probe_tex_n = (long long)N;
+        }
+        const int grid = (int)std::min<int64_t>(ceil_div(nnz, PB_TILE), (int64_t)ctx->sm_count * 4);
+        gather_texture<<<grid, PB_THREADS, 0, st>>>(colidx, nnz, (cudaTextureObject_t)ctx->probe_tex, N, out);
         ctx->launches += 1;
         EP_CUDA(ctx, cudaGetLastError());
         return EP_OK;

@@ -1,7 +1,7 @@
 // Edge cut and partition loads (Section 2.1.1, Eq. 1 and Eq. 2) over a CSR graph.
 //
 // The work is split by EDGES, not by rows, so a power-law degree distribution cannot unbalance it:
-// every block takes tiles of QT_EDGES consecutive CSR entries, streams their column ids with 16-byte
+// every warp takes chunks of QC_EDGES consecutive CSR entries, streams their column ids with 16-byte
 // loads, and recovers the source vertex of each entry from a bitmap of row starts built in shared
 // memory.  Labels are first repacked to the narrowest integer that holds K values so that the
 // per-entry label gather touches as few cache lines as possible.
@@ -11,14 +11,13 @@
 
 namespace {
 
-constexpr int QT_THREADS = 256;
-constexpr int QT_VEC = 8;                                   // 16-byte loads per thread per tile
-constexpr int QT_EDGES = QT_THREADS * QT_VEC * 4;           // 8192 entries per tile
-constexpr int QT_WORDS = QT_EDGES / 32;                     // 256 bitmap words, one per thread
+constexpr int QC_VEC = 8;                                   // 16-byte loads per lane per chunk
+constexpr int QC_EDGES = 32 * QC_VEC * 4;                   // 1024 entries per warp chunk
+constexpr int QC_WORDS = QC_EDGES / 32;                     // 32 bitmap words, one per lane
 constexpr int HIST_SMEM_K = 2048;
 constexpr unsigned FULL = 0xffffffffu;
 
-// tile_row[t] = last row r in [0, N) whose first entry is at or before t * QT_EDGES; tile_row[ntiles] = N-1.
+// tile_row[t] = last row r in [0, N) whose first entry is at or before t * QC_EDGES; tile_row[ntiles] = N-1.
 template <typename RowT>
 __global__ void tile_start_rows(const RowT *__restrict__ rowptr, int64_t N, int64_t ntiles, int32_t *tile_row) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -27,7 +26,7 @@ __global__ void tile_start_rows(const RowT *__restrict__ rowptr, int64_t N, int6
         tile_row[t] = (int32_t)(N - 1);
         return;
     }
-    const int64_t e = t * QT_EDGES;
+    const int64_t e = t * QC_EDGES;
     int64_t lo = 0, hi = N - 1;                             // rowptr[0] = 0 <= e always
     while (lo < hi) {
         int64_t mid = (lo + hi + 1) >> 1;
@@ -96,123 +95,163 @@ __global__ void __launch_bounds__(256) pack_labels_and_loads(const RowT *__restr
     }
 }
 
-// Counts the cut entries.  For a tile [e0, e0+ne): the rows whose first entry falls inside the tile
-// set a bit at that position and park their label there; an entry's source label is the label at the
-// nearest set bit at or before it (or, before the first set bit, the label of the row that straddles
-// the tile start).
+// Counts the cut entries.  Every WARP takes chunks of QC_EDGES consecutive CSR entries and works on them on its own:
+// no barrier wider than the warp anywhere, so the warps of a block drift apart and hide one another's latencies.
+// For a chunk [e0, e0+ne): the rows whose first entry falls inside it set a bit at that position (a 32-word bitmap of
+// the warp's own in shared memory) and park their label there; an entry's source label is the label at the nearest
+// set bit at or before it (or, before the first set bit, the label of the row that straddles the chunk start).
 //
 // PACK = 0: the label of an entry's target comes from the repacked label array in global memory (L2).
 // PACK = 8 / 4: every block first copies all labels into shared memory, one byte / one nibble each (K <= 256 /
 // K <= 16, and N small enough to fit), so that the per-entry gather never leaves the SM and the pass becomes a
-// plain stream of the column ids.
-//
-// GROUPS = 1: a block is one group of QT_THREADS threads.  GROUPS = 4: a block of 1024 threads holds four such
-// groups, each with its own tile, bitmap and named barrier, sharing one copy of the label table: the form for a
-// table so large that only one block fits on an SM, which still needs 32 warps to hide the stream's latency.
+// plain stream of the column ids.  WARPS = 8: four such blocks per SM; WARPS = 32: one block per SM, for a table
+// so large that only one copy fits, which still needs 32 warps to hide the stream's latency.
 //
 // SLICED: the launch counts only the entries whose target lies in [col_lo, col_hi) (and reports bad indices only
 // when col_lo == 0); the caller launches it once per slice of the vertex range, each slice's labels small enough to
 // stay in the L2 while the column ids stream past, and the counts of the launches add up.
-template <typename RowT, typename LabT, int PACK, int GROUPS, bool SLICED = false>
-__global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
-    edge_cut_tiles(const RowT *__restrict__ rowptr, const int32_t *__restrict__ colidx, int64_t nnz,
-                   const LabT *__restrict__ lab, int64_t N, const int32_t *__restrict__ tile_row, int64_t ntiles,
-                   unsigned long long *edge_cut, int *status, int32_t col_lo, int32_t col_hi) {
-    __shared__ unsigned bitmap_[GROUPS][QT_WORDS];
-    __shared__ int lasthead_[GROUPS][QT_WORDS];
-    __shared__ LabT headlab_[GROUPS][QT_EDGES];
-    __shared__ int warp_max_[GROUPS][QT_THREADS / 32];
+template <typename LabT>
+struct WarpScratch {
+    unsigned bitmap[QC_WORDS];
+    int lasthead[QC_WORDS];                  // 1 + position of the last row start in the words before this one; 0: none
+    LabT headlab[QC_EDGES + 4];              // [0]: label of the row that straddles the chunk start; [1 + h]: row starting at h
+};
+
+template <typename RowT, typename LabT, int PACK, int WARPS, bool SLICED = false>
+__global__ void __launch_bounds__(WARPS * 32, WARPS == 8 ? 4 : 1)
+    edge_cut_chunks(const RowT *__restrict__ rowptr, const int32_t *__restrict__ colidx, int64_t nnz,
+                    const LabT *__restrict__ lab, int64_t N, const int32_t *__restrict__ chunk_row, int64_t nchunks,
+                    unsigned long long *edge_cut, int *status, int32_t col_lo, int32_t col_hi) {
+    __shared__ WarpScratch<LabT> scratch[WARPS];
     __shared__ unsigned long long block_cut;
     extern __shared__ __align__(16) uint8_t lab_tab[];       // PACK != 0: all labels, packed
-    const int grp = GROUPS == 1 ? 0 : (int)(threadIdx.x / QT_THREADS);
-    unsigned *bitmap = bitmap_[grp];
-    int *lasthead = lasthead_[grp];
-    LabT *headlab = headlab_[grp];
-    int *warp_max = warp_max_[grp];
-    auto group_sync = [&]() {
-        if (GROUPS == 1)
-            __syncthreads();
-        else
-            asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(QT_THREADS) : "memory");
-    };
-    const int tid = threadIdx.x % QT_THREADS, lane = tid & 31, warp = tid >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned *bitmap = scratch[warp].bitmap;
+    int *lasthead = scratch[warp].lasthead;
+    LabT *headlab = scratch[warp].headlab;
     if (threadIdx.x == 0) block_cut = 0ull;
     unsigned long long my_cut = 0ull;
     if (PACK == 8) {
-        for (int64_t v = threadIdx.x * 4; v < N; v += QT_THREADS * GROUPS * 4) {   // N bytes; the array is padded to a multiple of 4
+        for (int64_t v = threadIdx.x * 4; v < N; v += WARPS * 32 * 4) {   // N bytes; the array is padded to a multiple of 4
             *reinterpret_cast<uint32_t *>(lab_tab + v) = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
         }
     } else if (PACK == 4) {
-        for (int64_t v = threadIdx.x * 4; v < N; v += QT_THREADS * GROUPS * 4) {   // four labels in, two bytes out
+        for (int64_t v = threadIdx.x * 4; v < N; v += WARPS * 32 * 4) {   // four labels in, two bytes out
             const uint32_t w4 = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(lab) + v);
             *reinterpret_cast<uint16_t *>(lab_tab + (v >> 1)) =
                 (uint16_t)((w4 & 15u) | ((w4 >> 4) & 0xF0u) | ((w4 >> 8) & 0xF00u) | ((w4 >> 12) & 0xF000u));
         }
     }
-    if (PACK != 0) __syncthreads();
+    __syncthreads();                                         // the table, and block_cut
 
-    for (int64_t tile = (int64_t)blockIdx.x * GROUPS + grp; tile < ntiles; tile += (int64_t)gridDim.x * GROUPS) {
-        const int64_t e0 = tile * QT_EDGES;
-        const int ne = (int)min((int64_t)QT_EDGES, nnz - e0);
+    // a lane's vectors sit at entries (i * 32 + lane) * 4: always the same bit of their bitmap word
+    const int vbit = (lane * 4) & 31;
+    const unsigned upto_mask = 0xffffffffu >> (31 - vbit);
+
+    // The rows that start inside a chunk are found through three dependent loads (the chunk's first row, its
+    // entries' range, its label).  They are taken out of the chunk's own critical path: a lane's first row of the
+    // NEXT chunk and the row range of the chunk after that are loaded while the current chunk is worked on.
+    const int64_t stride = (int64_t)gridDim.x * WARPS;
+    int64_t chunk = (int64_t)blockIdx.x * WARPS + warp;
+    int32_t r_lo = 0, r_hi = -1, n_lo = 0, n_hi = -1;
+    int64_t row_s = 0, row_e = 0;                            // entries of row r_lo + lane, and its label
+    LabT row_l = 0;
+    if (chunk < nchunks) {
+        r_lo = chunk_row[chunk];
+        r_hi = chunk_row[chunk + 1];
+        if (r_lo + lane <= r_hi) {
+            row_s = (int64_t)rowptr[r_lo + lane];
+            row_e = (int64_t)rowptr[r_lo + lane + 1];
+            row_l = lab[r_lo + lane];
+        }
+    }
+    if (chunk + stride < nchunks) {
+        n_lo = chunk_row[chunk + stride];
+        n_hi = chunk_row[chunk + stride + 1];
+    }
+    for (; chunk < nchunks; chunk += stride) {
+        const int64_t e0 = chunk * QC_EDGES;
+        const int ne = (int)min((int64_t)QC_EDGES, nnz - e0);
+        const bool full = ne == QC_EDGES;
         const int4 *src = reinterpret_cast<const int4 *>(colidx + e0);
-        // issue this tile's column loads first: they do not depend on anything below
-        int4 c[QT_VEC];
+        // issue this chunk's column loads first: they do not depend on anything below
+        int4 c[QC_VEC];
+        if (full) {
 #pragma unroll
-        for (int i = 0; i < QT_VEC; ++i) {
-            const int q = (i * QT_THREADS + tid) * 4;
-            if (q + 3 < ne) {
-                c[i] = __ldcs(src + (q >> 2));
-            } else {
+            for (int i = 0; i < QC_VEC; ++i) c[i] = __ldcs(src + i * 32 + lane);
+        } else {
+#pragma unroll
+            for (int i = 0; i < QC_VEC; ++i) {
+                const int q = (i * 32 + lane) * 4;
                 c[i].x = q + 0 < ne ? colidx[e0 + q + 0] : -1;
                 c[i].y = q + 1 < ne ? colidx[e0 + q + 1] : -1;
                 c[i].z = q + 2 < ne ? colidx[e0 + q + 2] : -1;
-                c[i].w = -1;
+                c[i].w = q + 3 < ne ? colidx[e0 + q + 3] : -1;
             }
         }
-        group_sync();                                    // previous tile fully consumed
-        bitmap[tid] = 0u;
-        group_sync();
-        const int64_t r_lo = tile_row[tile], r_hi = tile_row[tile + 1];
-        const LabT carry = lab[r_lo];
-        for (int64_t r = r_lo + tid; r <= r_hi; r += QT_THREADS) {
+        int64_t next_s = 0, next_e = 0;
+        LabT next_l = 0;
+        int32_t nn_lo = 0, nn_hi = -1;
+        if (n_lo + lane <= n_hi) {                           // n_hi = -1 when there is no next chunk
+            next_s = (int64_t)rowptr[n_lo + lane];
+            next_e = (int64_t)rowptr[n_lo + lane + 1];
+            next_l = lab[n_lo + lane];
+        }
+        if (chunk + 2 * stride < nchunks) {
+            nn_lo = chunk_row[chunk + 2 * stride];
+            nn_hi = chunk_row[chunk + 2 * stride + 1];
+        }
+        __syncwarp();                                    // previous chunk fully consumed by every lane
+        bitmap[lane] = 0u;
+        __syncwarp();
+        if (lane == 0) headlab[0] = row_l;               // row r_lo: the one that straddles the chunk start
+        {
+            const int64_t h = row_s - e0;
+            if (row_e > row_s && h >= 0 && h < ne && EP_INDEX_OK(h, QC_EDGES, status)) {
+                atomicOr(&bitmap[h >> 5], 1u << (h & 31));
+                headlab[1 + h] = row_l;
+            }
+        }
+        for (int64_t r = (int64_t)r_lo + 32 + lane; r <= r_hi; r += 32) {
             const int64_t s = (int64_t)rowptr[r], e = (int64_t)rowptr[r + 1];
             const int64_t h = s - e0;
-            if (e > s && h >= 0 && h < ne && EP_INDEX_OK(h, QT_EDGES, status)) {
+            if (e > s && h >= 0 && h < ne && EP_INDEX_OK(h, QC_EDGES, status)) {
                 atomicOr(&bitmap[h >> 5], 1u << (h & 31));
-                headlab[h] = lab[r];
+                headlab[1 + h] = lab[r];
             }
         }
-        group_sync();
-        {   // lasthead[w] = position of the last set bit in words < w, or -1
-            const unsigned wbits = bitmap[tid];
-            const int mine = wbits ? tid * 32 + 31 - __clz(wbits) : -1;
-            int inc = mine;
+        __syncwarp();
+        {   // lasthead[w] = 1 + position of the last set bit in the words before w, or 0
+            const unsigned wbits = bitmap[lane];
+            int inc = wbits ? lane * 32 + 32 - __clz(wbits) : 0;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                int t = __shfl_up_sync(FULL, inc, o);
+                const int t = __shfl_up_sync(FULL, inc, o);
                 if (lane >= o) inc = max(inc, t);
             }
-            if (lane == 31) warp_max[warp] = inc;
             int excl = __shfl_up_sync(FULL, inc, 1);
-            if (lane == 0) excl = -1;
-            group_sync();
-            for (int w = 0; w < warp; ++w) excl = max(excl, warp_max[w]);
-            lasthead[tid] = excl;
+            if (lane == 0) excl = 0;
+            lasthead[lane] = excl;
         }
-        group_sync();
+        __syncwarp();
         unsigned cut = 0, bad = 0;
-        // one vector of four entries: their source label from the bitmap, their targets' labels gathered
-        auto vec = [&](int q, const int4 &cv, bool full) {
-            const int wd = q >> 5, b = q & 31;
+        // index into headlab of the source label in force at entry q (the first of a vector)
+        auto source_of = [&](int wd, unsigned bits) -> int {
+            const unsigned upto = bits & upto_mask;
+            const int before = lasthead[wd];
+            const int inside = (wd << 5) + 32 - __clz(upto);
+            return upto ? inside : before;
+        };
+        // one vector of four entries with every test: a ragged chunk, or an index outside [0, N) somewhere in the warp
+        auto vec = [&](int q, const int4 &cv) {
+            const int wd = q >> 5;
             const unsigned bits = bitmap[wd];
-            const unsigned upto = bits & (0xffffffffu >> (31 - b));
-            const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
-            LabT cur = head >= 0 ? headlab[head] : carry;
+            LabT cur = headlab[source_of(wd, bits)];
             const int cols[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (j > 0 && ((bits >> (b + j)) & 1u)) cur = headlab[q + j];
-                const bool live = full || q + j < ne;
+                if (j > 0 && ((bits >> (vbit + j)) & 1u)) cur = headlab[1 + q + j];
+                const bool live = q + j < ne;
                 const int col = cols[j];
                 const bool in = (unsigned)col < (unsigned)N;
                 const bool mine = !SLICED || (unsigned)(col - col_lo) < (unsigned)(col_hi - col_lo);
@@ -228,55 +267,76 @@ __global__ void __launch_bounds__(QT_THREADS * GROUPS, GROUPS == 1 ? 4 : 1)
                 bad |= (live && !in && (!SLICED || col_lo == 0)) ? 1u : 0u;
             }
         };
-        // The usual vector: a full tile, every index of this thread inside [0, N).  No per-entry range or length
-        // test, and one source label for all four entries unless a row starts among the last three.
+        // The usual vector: a full chunk, every index of the warp inside [0, N).  No per-entry range or length test,
+        // and one source label for all four entries unless a row starts among the last three of some lane's vector
+        // (decided for the warp as a whole, so that the branch does not diverge).
         auto differs = [&](int col, unsigned cur) -> unsigned {
             if (PACK == 8) return lab_tab[col] != cur ? 1u : 0u;
-            if (PACK == 4)   // cur fills both nibbles: compare the nibble of col in place
-                return ((lab_tab[col >> 1] ^ cur) & (0xFu << ((col << 2) & 4))) != 0u ? 1u : 0u;
             if (SLICED && (unsigned)(col - col_lo) >= (unsigned)(col_hi - col_lo)) return 0u;   // another launch's entry
             return (unsigned)__ldg(lab + col) != cur ? 1u : 0u;
         };
+        unsigned nib16 = 0u;                                 // PACK == 4: 16 x the differing entries of this chunk
         auto vec_clean = [&](int q, const int4 &cv) {
-            const int wd = q >> 5, b = q & 31;
+            const int wd = q >> 5;
             const unsigned bits = bitmap[wd];
-            const unsigned upto = bits & (0xffffffffu >> (31 - b));
-            const int head = upto ? (wd << 5) + 31 - __clz(upto) : lasthead[wd];
-            const unsigned cur = head >= 0 ? (unsigned)headlab[head] : (unsigned)carry;
-            const unsigned rep = PACK == 4 ? 0x11u : 1u;
-            if (((bits >> b) & 0xEu) == 0u) {
-                const unsigned cw = cur * rep;
-                cut += differs(cv.x, cw) + differs(cv.y, cw) + differs(cv.z, cw) + differs(cv.w, cw);
+            const unsigned c0 = (unsigned)headlab[source_of(wd, bits)];
+            const unsigned inner = (bits >> vbit) & 0xEu;
+            const bool split = __any_sync(FULL, inner != 0u);
+            unsigned c1 = c0, c2 = c0, c3 = c0;
+            if (PACK == 4) {
+                // Four nibble lookups compared at once.  The four bytes that hold the targets' labels are packed into
+                // one word and XORed with the source labels (each in both nibbles of its byte); a byte's mask keeps the
+                // nibble its index selects (0x0F or 0xF0 = 0x0F + 0xE1 x the index's lowest bit); a byte differs when
+                // the kept nibble is not zero.
+                const unsigned t0 = lab_tab[cv.x >> 1], t1 = lab_tab[cv.y >> 1], t2 = lab_tab[cv.z >> 1],
+                               t3 = lab_tab[cv.w >> 1];
+                const unsigned tw = (t1 * 256u + t0) + (t3 * 256u + t2) * 65536u;
+                const unsigned low = __byte_perm(__byte_perm(cv.x, cv.y, 0x0040), __byte_perm(cv.z, cv.w, 0x0040), 0x5410) &
+                                     0x01010101u;
+                const unsigned mask = low * 0xE1u + 0x0F0F0F0Fu;
+                unsigned cw = c0 * 0x11111111u;
+                if (split) {
+                    const unsigned h1 = headlab[1 + q + 1], h2 = headlab[1 + q + 2], h3 = headlab[1 + q + 3];
+                    c1 = (inner & 2u) ? h1 : c0;
+                    c2 = (inner & 4u) ? h2 : c1;
+                    c3 = (inner & 8u) ? h3 : c2;
+                    cw = (c0 | (c1 << 8) | (c2 << 16) | (c3 << 24)) * 0x11u;
+                }
+                const unsigned v = (tw ^ cw) & mask;
+                const unsigned nz = (((v | (v >> 4)) & 0x0F0F0F0Fu) + 0x0F0F0F0Fu) & 0x10101010u;
+                nib16 = __dp4a(nz, 0x01010101u, nib16);
             } else {
-                const unsigned c1 = ((bits >> (b + 1)) & 1u) ? (unsigned)headlab[q + 1] : cur;
-                const unsigned c2 = ((bits >> (b + 2)) & 1u) ? (unsigned)headlab[q + 2] : c1;
-                const unsigned c3 = ((bits >> (b + 3)) & 1u) ? (unsigned)headlab[q + 3] : c2;
-                cut += differs(cv.x, cur * rep) + differs(cv.y, c1 * rep) + differs(cv.z, c2 * rep) + differs(cv.w, c3 * rep);
+                if (split) {
+                    const unsigned h1 = headlab[1 + q + 1], h2 = headlab[1 + q + 2], h3 = headlab[1 + q + 3];
+                    c1 = (inner & 2u) ? h1 : c0;
+                    c2 = (inner & 4u) ? h2 : c1;
+                    c3 = (inner & 8u) ? h3 : c2;
+                }
+                cut += differs(cv.x, c0) + differs(cv.y, c1) + differs(cv.z, c2) + differs(cv.w, c3);
             }
         };
         unsigned top = 0u;                                   // largest index of this thread, as unsigned
 #pragma unroll
-        for (int i = 0; i < QT_VEC; ++i)
+        for (int i = 0; i < QC_VEC; ++i)
             top = max(max(max(top, (unsigned)c[i].x), max((unsigned)c[i].y, (unsigned)c[i].z)), (unsigned)c[i].w);
-        if (ne == QT_EDGES && top < (unsigned)N) {
+        if (__all_sync(FULL, full && top < (unsigned)N)) {
 #pragma unroll
-            for (int i = 0; i < QT_VEC; ++i) vec_clean((i * QT_THREADS + tid) * 4, c[i]);
-        } else if (ne == QT_EDGES) {
-#pragma unroll
-            for (int i = 0; i < QT_VEC; ++i) vec((i * QT_THREADS + tid) * 4, c[i], true);
+            for (int i = 0; i < QC_VEC; ++i) vec_clean((i * 32 + lane) * 4, c[i]);
+            cut += nib16 >> 4;
         } else {
 #pragma unroll
-            for (int i = 0; i < QT_VEC; ++i) {
-                const int q = (i * QT_THREADS + tid) * 4;
-                if (q < ne) vec(q, c[i], false);
+            for (int i = 0; i < QC_VEC; ++i) {
+                const int q = (i * 32 + lane) * 4;
+                if (q < ne) vec(q, c[i]);
             }
         }
         if (bad) ep_raise(status, EP_ERR_BAD_INDEX);
         my_cut += cut;
+        r_lo = n_lo, r_hi = n_hi, n_lo = nn_lo, n_hi = nn_hi;
+        row_s = next_s, row_e = next_e, row_l = next_l;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) my_cut += __shfl_xor_sync(FULL, my_cut, o);
-    __syncthreads();
     if (lane == 0 && my_cut) atomicAdd(&block_cut, my_cut);
     __syncthreads();
     if (threadIdx.x == 0 && block_cut) atomicAdd(edge_cut, block_cut);
@@ -300,7 +360,7 @@ static size_t quality_layout(int64_t N, int64_t nnz, int K, void *ws, QualityBuf
     Arena a(ws);
     QualityBuffers b{};
     b.lab = a.take<char>(((size_t)N + 4) * label_width(K));
-    b.tile_row = a.take<int32_t>(ceil_div(nnz, QT_EDGES) + 1);
+    b.tile_row = a.take<int32_t>(ceil_div(nnz, QC_EDGES) + 1);
     if (out) *out = b;
     return a.used;
 }
@@ -312,7 +372,7 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
                           int64_t N, int K, unsigned long long *edge_cut, unsigned long long *pv,
                           unsigned long long *pe, const QualityBuffers &b, cudaStream_t stream) {
     LabT *lab = static_cast<LabT *>(b.lab);
-    const int64_t ntiles = ceil_div(nnz, QT_EDGES);
+    const int64_t ntiles = ceil_div(nnz, QC_EDGES);
     const int pgrid = (int)std::max<int64_t>(1, std::min<int64_t>((int64_t)ctx->sm_count * 8, ceil_div(N, 256)));
     {
         Timed tm(ctx, stream, EP_TIMER_QUALITY_PREP);
@@ -323,7 +383,7 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
     }
     if (ntiles > 0) {
         Timed tm(ctx, stream, EP_TIMER_EDGE_CUT);
-        // labels in shared memory when they fit beside the kernel's static shared memory (about 10.3 KB per group)
+        // labels in shared memory when they fit beside the kernel's static shared memory (1.25 KB per warp)
         const size_t stat1 = 12 * 1024, stat4 = 44 * 1024;
         const size_t tab4 = ((size_t)N + 7) / 8 * 4 + 16, tab8 = ((size_t)N + 3) / 4 * 4 + 16;
         const size_t room = (size_t)ctx->smem_optin - stat4;
@@ -334,38 +394,38 @@ static int quality_launch(ep_ctx *ctx, const RowT *rowptr, const int32_t *colidx
         if constexpr (sizeof(LabT) == 1) if (use_tab) {
             launched = true;
             const size_t tab = pack == 4 ? tab4 : tab8;
-            // four small blocks per SM while four copies of the table fit, else one block of four groups
+            // four blocks of 8 warps per SM while four copies of the table fit, else one block of 32 warps
             const bool small = (tab + stat1) * 4 <= (size_t)ctx->smem_optin;
 #define EP_EC(P, G)                                                                                                  \
     do {                                                                                                             \
-        auto kern = edge_cut_tiles<RowT, LabT, P, G>;                                                                \
+        auto kern = edge_cut_chunks<RowT, LabT, P, G>;                                                               \
         EP_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab));             \
-        const int grid = (int)std::min<int64_t>(ceil_div(ntiles, (int64_t)G), (int64_t)ctx->sm_count * (G == 1 ? 4 : 1)); \
-        kern<<<grid, QT_THREADS * G, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut,       \
-                                                    ctx->d_status, 0, 0);                                            \
+        const int grid = (int)std::min<int64_t>(ceil_div(ntiles, (int64_t)G), (int64_t)ctx->sm_count * (G == 8 ? 4 : 1)); \
+        kern<<<grid, 32 * G, tab, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut,               \
+                                            ctx->d_status, 0, 0);                                                    \
     } while (0)
-            if (pack == 4 && small) EP_EC(4, 1);
-            else if (pack == 4) EP_EC(4, 4);
-            else if (small) EP_EC(8, 1);
-            else EP_EC(8, 4);
+            if (pack == 4 && small) EP_EC(4, 8);
+            else if (pack == 4) EP_EC(4, 32);
+            else if (small) EP_EC(8, 8);
+            else EP_EC(8, 32);
 #undef EP_EC
         }
         int launches = 1;
         if (!launched) {
-            const int grid = (int)std::min<int64_t>(ntiles, (int64_t)ctx->sm_count * 4);
+            const int grid = (int)std::min<int64_t>(ceil_div(ntiles, (int64_t)8), (int64_t)ctx->sm_count * 4);
             // Labels that cannot stay in the L2 beside the stream cost a DRAM sector per entry.  Then the vertex range
             // is cut into slices whose labels do fit, and the column ids are streamed once per slice: reading them
             // again is cheaper than missing on every gather.
             const size_t lab_total = (size_t)N * sizeof(LabT);
             const int slices = (int)std::min<size_t>(8, ceil_div(lab_total, (size_t)ctx->opt_slice_kb << 10));
             if (slices <= 1) {
-                edge_cut_tiles<RowT, LabT, 0, 1><<<grid, QT_THREADS, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row,
-                                                                                ntiles, edge_cut, ctx->d_status, 0, 0);
+                edge_cut_chunks<RowT, LabT, 0, 8><<<grid, 256, 0, stream>>>(rowptr, colidx, nnz, lab, N, b.tile_row, ntiles,
+                                                                            edge_cut, ctx->d_status, 0, 0);
             } else {
                 launches = slices;
                 for (int sl = 0; sl < slices; ++sl) {
                     const int32_t lo = (int32_t)(N * sl / slices), hi = (int32_t)(N * (sl + 1) / slices);
-                    edge_cut_tiles<RowT, LabT, 0, 1, true><<<grid, QT_THREADS, 0, stream>>>(
+                    edge_cut_chunks<RowT, LabT, 0, 8, true><<<grid, 256, 0, stream>>>(
                         rowptr, colidx, nnz, lab, N, b.tile_row, ntiles, edge_cut, ctx->d_status, lo, hi);
                 }
             }

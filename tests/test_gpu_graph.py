@@ -218,7 +218,7 @@ def test_host_buffer_entry_points_match_the_device_ones(ctx):
     assert torch.equal(hr.perm, r.perm.cpu()) and torch.equal(hr.inv_perm, r.inv_perm.cpu())
 
 
-@pytest.mark.parametrize("cluster_size", [0, 2, 8, 16])
+@pytest.mark.parametrize("cluster_size", [-1, 0, 2, 8, 16])
 def test_gather_yardsticks_sum_what_they_gather(ctx, cluster_size):
     """ep_probe_gather is the edge-cut pass reduced to its label lookups (a measuring stick for the bench): whatever
     memory serves the lookups, the sum must be that of the gathered bytes; entries outside [0, N) are skipped."""

@@ -112,6 +112,7 @@ struct TcState;                                   // tensor maps of one ep_kmean
 // Tensor map (128-byte swizzle) over a row-major [rows x d] fp32 matrix with boxes of box_rows x 32 floats;
 // `map` points at a CUtensorMap.
 bool tc_encode_kblock_map(void *map, const float *base, int64_t rows, int d, int box_rows);
+bool tc_encode_rowtile_map(void *map, const float *base, int64_t rows, int d, int box_rows);
 bool kmeans_tc_shape_ok(const ep_ctx *ctx, int d, int K);
 size_t kmeans_tc_state_bytes();
 size_t kmeans_tc_cand_bytes(const ep_ctx *ctx, int64_t N, int K);

@@ -621,6 +621,21 @@ bool tc_encode_kblock_map(void *map_out, const float *base, int64_t rows, int d,
 }
 
 
+// The same matrix (d a multiple of 32) seen as [d / 32 k-blocks][rows][32 floats], so that ONE box brings a tile of
+// `box_rows` rows with all its k-blocks, laid out in shared memory k-block after k-block exactly as the boxes of the map
+// above leave them one by one.  Coordinates: (0, first row, 0).
+bool tc_encode_rowtile_map(void *map_out, const float *base, int64_t rows, int d, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || d % 32 != 0 || d / 32 > 256 || box_rows > 256) return false;
+    CUtensorMap *map = static_cast<CUtensorMap *>(map_out);
+    const cuuint64_t dims[3] = {(cuuint64_t)32, (cuuint64_t)rows, (cuuint64_t)(d / 32)};
+    const cuuint64_t strides[2] = {(cuuint64_t)d * sizeof(float), (cuuint64_t)32 * sizeof(float)};
+    const cuuint32_t box[3] = {(cuuint32_t)32, (cuuint32_t)box_rows, (cuuint32_t)(d / 32)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 struct TcState {
     CUtensorMap map_x, map_c;

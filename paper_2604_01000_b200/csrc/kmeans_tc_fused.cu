@@ -281,7 +281,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 int d, int K, int npad, int num_kb, int stages, uint32_t idesc, uint32_t tmem_cols, uint32_t key_mask,
                 int32_t *__restrict__ assign, float *psum, int *pcnt,
                 int4 *late_list, int64_t late_cap, int late_chunk, int T, int update_here, int use_prev0, int keep_centroids,
-                double *objterm, double *objective, const double *__restrict__ x2part, int x2n, unsigned *grid_bar,
+                double *objterm, double *objective, const double *__restrict__ x2part, int x2n, int x_one_box,
+                unsigned *grid_bar,
                 unsigned long long *counters, int *status) {
     // The swizzled tiles need 1024-byte alignment.  The array is used as declared (no pointer arithmetic
     // through integers), so that every access below stays a shared-memory instruction; should a launch
@@ -389,25 +390,31 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     __syncthreads();
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- TMA producer: the whole warp runs the
+        // loop (warp-uniform control flow and operands), one elected lane issues.  x_one_box: map_x is the
+        // three-dimensional view of X and one box brings a whole tile; else one box per k-block.
+        {
             // the centroids' TF32 copy of this iteration (written by other blocks through ordinary stores)
             asm volatile("fence.proxy.async;" ::: "memory");
-            mbar_expect_tx(&sh->c_full, (uint32_t)(num_kb * c_kb_bytes));
+            mbar_expect_tx_elected(&sh->c_full, (uint32_t)(num_kb * c_kb_bytes));
 #pragma unroll 1
             for (int kb = 0; kb < num_kb; ++kb)
-                tma_load_2d(c_smem + (size_t)kb * c_kb_bytes, &map_c, kb * KBLK, 0, &sh->c_full);
+                tma_load_2d_elected(smem_u32(c_smem) + (uint32_t)(kb * c_kb_bytes), &map_c, kb * KBLK, 0, &sh->c_full);
             uint32_t it = it_base;
             for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
-                if (!mbar_wait(&sh->x_empty[s], ph ^ 1u, abort_flag)) break;
-                mbar_expect_tx(&sh->x_full[s], (uint32_t)stage_bytes);
+                if (!__all_sync(FULL, mbar_wait(&sh->x_empty[s], ph ^ 1u, abort_flag))) break;
+                mbar_expect_tx_elected(&sh->x_full[s], (uint32_t)stage_bytes);
+                const uint32_t dst = smem_u32(x_smem) + s * (uint32_t)stage_bytes;
+                if (x_one_box) {
+                    tma_load_3d_elected(dst, &map_x, 0, (int)(tile * BMR), 0, &sh->x_full[s]);
+                } else {
 #pragma unroll 1
-                for (int kb = 0; kb < num_kb; ++kb)
-                    tma_load_2d(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK,
-                                (int)(tile * BMR), &sh->x_full[s]);
+                    for (int kb = 0; kb < num_kb; ++kb)
+                        tma_load_2d_elected(dst + (uint32_t)(kb * X_KB_BYTES), &map_x, kb * KBLK, (int)(tile * BMR), &sh->x_full[s]);
+                }
             }
-            if (*abort_flag) {
+            if (lane == 0 && *abort_flag) {
                 // On the way out after an abort: the loads already issued get time to land, so that nothing of this
                 // block's own still writes into its shared memory when it leaves.
                 mbar_wait_quiet(&sh->c_full, ipar, DRAIN_LIMIT_CLOCKS);
@@ -417,29 +424,27 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            bool ok = mbar_wait(&sh->c_full, ipar, abort_flag);
+        // ---------------------------------------------------------------- MMA issuer: the whole warp runs the loop,
+        // one elected lane issues (see the elected forms in tc_device.cuh)
+        {
+            bool ok = __all_sync(FULL, mbar_wait(&sh->c_full, ipar, abort_flag));
             uint32_t it = it_base;
             for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
-                if (!(ok = mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag))) break;
-                if (!(ok = mbar_wait(&sh->x_full[s], ph, abort_flag))) break;
+                if (!(ok = __all_sync(FULL, mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag)))) break;
+                if (!(ok = __all_sync(FULL, mbar_wait(&sh->x_full[s], ph, abort_flag)))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)KMAX;
+                const uint32_t a_addr = smem_u32(x_smem) + s * (uint32_t)stage_bytes, b_addr = smem_u32(c_smem);
+                static_assert(KBLK == 32, "umma_tf32_kblock_elected issues the four K-steps of a 32-float k-block");
 #pragma unroll 1
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)s * stage_bytes + (size_t)kb * X_KB_BYTES));
-                    const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)kb * c_kb_bytes));
-#pragma unroll
-                    for (int ks = 0; ks < KBLK / 8; ++ks)
-                        umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), idesc,
-                                  (kb | ks) != 0 ? 1u : 0u);
-                }
-                umma_commit(&sh->t_full[buf]);
+                for (int kb = 0; kb < num_kb; ++kb)
+                    umma_tf32_kblock_elected(d_tmem, umma_desc(a_addr + (uint32_t)(kb * X_KB_BYTES)),
+                                             umma_desc(b_addr + (uint32_t)(kb * c_kb_bytes)), idesc, (uint32_t)kb);
+                umma_commit_elected(&sh->t_full[buf]);
             }
-            if (!ok || *abort_flag) {
+            if (lane == 0 && (!ok || *abort_flag)) {
                 // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
                 // here must have completed
                 umma_commit(&sh->drain);                  // only ever used once: the block leaves after an abort
@@ -987,7 +992,7 @@ namespace ep {
 
 struct TcFusedState {
     CUtensorMap map_x, map_c;
-    int npad, num_kb, stages, grid, late_chunk;
+    int npad, num_kb, stages, grid, late_chunk, x_one_box;
     int64_t late_cap;
     size_t smem;
     uint32_t tmem_cols;
@@ -1057,7 +1062,10 @@ int kmeans_tcf_prepare(ep_ctx *ctx, const float *emb, int64_t N, int d, int K, c
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)st->npad) cols <<= 1;
     st->tmem_cols = cols;
-    if (!tc_encode_kblock_map(&st->map_x, emb, N, d, tcf_tile_rows(d)) || !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
+    // one box per tile where the rows are whole k-blocks; else (and should the driver refuse the view) a box per k-block
+    st->x_one_box = (d % KBLK == 0 && tc_encode_rowtile_map(&st->map_x, emb, N, d, tcf_tile_rows(d))) ? 1 : 0;
+    if ((!st->x_one_box && !tc_encode_kblock_map(&st->map_x, emb, N, d, tcf_tile_rows(d))) ||
+        !tc_encode_kblock_map(&st->map_c, ct, K, d, st->npad))
         return fail(ctx, EP_ERR_CUDA, "cuTensorMapEncodeTiled failed for N=%lld d=%d K=%d", (long long)N, d, K);
     return EP_OK;
 }
@@ -1077,11 +1085,12 @@ static int tcf_launch(ep_ctx *ctx, const TcFusedState &st, const float *emb, flo
     int npad = st.npad, num_kb = st.num_kb, stages = st.stages, late_chunk = st.late_chunk;
     uint32_t idesc = umma_idesc_tf32_m128(st.npad), tmem_cols = st.tmem_cols, key_mask = ~IDX_MASK;
     int64_t late_cap = st.late_cap;
+    int x_one_box = st.x_one_box;
     int *status = ctx->d_status;
     void *args[] = {&map_x, &map_c, &emb, &centroids, &cn, &ct, &clo, &rownorm, &N, &d, &K, &npad, &num_kb, &stages, &idesc,
                     &tmem_cols, &key_mask, &assign, &psum, &pcnt, &late_list, &late_cap, &late_chunk, &T, &update_here, &use_prev0,
                     &keep_centroids,
-                    &objterm, &objective, &x2part, &x2n, &grid_bar, &counters, &status};
+                    &objterm, &objective, &x2part, &x2n, &x_one_box, &grid_bar, &counters, &status};
     if (update_here)   // one block per SM, all resident together: they meet on a grid-wide barrier twice per iteration
         EP_CUDA(ctx, cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(st.grid), dim3(THREADS), args, st.smem, stream));
     else

@@ -81,6 +81,54 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
         : "memory");
 }
 
+// "Elected" forms for a warp that runs its issue loop as a whole (all lanes wait, count and compute the same
+// operands) and lets one lane, chosen by elect.sync, issue.  The operands of TMA and MMA instructions are
+// warp-level values; with the loop inside `if (lane == 0)` the same instructions cost far more issue time
+// (measured in the fused small-K kernel: 82 -> 54 clocks per tcgen05.mma, which had been the slowest link of the
+// pipeline for 256-column rows).
+__device__ __forceinline__ void mbar_expect_tx_elected(uint64_t *bar, uint32_t bytes) {
+    asm volatile("{\n.reg .pred pe;\nelect.sync _|pe, 0xffffffff;\n"
+                 "@pe mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n}" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_elected(uint32_t dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("{\n.reg .pred pe;\nelect.sync _|pe, 0xffffffff;\n"
+                 "@pe cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_elected(uint32_t dst, const CUtensorMap *map, int x, int y, int z,
+                                                    uint64_t *bar) {
+    asm volatile("{\n.reg .pred pe;\nelect.sync _|pe, 0xffffffff;\n"
+                 "@pe cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n}"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+                 : "memory");
+}
+// The four K-steps (8 floats each) of one 128-byte k-block; the first one overwrites the accumulator when
+// accumulate_first == 0.
+__device__ __forceinline__ void umma_tf32_kblock_elected(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                         uint32_t accumulate_first) {
+    asm volatile(
+        "{\n.reg .pred pe, pa, pt;\n.reg .b64 a1, a2, a3, b1, b2, b3;\n"
+        "elect.sync _|pe, 0xffffffff;\n"
+        "setp.ne.b32 pa, %4, 0;\n"
+        "setp.eq.b32 pt, 0, 0;\n"
+        "add.s64 a1, %1, 2;\nadd.s64 a2, %1, 4;\nadd.s64 a3, %1, 6;\n"
+        "add.s64 b1, %2, 2;\nadd.s64 b2, %2, 4;\nadd.s64 b3, %2, 6;\n"
+        "@pe tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, pa;\n"
+        "@pe tcgen05.mma.cta_group::1.kind::tf32 [%0], a1, b1, %3, pt;\n"
+        "@pe tcgen05.mma.cta_group::1.kind::tf32 [%0], a2, b2, %3, pt;\n"
+        "@pe tcgen05.mma.cta_group::1.kind::tf32 [%0], a3, b3, %3, pt;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_elected(uint64_t *bar) {
+    asm volatile("{\n.reg .pred pe;\nelect.sync _|pe, 0xffffffff;\n"
+                 "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+                 ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
 // Plain bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from global to this block's shared
 // memory; the barrier receives the bytes as they land.
 __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {

@@ -65,11 +65,11 @@ enum {
                                are streamed once per slice, so that a slice's labels stay in the L2.  The result
                                does not depend on it */
     ,
-    EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH = 6 /* the fused small-K tensor-core pass (2 <= K <= 64): 2 = all Lloyd iterations
-                               of a call inside one launch, the blocks updating the centroids themselves between grid-wide
-                               barriers; 1 = one launch per iteration plus the update kernel; 0 = by size (default: one
-                               launch while a pass reads at most 512 MiB).  The labels do not depend on it; centroids
-                               may differ in the last bit (another fixed order of the fp64 fold) */
+    EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH = 6 /* the fused small-K tensor-core pass (2 <= K <= 64): 0 (default) or 2 = all
+                               Lloyd iterations of a call inside one launch, the blocks updating the centroids themselves
+                               between grid-wide barriers; 1 = one launch per iteration plus the update kernel.  The
+                               labels do not depend on it; centroids may differ in the last bit (another fixed order of
+                               the fp64 fold) */
 };
 
 /* Timers kept while EP_OPT_PROFILE is 1. */

@@ -241,7 +241,7 @@ class Context:
             self._raise(rc)
 
     def set_kmeans_iterations_per_launch(self, mode: int):
-        """0 = by size, 1 = one launch per Lloyd iteration, 2 = all iterations in one launch (fused small-K pass)."""
+        """0 or 2 = all iterations in one launch (default), 1 = one launch per Lloyd iteration (fused small-K pass)."""
         rc = self._lib.ep_set_option(self._h, EP_OPT_KMEANS_ITERATIONS_PER_LAUNCH, int(mode))
         if rc != EP_OK:
             self._raise(rc)

@@ -736,7 +736,7 @@ size_t kmeans_workspace_layout(const ep_ctx *ctx, const KMeansPlan &p, void *wor
         b.rownorm = a.take<float2>(p.N);
         if (p.tc_fused) {
             b.late_list = a.take<int4>((size_t)kmeans_tcf_late_cap(ctx, p.N, p.d) * 4 * p.grid);
-            b.grid_bar = a.take<unsigned>(64);
+            b.grid_bar = a.take<unsigned>(64 + 64 * 16 * 4 * 2);   // the barrier word, then 32 KB for the update's shares
         } else {
             b.cand = a.take<char>(kmeans_tc_cand_bytes(ctx, p.N, p.K));
             b.cmaxima = a.take<float>(2);
@@ -780,11 +780,10 @@ int kmeans_run(ep_ctx *ctx, const KMeansPlan &p, const float *emb, int iters, co
     }
 
     const int T = iters > 0 ? iters : 1;
-    // Few centroids on the tensor cores.  Inputs up to a few hundred MB per pass run all their iterations, centroid
-    // updates included, inside one launch: there the gaps and prologues between launches cost more than the passes.
-    // Longer passes keep one launch per iteration and the update kernel of the other paths (it spreads over more SMs).
-    const bool one_launch = p.tc_fused && (ctx->opt_iters_per_launch == 2 ||
-                                           (ctx->opt_iters_per_launch == 0 && (size_t)N * d * sizeof(float) <= ((size_t)512 << 20)));
+    // Few centroids on the tensor cores: all iterations of the call, centroid updates included, run inside one launch
+    // (no gaps, prologues or second kernels between iterations; measured faster at every size from 10 K to 111 M rows).
+    // One launch per iteration plus the update kernel of the other paths remains as an option.
+    const bool one_launch = p.tc_fused && ctx->opt_iters_per_launch != 1;
     if (one_launch) {
         int rc = kmeans_tcf_run(ctx, *tcf_state, emb, centroids, b.cnorm, b.ct, b.clo, b.rownorm, N, d, K, assign, b.psum, b.pcnt,
                                 b.late_list, T, /*update_here=*/true, false, iters == 0, b.objterm, objective, b.x2part,

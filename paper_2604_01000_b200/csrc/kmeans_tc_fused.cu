@@ -180,68 +180,105 @@ __device__ __forceinline__ float tf32_nearest(float x) {
     return __uint_as_float(r);
 }
 
-// Centroid update of cluster k by the whole block: S_k = sum over the blocks' partial sums in fp64.  A thread takes
-// four columns; the thread groups (THREADS / (d / 4, rounded up to a warp) of them) take contiguous shares of the
-// slabs, in slab order, and the group sums are added in group order: a fixed tree.  c_k <- S_k / n_k when n_k > 0,
-// else unchanged; |c_k|^2 of the new centroid, its TF32-rounded copy and what that copy misses, and the cluster's share
-// n_k |c|^2 - 2 c.S_k of the objective (c = the centroid the rows were assigned against).  Everything other blocks
-// wrote is read past the L1.  buf: 4 x THREADS + 64 doubles of shared memory.
-__device__ __noinline__ void update_cluster(int k, int K, int d, int parts, const float *psum, const int *pcnt, float *C,
-                                               float *cnorm, float *ct, float *clo, double *objterm, int keep_centroids,
-                                               double *buf) {
-    const int d4 = d >> 2, d4pad = (d4 + 31) / 32 * 32;
-    const int G = max(1, THREADS / d4pad);
-    const int g = threadIdx.x / d4pad, q = threadIdx.x - g * d4pad;
-    double *red = buf + 4 * THREADS;
+// The centroid update shared out over the whole grid: a unit is W four-float columns of one cluster (W a power of
+// two, at most 32), so that K x ceil(d / 4W) units keep about every block busy and a block pulls only 16 W bytes of
+// each slab.  Groups of W threads take contiguous shares of the slabs in slab order; the groups of a warp are added by
+// a butterfly, the warps in warp order: a fixed tree.  The unit writes its columns of c_k and of the TF32 copy, and to
+// tpart[unit] its share of (n_k |c|^2 - 2 c.S_k, |c'|^2, |c' - tf32(c')|^2); whoever needs |c'|^2, the residual or the
+// objective of a cluster adds the shares of its units in unit order (cluster_terms).  buf: 4 x 16 x 32 + 64 doubles.
+constexpr int UPDATE_MAX_CHUNKS = 16;
+__device__ __forceinline__ int update_chunk_width(int K, int d4, int grid) {
+    int W = 1;
+    while (W < 32 && (K * ((d4 + W - 1) / W) > grid || (d4 + W - 1) / W > UPDATE_MAX_CHUNKS)) W <<= 1;
+    return W;
+}
+__device__ __noinline__ void update_unit(int k, int c, int W, int K, int d, int parts, const float *psum, const int *pcnt,
+                                            float *C, float *ct, double *tpart_unit, int keep_centroids, double *buf) {
+    const int d4 = d >> 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = THREADS / W, g = threadIdx.x / W, q = threadIdx.x & (W - 1);
+    const int col = c * W + q;                                   // this thread's four columns
+    double *red = buf + 4 * (THREADS / 32) * 32;
+    // every load is issued before anything waits on one
     double sums[4] = {0.0, 0.0, 0.0, 0.0};
     for (int p = threadIdx.x; p < parts; p += THREADS) sums[0] += (double)__ldcg(pcnt + (size_t)p * K + k);
+    float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (g == 0 && col < d4) c4 = __ldcg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + col);
+    double part[4] = {0.0, 0.0, 0.0, 0.0};
+    if (col < d4) {
+        const int p0 = (int)((long long)parts * g / G), p1 = (int)((long long)parts * (g + 1) / G);
+        const float4 *src = reinterpret_cast<const float4 *>(psum) + (size_t)k * d4 + col;
+        const size_t pitch = (size_t)K * d4;
+#pragma unroll 1
+        for (int pb = p0; pb < p1; pb += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                v[u] = pb + u < p1 ? __ldcg(src + (size_t)(pb + u) * pitch) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                part[0] += (double)v[u].x;
+                part[1] += (double)v[u].y;
+                part[2] += (double)v[u].z;
+                part[3] += (double)v[u].w;
+            }
+        }
+    }
     block_sum4(sums, red);
     const long long n = (long long)sums[0];                     // counts are far below 2^53: exact
-    double part[4] = {0.0, 0.0, 0.0, 0.0};
-    if (g < G && q < d4) {
-        const int p0 = (int)((long long)parts * g / G), p1 = (int)((long long)parts * (g + 1) / G);
-        const float4 *src = reinterpret_cast<const float4 *>(psum) + (size_t)k * d4 + q;
-        const size_t pitch = (size_t)K * d4;
-#pragma unroll 8
-        for (int p = p0; p < p1; ++p) {
-            const float4 v = __ldcg(src + (size_t)p * pitch);
-            part[0] += (double)v.x;
-            part[1] += (double)v.y;
-            part[2] += (double)v.z;
-            part[3] += (double)v.w;
+    for (int o = 16; o >= W; o >>= 1)                            // the groups of this warp (lanes that differ above q)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) part[i] += __shfl_xor_sync(FULL, part[i], o);
+    __syncthreads();
+    if (lane < W)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) buf[(i * (THREADS / 32) + warp) * 32 + lane] = part[i];
+    __syncthreads();
+    if (warp == 0) {
+        double t[3] = {0.0, 0.0, 0.0};                          // n |c|^2 - 2 c.S, |c'|^2, |c' - tf32(c')|^2 of these columns
+        if (lane < W && col < d4) {
+            const float cold[4] = {c4.x, c4.y, c4.z, c4.w};
+            float cnew[4], crnd[4];
+            double cs = 0.0, cc = 0.0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                double S = 0.0;
+                for (int w = 0; w < THREADS / 32; ++w) S += buf[(i * (THREADS / 32) + w) * 32 + lane];
+                cnew[i] = (n > 0 && !keep_centroids) ? (float)(S / (double)n) : cold[i];
+                crnd[i] = tf32_nearest(cnew[i]);
+                const double lo = (double)cnew[i] - (double)crnd[i];
+                cs += (double)cold[i] * S;
+                cc += (double)cold[i] * (double)cold[i];
+                t[1] += (double)cnew[i] * (double)cnew[i];
+                t[2] += lo * lo;
+            }
+            t[0] = (double)n * cc - 2.0 * cs;
+            reinterpret_cast<float4 *>(C)[(size_t)k * d4 + col] = make_float4(cnew[0], cnew[1], cnew[2], cnew[3]);
+            reinterpret_cast<float4 *>(ct)[(size_t)k * d4 + col] = make_float4(crnd[0], crnd[1], crnd[2], crnd[3]);
+        }
+        for (int o = W >> 1; o >= 1; o >>= 1)
+#pragma unroll
+            for (int i = 0; i < 3; ++i) t[i] += __shfl_xor_sync(FULL, t[i], o);
+        if (lane == 0) {
+            tpart_unit[0] = t[0];
+            tpart_unit[1] = t[1];
+            tpart_unit[2] = t[2];
         }
     }
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < 4; ++i) buf[i * THREADS + threadIdx.x] = part[i];
-    __syncthreads();
-    double t[4] = {0.0, 0.0, 0.0, 0.0};                          // c.S, |c|^2, |c'|^2, |c' - tf32(c')|^2
-    if (g == 0 && q < d4) {
-        float cold[4], cnew[4], crnd[4];
-        const float4 c4 = __ldcg(reinterpret_cast<const float4 *>(C) + (size_t)k * d4 + q);
-        cold[0] = c4.x, cold[1] = c4.y, cold[2] = c4.z, cold[3] = c4.w;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            double S = buf[i * THREADS + q];
-            for (int gg = 1; gg < G; ++gg) S += buf[i * THREADS + gg * d4pad + q];
-            cnew[i] = (n > 0 && !keep_centroids) ? (float)(S / (double)n) : cold[i];
-            crnd[i] = tf32_nearest(cnew[i]);
-            const double lo = (double)cnew[i] - (double)crnd[i];
-            t[0] += (double)cold[i] * S;
-            t[1] += (double)cold[i] * (double)cold[i];
-            t[2] += (double)cnew[i] * (double)cnew[i];
-            t[3] += lo * lo;
-        }
-        reinterpret_cast<float4 *>(C)[(size_t)k * d4 + q] = make_float4(cnew[0], cnew[1], cnew[2], cnew[3]);
-        reinterpret_cast<float4 *>(ct)[(size_t)k * d4 + q] = make_float4(crnd[0], crnd[1], crnd[2], crnd[3]);
+}
+// A cluster's (objective term, |c|^2, residual |c - tf32(c)|) from the shares of its units, in unit order.
+__device__ __forceinline__ void cluster_terms(const double *tpart, int k, int chunks, double &obj, float &cnorm, float &clo) {
+    double t0 = 0.0, t1 = 0.0, t2 = 0.0;
+    for (int c = 0; c < chunks; ++c) {
+        const double *u = tpart + (size_t)(k * chunks + c) * 4;
+        t0 += __ldcg(u + 0);
+        t1 += __ldcg(u + 1);
+        t2 += __ldcg(u + 2);
     }
-    block_sum4(t, red);
-    if (threadIdx.x == 0) {
-        cnorm[k] = (float)t[2];
-        objterm[k] = (double)n * t[1] - 2.0 * t[0];
-        clo[k] = (float)(sqrt(t[3]) * 1.000001);
-    }
-    __syncthreads();
+    obj = t0;
+    cnorm = (float)t1;
+    clo = (float)(sqrt(t2) * 1.000001);
 }
 
 // J of an iteration = sum_i |x_i|^2 + sum_k (n_k |c_k|^2 - 2 c_k.S_k), both summed in a fixed order, by one block.
@@ -383,9 +420,27 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     uint32_t chunk_it = 0;
     const long long clk_start = clock64();
     if (threadIdx.x < 4) sh->late_n[threadIdx.x] = 0;
+    // |c|^2 and the TF32 residual of every centroid: from the caller's arrays, or (after an update inside this launch)
+    // from the shares the update's units left, which every block adds up in the same order
+    float *clo_s = reinterpret_cast<float *>(sh->hcnt[0]);      // warp 2's scratch, not in use before its first tile
+    double *tpart = reinterpret_cast<double *>(grid_bar + 64);
+    const int upd_W = update_chunk_width(K, d >> 2, (int)gridDim.x), upd_chunks = ((d >> 2) + upd_W - 1) / upd_W;
     for (int k = threadIdx.x; k < MAX_K; k += blockDim.x) {
         sh->cnt[k] = 0;
-        sh->cn[k] = k < KMAX ? __ldcg(cn + k) : CUDART_INF_F;     // cn is padded with a huge value beyond K
+        float cnk = CUDART_INF_F, clk = 0.f;                     // beyond K: a huge norm, so that no row goes there
+        if (k < K) {
+            if (PERSISTENT && iter > 0) {
+                double obj;
+                cluster_terms(tpart, k, upd_chunks, obj, cnk, clk);
+            } else {
+                cnk = __ldcg(cn + k);
+                clk = __ldcg(clo + k);
+            }
+        } else if (k < KMAX) {
+            cnk = __ldcg(cn + k);
+        }
+        sh->cn[k] = cnk;
+        clo_s[k] = clk;
     }
     __syncthreads();
 
@@ -568,8 +623,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float m2 = 0.f, ml = 0.f;                          // largest centroid norm and rounding residual
 #pragma unroll 1
         for (int k = lane; k < K; k += 32) {
-            m2 = fmaxf(m2, __ldcg(cn + k));
-            ml = fmaxf(ml, __ldcg(clo + k));
+            m2 = fmaxf(m2, sh->cn[k]);
+            ml = fmaxf(ml, clo_s[k]);
         }
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) {
@@ -944,12 +999,25 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (!grid_barrier(grid_bar, grid_arrivals, abort_flag)) break;
         double *buf = reinterpret_cast<double *>(x_smem);     // the block's sums are published: the ring is free again
 #pragma unroll 1
-        for (int k = blockIdx.x; k < K; k += gridDim.x)
-            update_cluster(k, K, d, (int)gridDim.x, psum, pcnt, centroids, cn, ct, clo, objterm, keep_centroids, buf);
+        for (int u = blockIdx.x; u < K * upd_chunks; u += gridDim.x)
+            update_unit(u / upd_chunks, u % upd_chunks, upd_W, K, d, (int)gridDim.x, psum, pcnt, centroids, ct,
+                        tpart + (size_t)u * 4, keep_centroids, buf);
         asm volatile("fence.proxy.async;" ::: "memory");      // ct is next read by the TMA loads of other blocks
         grid_arrivals += gridDim.x;
         if (!grid_barrier(grid_bar, grid_arrivals, abort_flag)) break;
         if (threadIdx.x == 0) even_out_phases(nt, chunk_it);      // nothing of this iteration is in flight any more
+        if (blockIdx.x == 0) {
+            // the caller's arrays (what a later launch, or the objective below, reads) from the units' shares
+            for (int k = threadIdx.x; k < K; k += THREADS) {
+                double obj;
+                float cnk, clk;
+                cluster_terms(tpart, k, upd_chunks, obj, cnk, clk);
+                objterm[k] = obj;
+                cn[k] = cnk;
+                clo[k] = clk;
+            }
+            __syncthreads();
+        }
         if (counters && blockIdx.x == 0 && threadIdx.x == 0) {
             const long long clk_end = clock64();
             atomicAdd(&counters[5], (unsigned long long)(clk_published - clk_start));

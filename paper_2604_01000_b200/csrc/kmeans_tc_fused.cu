@@ -133,8 +133,9 @@ constexpr long long GRID_WAIT_CLOCKS = 4000000000ll;
 __device__ __noinline__ bool grid_barrier(unsigned *bar, unsigned target, volatile int *abort_flag) {
     __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(bar, 1u);
+        // the arrival releases what this block wrote (the __syncthreads above ordered the other threads' writes before
+        // it); the acquiring load that sees the last arrival makes every block's writes visible here
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
         const long long t0 = clock64();
         for (unsigned spins = 0;; ++spins) {
             unsigned seen;
@@ -144,9 +145,7 @@ __device__ __noinline__ bool grid_barrier(unsigned *bar, unsigned target, volati
                 *abort_flag = 1;
                 break;
             }
-            __nanosleep(40);
         }
-        __threadfence();
     }
     __syncthreads();
     return *abort_flag == 0;

@@ -721,7 +721,7 @@ def main():
 
         run_host_steps(2)
         barrier()
-        e_steps = max(2, min(args.steps, 4))
+        e_steps = max(2, min(args.steps, 8))
         start.record()
         run_host_steps(e_steps)
         stop.record()

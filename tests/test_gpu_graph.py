@@ -136,7 +136,7 @@ def test_odd_csr_shapes_one_table_per_sm(ctx):
             _quality_matches(ctx, rp, torch.from_numpy(colidx).cuda(), _random_labels(N, K, 4), K)
 
 
-@pytest.mark.parametrize("nnz", [0, 1, 3, 4, 5, 8191, 8192, 8193, 16_387])
+@pytest.mark.parametrize("nnz", [0, 1, 3, 4, 5, 1023, 1024, 1025, 2047, 2049, 8191, 8192, 8193, 16_387])
 def test_tile_boundaries(ctx, nnz):
     rng = np.random.default_rng(nnz)
     N = 97
@@ -145,6 +145,37 @@ def test_tile_boundaries(ctx, nnz):
     colidx = rng.integers(0, N, size=nnz).astype(np.int32)
     ci = torch.from_numpy(colidx).cuda() if nnz else torch.empty(0, dtype=torch.int32, device="cuda")
     _quality_matches(ctx, torch.from_numpy(rowptr).cuda(), ci, _random_labels(N, 5, 7), 5)
+
+
+@pytest.mark.parametrize("K", [3, 16, 200, 70_000])
+@pytest.mark.parametrize("shape", ["short_rows", "dense_small", "starts_on_chunk_boundaries"])
+def test_row_starts_everywhere_in_a_chunk(ctx, shape, K):
+    """A warp works through 1024-entry chunks of the CSR arrays and rebuilds every entry's row from the row starts inside
+    its chunk: hundreds of one- and two-entry rows per chunk (more than the 32 whose look-ups run ahead), rows that
+    start inside a four-entry vector, on a chunk's first entry or on its last, with the labels gathered from global
+    memory, from a byte table and from a nibble table in shared memory."""
+    rng = np.random.default_rng(K + len(shape))
+    if shape == "short_rows":
+        N = 60_000
+        deg = rng.integers(0, 4, size=N)
+    elif shape == "dense_small":
+        N = 3_000                                       # 148 N <= 2 nnz: the labels go to shared memory when K <= 256
+        deg = rng.integers(150, 260, size=N)
+    else:
+        N = 4_000
+        deg = rng.integers(100, 400, size=N)
+        pos = 0
+        for i in range(N):                              # every seventh row ends on a multiple of 1024, one before or one after
+            if i % 7 == 0:
+                end = (pos + int(deg[i]) + 1023) // 1024 * 1024 + (i // 7) % 3 - 1
+                deg[i] = end - pos
+            pos += int(deg[i])
+    rowptr = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+    nnz = int(rowptr[-1])
+    colidx = rng.integers(0, N, size=nnz).astype(np.int32)
+    labels = _random_labels(N, K, 11)
+    for dtype in (torch.int32, torch.int64):
+        _quality_matches(ctx, torch.from_numpy(rowptr).to(dtype).cuda(), torch.from_numpy(colidx).cuda(), labels, K)
 
 
 def test_bad_indices_raise_a_status_without_faulting(ctx):

@@ -1033,39 +1033,23 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
 }
 
-// rownorm[i] = (|x_i|_2, |x_i - trunc_tf32(x_i)|_2), both rounded up a little; a warp per row, four rows of a warp in
-// flight at a time (one row's 16-byte loads per lane do not cover the memory latency).
+// rownorm[i] = (|x_i|_2, |x_i - trunc_tf32(x_i)|_2), both rounded up a little; one warp per row.
 __global__ void __launch_bounds__(256) row_norms(const float *__restrict__ emb, int64_t N, int d, float2 *__restrict__ out) {
-    constexpr int RN = 4;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, d4 = d >> 2;
-    const int64_t stride = (int64_t)gridDim.x * 8;
-    for (int64_t row0 = (int64_t)blockIdx.x * 8 + warp; row0 < N; row0 += stride * RN) {
-        float x2[RN], xl2[RN];
-#pragma unroll
-        for (int u = 0; u < RN; ++u) x2[u] = xl2[u] = 0.f;
+    for (int64_t row = (int64_t)blockIdx.x * 8 + warp; row < N; row += (int64_t)gridDim.x * 8) {
+        float x2 = 0.f, xl2 = 0.f;
         for (int q = lane; q < d4; q += 32) {
-            float4 x[RN];
-#pragma unroll
-            for (int u = 0; u < RN; ++u) {
-                const int64_t row = row0 + u * stride;
-                x[u] = row < N ? ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < RN; ++u) {
-                x2[u] = dot4(x[u], x[u], x2[u]);
-                const float4 r = make_float4(x[u].x - __uint_as_float(__float_as_uint(x[u].x) & 0xFFFFE000u),
-                                             x[u].y - __uint_as_float(__float_as_uint(x[u].y) & 0xFFFFE000u),
-                                             x[u].z - __uint_as_float(__float_as_uint(x[u].z) & 0xFFFFE000u),
-                                             x[u].w - __uint_as_float(__float_as_uint(x[u].w) & 0xFFFFE000u));
-                xl2[u] = dot4(r, r, xl2[u]);
-            }
+            const float4 x = ldg_stream(reinterpret_cast<const float4 *>(emb) + row * d4 + q);
+            x2 = dot4(x, x, x2);
+            const float4 r = make_float4(x.x - __uint_as_float(__float_as_uint(x.x) & 0xFFFFE000u),
+                                         x.y - __uint_as_float(__float_as_uint(x.y) & 0xFFFFE000u),
+                                         x.z - __uint_as_float(__float_as_uint(x.z) & 0xFFFFE000u),
+                                         x.w - __uint_as_float(__float_as_uint(x.w) & 0xFFFFE000u));
+            xl2 = dot4(r, r, xl2);
         }
-#pragma unroll
-        for (int u = 0; u < RN; ++u) {
-            const int64_t row = row0 + u * stride;
-            const float a = warp_sum(x2[u]), b = warp_sum(xl2[u]);
-            if (lane == 0 && row < N) out[row] = make_float2(sqrtf(a) * 1.000001f, sqrtf(b) * 1.000001f);
-        }
+        x2 = warp_sum(x2);
+        xl2 = warp_sum(xl2);
+        if (lane == 0) out[row] = make_float2(sqrtf(x2) * 1.000001f, sqrtf(xl2) * 1.000001f);
     }
 }
 

@@ -41,6 +41,10 @@ NCU_TRAFFIC = {
     ("kmeans_assign_K16", "cfg3"): {"bytes_per_launch": (7_215_130_000 + 104_238_336) // 30,
                                     "launch": "all rows, one iteration (a thirtieth of the 30-iteration launch)",
                                     "source": "profiles/kmeans_tc_fused_K16_cfg3_all_iterations.md"},
+    # captured on 12 M rows of the same recipe: (522.2 + 4.6) bytes per row and iteration there, times cfg5's rows
+    ("kmeans_assign_K64", "cfg5"): {"bytes_per_launch": int(111_059_956 * (125_337_159_000 + 1_102_900_000) / (20 * 12_000_000)),
+                                    "launch": "all rows, one iteration, scaled by the rows from a 12 M-row capture",
+                                    "source": "profiles/kmeans_tc_fused_K64_cfg5_12M_rows_all_iterations.md"},
     ("edge_cut", "cfg4"): {"bytes_per_launch": 507_021_824 + 3_238_656, "launch": "all entries",
                            "source": "profiles/edge_cut_chunks_cfg4.md"},
     ("edge_cut", "cfg3"): {"bytes_per_launch": 438_612_224 + 3_328_512, "launch": "all entries",

@@ -117,29 +117,31 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const uint32_t tmem_base = sh->tmem_base;
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- TMA producer: the whole warp runs the loop
+        // (uniform control flow and operands), one elected lane issues (see the elected forms in tc_device.cuh)
+        {
             uint32_t it = 0;
             bool ok = true;
             int64_t x_tile = -1;                                   // local index of the last tile any k-block was loaded for
+            const uint32_t x_base = smem_u32(x_smem), c_base = smem_u32(c_smem);
             for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
                 const int row0 = (int)(row_begin + tile * BM);
                 for (int nt = 0; ok && nt < num_nt; ++nt) {
                     for (int kb = 0; kb < num_kb; ++kb, ++it) {
                         if (nt == 0) {   // this tile's rows, one k-block at a time, as the previous tile lets go of them
-                            if (!(ok = mbar_wait(&sh->x_empty[kb], (uint32_t)(lt & 1) ^ 1u, abort_flag))) break;
-                            mbar_expect_tx(&sh->x_full[kb], X_KB_BYTES);
-                            tma_load_2d(x_smem + (size_t)kb * X_KB_BYTES, &map_x, kb * KBLK, row0, &sh->x_full[kb]);
+                            if (!(ok = __all_sync(FULL, mbar_wait(&sh->x_empty[kb], (uint32_t)(lt & 1) ^ 1u, abort_flag)))) break;
+                            mbar_expect_tx_elected(&sh->x_full[kb], X_KB_BYTES);
+                            tma_load_2d_elected(x_base + (uint32_t)kb * X_KB_BYTES, &map_x, kb * KBLK, row0, &sh->x_full[kb]);
                             x_tile = lt;
                         }
                         const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
-                        if (!(ok = mbar_wait(&sh->c_empty[s], ph ^ 1u, abort_flag))) break;
-                        mbar_expect_tx(&sh->c_full[s], C_STAGE_BYTES);
-                        tma_load_2d(c_smem + (size_t)s * C_STAGE_BYTES, &map_c, kb * KBLK, nt * BN, &sh->c_full[s]);
+                        if (!(ok = __all_sync(FULL, mbar_wait(&sh->c_empty[s], ph ^ 1u, abort_flag)))) break;
+                        mbar_expect_tx_elected(&sh->c_full[s], C_STAGE_BYTES);
+                        tma_load_2d_elected(c_base + s * (uint32_t)C_STAGE_BYTES, &map_c, kb * KBLK, nt * BN, &sh->c_full[s]);
                     }
                 }
             }
-            if (!ok || *abort_flag) {
+            if (lane == 0 && (!ok || *abort_flag)) {
                 // On the way out after an abort: the loads already issued get time to land, so that nothing of this
                 // block's own still writes into its shared memory when it leaves.  (A k-block of x whose barrier is
                 // still in an earlier phase was not loaded for the last tile: the wait then runs to its limit.)
@@ -152,34 +154,33 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer: the whole warp runs the loop,
+        // one elected lane issues
+        {
             uint32_t it = 0, acc = 0;
             bool ok = true;
+            const uint32_t x_base = smem_u32(x_smem), c_base = smem_u32(c_smem);
+            static_assert(KBLK == 32, "umma_tf32_kblock_elected issues the four K-steps of a 32-float k-block");
             for (int64_t lt = 0, tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
                 for (int nt = 0; ok && nt < num_nt; ++nt, ++acc) {
                     const uint32_t buf = acc & 1u, use = (acc >> 1) & 1u;
-                    if (!(ok = mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag))) break;
+                    if (!(ok = __all_sync(FULL, mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag)))) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * BN;
                     for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                        if (nt == 0 && !(ok = mbar_wait(&sh->x_full[kb], (uint32_t)(lt & 1), abort_flag))) break;
+                        if (nt == 0 && !(ok = __all_sync(FULL, mbar_wait(&sh->x_full[kb], (uint32_t)(lt & 1), abort_flag)))) break;
                         const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
-                        if (!(ok = mbar_wait(&sh->c_full[s], ph, abort_flag))) break;
+                        if (!(ok = __all_sync(FULL, mbar_wait(&sh->c_full[s], ph, abort_flag)))) break;
                         tc_fence_after();
-                        const uint64_t adesc = umma_desc(smem_u32(x_smem + (size_t)kb * X_KB_BYTES));
-                        const uint64_t bdesc = umma_desc(smem_u32(c_smem + (size_t)s * C_STAGE_BYTES));
-#pragma unroll
-                        for (int ks = 0; ks < KBLK / 8; ++ks)   // 8 tf32 = 32 bytes per step: +2 in 16-byte units
-                            umma_tf32(d_tmem, adesc + (uint64_t)(2 * ks), bdesc + (uint64_t)(2 * ks), IDESC,
-                                      (kb | ks) != 0 ? 1u : 0u);
-                        umma_commit(&sh->c_empty[s]);
-                        if (nt == num_nt - 1) umma_commit(&sh->x_empty[kb]);
+                        umma_tf32_kblock_elected(d_tmem, umma_desc(x_base + (uint32_t)kb * X_KB_BYTES),
+                                                 umma_desc(c_base + s * (uint32_t)C_STAGE_BYTES), IDESC, (uint32_t)kb);
+                        umma_commit_elected(&sh->c_empty[s]);
+                        if (nt == num_nt - 1) umma_commit_elected(&sh->x_empty[kb]);
                     }
-                    if (ok) umma_commit(&sh->t_full[buf]);
+                    if (ok) umma_commit_elected(&sh->t_full[buf]);
                 }
             }
-            if (!ok || *abort_flag) {
+            if (lane == 0 && (!ok || *abort_flag)) {
                 // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
                 // here must have completed
                 umma_commit(&sh->drain);

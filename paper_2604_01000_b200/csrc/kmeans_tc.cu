@@ -180,11 +180,11 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     if (ok) umma_commit_elected(&sh->t_full[buf]);
                 }
             }
-            if (lane == 0 && (!ok || *abort_flag)) {
+            if (__any_sync(FULL, !ok || *abort_flag)) {
                 // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
-                // here must have completed
-                umma_commit(&sh->drain);
-                mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
+                // here must have completed (the commit comes from the lane that issued them: the same election)
+                umma_commit_elected(&sh->drain);
+                if (lane == 0) mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
             }
         }
     } else if (warp >= EPI_WARP0) {

@@ -498,11 +498,11 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                                              umma_desc(b_addr + (uint32_t)(kb * c_kb_bytes)), idesc, (uint32_t)kb);
                 umma_commit_elected(&sh->t_full[buf]);
             }
-            if (lane == 0 && (!ok || *abort_flag)) {
+            if (__any_sync(FULL, !ok || *abort_flag)) {
                 // after an abort the accumulators are given back at the end of the kernel: first every MMA issued
-                // here must have completed
-                umma_commit(&sh->drain);                  // only ever used once: the block leaves after an abort
-                mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
+                // here must have completed (the commit comes from the lane that issued them: the same election)
+                umma_commit_elected(&sh->drain);                  // only ever used once: the block leaves after an abort
+                if (lane == 0) mbar_wait_quiet(&sh->drain, 0u, DRAIN_LIMIT_CLOCKS);
             }
         }
     }

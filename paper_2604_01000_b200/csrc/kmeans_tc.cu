@@ -120,7 +120,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // ---------------------------------------------------------------- TMA producer: the whole warp runs the loop
         // (uniform control flow and operands), one elected lane issues (see the elected forms in tc_device.cuh)
         {
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, ph = 0;                        // centroid tiles issued; ring stage and phase of the next one
             bool ok = true;
             int64_t x_tile = -1;                                   // local index of the last tile any k-block was loaded for
             const uint32_t x_base = smem_u32(x_smem), c_base = smem_u32(c_smem);
@@ -134,10 +134,13 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             tma_load_2d_elected(x_base + (uint32_t)kb * X_KB_BYTES, &map_x, kb * KBLK, row0, &sh->x_full[kb]);
                             x_tile = lt;
                         }
-                        const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                         if (!(ok = __all_sync(FULL, mbar_wait(&sh->c_empty[s], ph ^ 1u, abort_flag)))) break;
                         mbar_expect_tx_elected(&sh->c_full[s], C_STAGE_BYTES);
                         tma_load_2d_elected(c_base + s * (uint32_t)C_STAGE_BYTES, &map_c, kb * KBLK, nt * BN, &sh->c_full[s]);
+                        if (++s == (uint32_t)stages) {             // (no division in the issue loops)
+                            s = 0;
+                            ph ^= 1u;
+                        }
                     }
                 }
             }
@@ -157,7 +160,7 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // ---------------------------------------------------------------- MMA issuer: the whole warp runs the loop,
         // one elected lane issues
         {
-            uint32_t it = 0, acc = 0;
+            uint32_t it = 0, acc = 0, s = 0, ph = 0;
             bool ok = true;
             const uint32_t x_base = smem_u32(x_smem), c_base = smem_u32(c_smem);
             static_assert(KBLK == 32, "umma_tf32_kblock_elected issues the four K-steps of a 32-float k-block");
@@ -169,13 +172,16 @@ kmeans_tc_screen(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     const uint32_t d_tmem = tmem_base + buf * BN;
                     for (int kb = 0; kb < num_kb; ++kb, ++it) {
                         if (nt == 0 && !(ok = __all_sync(FULL, mbar_wait(&sh->x_full[kb], (uint32_t)(lt & 1), abort_flag)))) break;
-                        const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
                         if (!(ok = __all_sync(FULL, mbar_wait(&sh->c_full[s], ph, abort_flag)))) break;
                         tc_fence_after();
                         umma_tf32_kblock_elected(d_tmem, umma_desc(x_base + (uint32_t)kb * X_KB_BYTES),
                                                  umma_desc(c_base + s * (uint32_t)C_STAGE_BYTES), IDESC, (uint32_t)kb);
                         umma_commit_elected(&sh->c_empty[s]);
                         if (nt == num_nt - 1) umma_commit_elected(&sh->x_empty[kb]);
+                        if (++s == (uint32_t)stages) {
+                            s = 0;
+                            ph ^= 1u;
+                        }
                     }
                     if (ok) umma_commit_elected(&sh->t_full[buf]);
                 }

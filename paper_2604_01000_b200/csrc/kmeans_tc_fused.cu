@@ -454,9 +454,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 #pragma unroll 1
             for (int kb = 0; kb < num_kb; ++kb)
                 tma_load_2d_elected(smem_u32(c_smem) + (uint32_t)(kb * c_kb_bytes), &map_c, kb * KBLK, 0, &sh->c_full);
-            uint32_t it = it_base;
-            for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-                const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
+            uint32_t it = it_base, s = 0, ph = 0;             // ring stage and phase of the next tile: counters, no division
+            for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it, ph ^= (++s == (uint32_t)stages), s = s == (uint32_t)stages ? 0u : s) {
                 if (!__all_sync(FULL, mbar_wait(&sh->x_empty[s], ph ^ 1u, abort_flag))) break;
                 mbar_expect_tx_elected(&sh->x_full[s], (uint32_t)stage_bytes);
                 const uint32_t dst = smem_u32(x_smem) + s * (uint32_t)stage_bytes;
@@ -482,9 +481,8 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // one elected lane issues (see the elected forms in tc_device.cuh)
         {
             bool ok = __all_sync(FULL, mbar_wait(&sh->c_full, ipar, abort_flag));
-            uint32_t it = it_base;
-            for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                const uint32_t s = it % (uint32_t)stages, ph = (it / (uint32_t)stages) & 1u;
+            uint32_t it = it_base, s = 0, ph = 0;
+            for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it, ph ^= (++s == (uint32_t)stages), s = s == (uint32_t)stages ? 0u : s) {
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
                 if (!(ok = __all_sync(FULL, mbar_wait(&sh->t_empty[buf], use ^ 1u, abort_flag)))) break;
                 if (!(ok = __all_sync(FULL, mbar_wait(&sh->x_full[s], ph, abort_flag)))) break;
@@ -752,14 +750,13 @@ kmeans_tc_fused(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int v = 0; v < VPL; ++v) acc[i][v] = make_float4(0.f, 0.f, 0.f, 0.f);
         bool planned = mbar_wait(&sh->plan_full, ipar, abort_flag);
         EP_CLK_DECL
-        uint32_t it = it_base;
-        for (int64_t tile = blockIdx.x; planned && tile < num_tiles; tile += gridDim.x, ++it) {
-            const uint32_t s = it % (uint32_t)stages;
+        uint32_t it = it_base, s = 0, ph = 0;
+        for (int64_t tile = blockIdx.x; planned && tile < num_tiles; tile += gridDim.x, ++it, ph ^= (++s == (uint32_t)stages), s = s == (uint32_t)stages ? 0u : s) {
             const uint32_t par = it & 1u, use = (it >> 1) & 1u;
             const uint8_t *xl = x_smem + (size_t)s * stage_bytes + (size_t)(lane >> 3) * X_KB_BYTES;   // this lane's first k-block
             EP_CLK(pc_work)
             if (!mbar_wait(&sh->ord_full[par], use, abort_flag)) break;
-            if (!mbar_wait(&sh->x_full[s], (it / (uint32_t)stages) & 1u, abort_flag)) break;   // long complete: makes the tile visible here
+            if (!mbar_wait(&sh->x_full[s], ph, abort_flag)) break;   // long complete: makes the tile visible here
             EP_CLK(pc_wait)
             // The rows of this warp's clusters are one stretch of order[], slot after slot; lane i holds where
             // slot i starts (lane OWN: where the stretch ends).

@@ -32,7 +32,7 @@ import synth  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries under profiles/;
 # the key carries the launch the capture covers.  Set an entry to None when its kernel changes.
 NCU_TRAFFIC = {
-    ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_285_287_000 + 611_309_312, "launch": "all rows, one iteration",
+    ("kmeans_assign_K4096", "cfg4"): {"bytes_per_launch": 1_283_199_000 + 610_001_664, "launch": "all rows, one iteration",
                                       "source": "profiles/kmeans_tc_screen_K4096_cfg4.md"},
     # one launch runs the call's 30 iterations: a thirtieth of its DRAM bytes per pass
     ("kmeans_assign_K32", "cfg4"): {"bytes_per_launch": (38_639_230_000 + 405_837_568) // 30,

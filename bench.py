@@ -454,6 +454,8 @@ def main():
             e["roofline"] = {"bound": "tensor", "achieved": tfs, "peak": tf32_peak, "unit": "TFLOP/s",
                              "frac": tfs / tf32_peak, "traffic": None, "peak_source": tf32_source}
         e["share_of_step"] = tot / ms
+        if clocks.get("sm_mhz"):      # latency-bound passes follow the SM clock, which the step's power draw sets
+            e["mclk_per_pass_at_median_sm_clock"] = tot / passes_timed * clocks["sm_mhz"] * 1e-3
         passes[name] = e
 
     S = args.steps
